@@ -1,0 +1,183 @@
+/*
+ * moe_pd.h -- C ABI of the phase-owned MoE layer for in-place prefill/decode multiplexing.
+ *
+ * The layer is the one prefill (P) and decode (D) both execute on shared devices:
+ *   route -> dispatch layout (counts, exclusive scan, stable permutation, row movement)
+ *         -> grouped SwiGLU expert FFN (+ shared expert) -> weighted combine.
+ * The paper's Section "DeepEP Communication-State Isolation" requires that everything a
+ * communication/layout kernel MODIFIES (buffers, counters, workspace, stream, events,
+ * D's double-buffer index) is owned by exactly one phase, while initialisation and the
+ * model weights are shared (Table "Ownership in the concurrent DeepEP runtime").  Here
+ * that is one `moe_ctx` per phase: two contexts never share a mutable byte, and the
+ * only memory reachable from both is the read-only weights the caller passes in.
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned,
+ *     dense row-major.  The library never frees or keeps them beyond the stream work
+ *     of the step they belong to.  Only `moe_layer_host` takes HOST pointers, and says so.
+ *   - Calls validate on the host, enqueue kernels on the context's stream and return.
+ *     They do not synchronise, allocate device memory or read device memory back
+ *     (except `moe_ctx_status`, `moe_ctx_destroy` and `moe_layer_host`, which say so).
+ *   - Every function returns a `moe_status`; no exception crosses the boundary.
+ *     `moe_last_error` gives a human-readable reason for the last failure on a context.
+ *   - Problems only the device can see (an expert index outside [0,E), a bounded wait
+ *     that ran out) make the kernel skip the offending work and record a code in the
+ *     context's device status word; nothing traps.  `moe_ctx_status` reads it.
+ *   - bf16 tensors are passed as `const void*` / `void*`.
+ *
+ * Per step, in order:  moe_route (optional) -> moe_dispatch_layout -> moe_grouped_ffn
+ * -> moe_combine.  Any other order returns MOE_ERR_STATE.
+ */
+#ifndef MOE_PD_H_
+#define MOE_PD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct moe_ctx moe_ctx; /* opaque; one per phase */
+
+/* Explicit phase identity: it selects state and kernel variant, and is never inferred
+ * from a host thread or a stream (Section "End-to-End Integration"). */
+typedef enum { MOE_PHASE_PREFILL = 0, MOE_PHASE_DECODE = 1 } moe_phase;
+
+typedef enum {
+  MOE_OK = 0,
+  MOE_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, bad shape                        */
+  MOE_ERR_CAPACITY = 2,    /* T > max_tokens, or workspace too small                      */
+  MOE_ERR_STATE = 3,       /* call out of order, overlapping workspaces, destroy while busy */
+  MOE_ERR_UNSUPPORTED = 4, /* shape outside what the kernels handle                       */
+  MOE_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed                           */
+  MOE_ERR_TIMEOUT = 6,     /* device: a bounded wait gave up                              */
+  MOE_ERR_BAD_INDEX = 7    /* device: an expert index was outside [0, E)                  */
+} moe_status;
+
+/* GEMM kernel variants.  AUTO follows the phase: large-M for P, small-M for D. */
+typedef enum {
+  MOE_GEMM_AUTO = 0,
+  MOE_GEMM_LARGE_M = 1,  /* tokens fill the 128-row MMA dimension; tensor-bound at prefill sizes */
+  MOE_GEMM_SMALL_M = 2,  /* swap-AB: weight rows fill the MMA M dimension, an expert's few tokens
+                            sit in N; streams the weights once -- HBM-bound by design          */
+  MOE_GEMM_VALIDATION = 3 /* plain CUDA-core kernel, slow; exists to localise tensor-core bugs   */
+} moe_gemm_variant;
+
+typedef struct {
+  int32_t hidden;       /* H, multiple of 64                                            */
+  int32_t n_experts;    /* E, 1..1024                                                   */
+  int32_t top_k;        /* k, 1..min(E,32)                                              */
+  int32_t inter;        /* I, routed expert intermediate size, multiple of 64           */
+  int32_t n_shared;     /* S in {0,1}: number of shared experts                         */
+  int32_t shared_inter; /* I_s, multiple of 64 (ignored when S = 0)                     */
+  int32_t max_tokens;   /* capacity; T of a call may be anything in [0, max_tokens]     */
+  int32_t phase;        /* moe_phase                                                    */
+  int32_t sm_budget;    /* 0 = all SMs; else the most CTAs a persistent kernel of this
+                           context may occupy (the analogue of the paper's separate
+                           communication-SM budgets per phase)                          */
+  int32_t gemm_variant; /* moe_gemm_variant                                             */
+  float routed_scale;   /* multiplies the routed weights; 1.0f unless the model says so */
+} moe_config;
+
+/* Bytes of device workspace `moe_ctx_create` needs for this configuration (0 on a bad config).
+ * A DECODE context holds two buffer sets, selected by a double-buffer index that flips at
+ * every moe_combine, so that its addresses stay stable across steps. */
+size_t moe_ctx_workspace_bytes(const moe_config* cfg);
+
+/* Creates a phase context bound to `cuda_stream` (a cudaStream_t; NULL = the legacy default
+ * stream) that owns [workspace, workspace + workspace_bytes) -- device memory the caller
+ * allocated (256-byte aligned) and keeps alive until moe_ctx_destroy.  The range is
+ * registered process-wide: a range overlapping a live context's, or a stream already bound
+ * to a live context of the other phase, is refused with MOE_ERR_STATE (construction
+ * validates isolation before any kernel runs).  Enqueues one memset on the stream. */
+moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                          moe_ctx** out);
+
+/* Destroys a context at a quiescent point.  If work may still be in flight on its stream
+ * it returns MOE_ERR_STATE and the context stays valid (an abandoned operation retires its
+ * buffer only at quiescent cleanup); otherwise it unregisters the workspace and frees the
+ * host object.  Device memory is the caller's and is not freed. */
+moe_status moe_ctx_destroy(moe_ctx* ctx);
+
+/* Synchronises the context's stream and returns the device status word (a moe_status:
+ * MOE_OK, MOE_ERR_TIMEOUT or MOE_ERR_BAD_INDEX) in *device_status, then clears it. */
+moe_status moe_ctx_status(moe_ctx* ctx, int32_t* device_status);
+
+/* Reason for the last non-OK return on this context (static storage inside the context;
+ * valid until the next call on it).  Never NULL.  With ctx == NULL: the reason for the
+ * last failed moe_ctx_create on this thread. */
+const char* moe_last_error(const moe_ctx* ctx);
+
+/* Stage a1 -- top-k routing over given router logits.
+ *   key[e]      = logits[t,e] + select_bias[e]  (one fp32 add; select_bias NULL: key = logits)
+ *   topk_idx[t] = the k experts of largest key, descending; equal keys (IEEE ==, so +0 and -0
+ *                 tie) go to the lower expert index
+ *   topk_w[t,j] = routed_scale * softmax over the k selected UNBIASED logits
+ * logits [T,E] fp32, select_bias [E] fp32 or NULL, topk_idx [T,k] int32, topk_w [T,k] fp32.
+ * Inputs must be finite; with NaN/Inf the selection is unspecified but still k distinct
+ * in-range indices.  T = 0 is a legal no-op. */
+moe_status moe_route(moe_ctx* ctx, const float* logits, const float* select_bias, int32_t T, int32_t* topk_idx,
+                     float* topk_w);
+
+/* Stages a2-a5 -- the local part of a dispatch: per-expert counts (the "receive counts"),
+ * their exclusive scan (the "tensor allocation"), the stable token-to-expert permutation and
+ * the routed row movement (Section "Exposing a Safe Prefill Boundary" lists these stages).
+ * With flat slot f = t*k + j and N = T*k:
+ *   counts[e]  = #{f : topk_idx[f] == e};   offsets[0] = 0, offsets[e+1] = offsets[e] + counts[e]
+ *   perm[p] = f and inv_perm[f] = p, where slots of one expert keep ascending f (stable)
+ *   x_perm[p,:] = x[perm[p] / k, :]   (bit copy into the context's workspace)
+ * topk_idx [T,k] int32 (the caller's own routing is welcome; moe_route is optional);
+ * x [T,H] bf16, or NULL to build the layout only (then moe_grouped_ffn is not allowed);
+ * counts [E], offsets [E+1], perm [N], inv_perm [N] int32 -- each may be NULL, in which
+ * case the context keeps that array privately.  Arrays the caller does pass must stay
+ * untouched until moe_combine of the same step has been enqueued.
+ * A slot whose index is outside [0,E) is dropped (inv_perm[f] = -1), the device status
+ * becomes MOE_ERR_BAD_INDEX, and the slot contributes nothing to the output.
+ * T = 0 zero-fills counts and offsets. */
+moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T, const void* x, int32_t* counts,
+                               int32_t* offsets, int32_t* perm, int32_t* inv_perm);
+
+/* Stages a6-a8 -- grouped SwiGLU expert FFN over the permuted rows, plus the shared expert:
+ *   act[p,i]    = silu(x_perm[p,:] . W_gate_up[e,i,:]) * (x_perm[p,:] . W_gate_up[e,I+i,:])
+ *   y_perm[p,c] = act[p,:] . W_down[e,c,:]          for p in expert e's segment
+ *   y_shared    = the same FFN with the shared weights on x[t,:] for every token (S = 1)
+ * bf16 operands, fp32 accumulation on the tensor cores, silu(z) = z / (1 + exp(-z)) in fp32;
+ * act, y_perm and y_shared are stored as bf16 (round to nearest even) in the workspace.
+ * w_gate_up [E,2I,H] bf16 (rows 0..I-1 gate, I..2I-1 up), w_down [E,H,I] bf16,
+ * ws_gate_up [2I_s,H], ws_down [H,I_s] bf16 (required iff S = 1), x [T,H] bf16 (read by the
+ * shared expert; required iff S = 1).  Weights are read-only and may be shared by contexts. */
+moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_down, const void* x,
+                           const void* ws_gate_up, const void* ws_down, int32_t T);
+
+/* Stage a9 -- weighted combine back to token order:
+ *   out[t,:] = sum_j topk_w[t,j] * y_perm[inv_perm[t*k+j],:]  (+ y_shared[t,:]),  fp32 sum, bf16 store.
+ * topk_w [T,k] fp32; inv_perm [N] int32 or NULL to use the layout of this step kept by the
+ * context; out [T,H] bf16.  Deterministic: fixed summation order, no atomics.
+ * Ends the step; a DECODE context then flips its double-buffer index. */
+moe_status moe_combine(moe_ctx* ctx, const float* topk_w, const int32_t* inv_perm, int32_t T, void* out);
+
+/* One whole step with HOST activations: copies logits_host [T,E] fp32 and x_host [T,H] bf16
+ * to the device (cudaMemcpyAsync into context-owned staging), runs a1..a9, copies out
+ * [T,H] bf16 back to out_host and synchronises the stream before returning.  Pinned host
+ * memory is recommended.  select_bias and all weights are DEVICE pointers as above. */
+moe_status moe_layer_host(moe_ctx* ctx, const float* logits_host, const float* select_bias, const void* x_host,
+                          int32_t T, const void* w_gate_up, const void* w_down, const void* ws_gate_up,
+                          const void* ws_down, void* out_host);
+
+/* Test/inspection only: device pointers into the context's CURRENT buffer set.  Rows
+ * [0, T*k) of x_perm [.,H], act [.,I], y_perm [.,H] and rows [0,T) of y_shared [.,H] are
+ * defined after the respective stage.  Any out-pointer may be NULL. */
+moe_status moe_ctx_debug_ptrs(moe_ctx* ctx, void** x_perm, void** act, void** y_perm, void** y_shared,
+                              int32_t** counts, int32_t** offsets);
+
+/* Kernels launched on this context since creation (for launch accounting in benchmarks). */
+int64_t moe_ctx_launch_count(const moe_ctx* ctx);
+
+/* Library version string, e.g. "moe_pd 0.1 (sm_100a)". */
+const char* moe_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_PD_H_ */

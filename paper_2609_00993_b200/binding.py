@@ -1,0 +1,258 @@
+"""Python binding of the C ABI in include/moe_pd.h -- argument marshalling only.
+
+Same names as the C entry points.  Tensors are torch CUDA tensors used for device memory and
+streams; every step of the layer runs in the library's kernels.  If the built library is missing
+the import of this module's functions fails loudly: there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmoe_pd.so")
+
+MOE_PHASE_PREFILL, MOE_PHASE_DECODE = 0, 1
+MOE_OK = 0
+MOE_ERR_INVALID_ARG, MOE_ERR_CAPACITY, MOE_ERR_STATE, MOE_ERR_UNSUPPORTED = 1, 2, 3, 4
+MOE_ERR_CUDA, MOE_ERR_TIMEOUT, MOE_ERR_BAD_INDEX = 5, 6, 7
+MOE_GEMM_AUTO, MOE_GEMM_LARGE_M, MOE_GEMM_SMALL_M, MOE_GEMM_VALIDATION = 0, 1, 2, 3
+
+STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_CAPACITY", 3: "MOE_ERR_STATE",
+                4: "MOE_ERR_UNSUPPORTED", 5: "MOE_ERR_CUDA", 6: "MOE_ERR_TIMEOUT", 7: "MOE_ERR_BAD_INDEX"}
+
+# every symbol include/moe_pd.h declares
+EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_destroy", "moe_ctx_status",
+           "moe_last_error", "moe_route", "moe_dispatch_layout", "moe_grouped_ffn", "moe_combine", "moe_layer_host",
+           "moe_ctx_debug_ptrs", "moe_ctx_launch_count")
+
+
+class moe_config(ctypes.Structure):
+    _fields_ = [("hidden", ctypes.c_int32), ("n_experts", ctypes.c_int32), ("top_k", ctypes.c_int32),
+                ("inter", ctypes.c_int32), ("n_shared", ctypes.c_int32), ("shared_inter", ctypes.c_int32),
+                ("max_tokens", ctypes.c_int32), ("phase", ctypes.c_int32), ("sm_budget", ctypes.c_int32),
+                ("gemm_variant", ctypes.c_int32), ("routed_scale", ctypes.c_float)]
+
+
+class MoeError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads libmoe_pd.so (built in-tree by paper_2609_00993_b200.build); raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_00993_b200.build` "
+                          "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    cfgp = ctypes.POINTER(moe_config)
+    lib.moe_version.restype = ctypes.c_char_p
+    lib.moe_version.argtypes = []
+    lib.moe_ctx_workspace_bytes.restype = sz
+    lib.moe_ctx_workspace_bytes.argtypes = [cfgp]
+    lib.moe_ctx_create.restype = i32
+    lib.moe_ctx_create.argtypes = [cfgp, vp, sz, vp, ctypes.POINTER(vp)]
+    lib.moe_ctx_destroy.restype = i32
+    lib.moe_ctx_destroy.argtypes = [vp]
+    lib.moe_ctx_status.restype = i32
+    lib.moe_ctx_status.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.moe_last_error.restype = ctypes.c_char_p
+    lib.moe_last_error.argtypes = [vp]
+    lib.moe_route.restype = i32
+    lib.moe_route.argtypes = [vp, vp, vp, i32, vp, vp]
+    lib.moe_dispatch_layout.restype = i32
+    lib.moe_dispatch_layout.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.moe_grouped_ffn.restype = i32
+    lib.moe_grouped_ffn.argtypes = [vp, vp, vp, vp, vp, vp, i32]
+    lib.moe_combine.restype = i32
+    lib.moe_combine.argtypes = [vp, vp, vp, i32, vp]
+    lib.moe_layer_host.restype = i32
+    lib.moe_layer_host.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.moe_ctx_debug_ptrs.restype = i32
+    lib.moe_ctx_debug_ptrs.argtypes = [vp] + [ctypes.POINTER(vp)] * 6
+    lib.moe_ctx_launch_count.restype = i64
+    lib.moe_ctx_launch_count.argtypes = [vp]
+    _lib = lib
+    return lib
+
+
+def moe_version() -> str:
+    return load_library().moe_version().decode()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _dev(t: Optional[torch.Tensor], dtype, name):
+    if t is None:
+        return
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}, got {t.dtype}")
+
+
+def make_config(hidden, n_experts, top_k, inter, shared_inter=0, max_tokens=1, phase=MOE_PHASE_PREFILL, sm_budget=0,
+                gemm_variant=MOE_GEMM_AUTO, routed_scale=1.0) -> moe_config:
+    return moe_config(hidden, n_experts, top_k, inter, 1 if shared_inter else 0, shared_inter, max_tokens, phase,
+                      sm_budget, gemm_variant, routed_scale)
+
+
+def moe_ctx_workspace_bytes(cfg: moe_config) -> int:
+    return int(load_library().moe_ctx_workspace_bytes(ctypes.byref(cfg)))
+
+
+class MoeContext:
+    """One phase context (`moe_ctx`).  The workspace is a torch allocation the context keeps alive;
+    `stream` is the torch CUDA stream all its calls enqueue on."""
+
+    def __init__(self, cfg: moe_config, stream: Optional[torch.cuda.Stream] = None, device="cuda",
+                 workspace: Optional[torch.Tensor] = None):
+        self.lib = load_library()
+        self.cfg = cfg
+        self.device = torch.device(device)
+        nbytes = moe_ctx_workspace_bytes(cfg)
+        if nbytes == 0:
+            raise MoeError(MOE_ERR_INVALID_ARG, "invalid configuration")
+        with torch.cuda.device(self.device):
+            self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+            self.workspace = workspace if workspace is not None else torch.empty(nbytes, dtype=torch.uint8,
+                                                                                 device=self.device)
+        self.workspace_bytes = nbytes
+        handle = ctypes.c_void_p()
+        st = self.lib.moe_ctx_create(ctypes.byref(cfg), ctypes.c_void_p(self.workspace.data_ptr()),
+                                     self.workspace.numel(), ctypes.c_void_p(self.stream.cuda_stream),
+                                     ctypes.byref(handle))
+        if st != MOE_OK:
+            raise MoeError(st, self.lib.moe_last_error(None).decode())
+        self.handle = handle
+
+    # -- plumbing
+    def _check(self, st: int):
+        if st != MOE_OK:
+            raise MoeError(st, self.lib.moe_last_error(self.handle).decode())
+
+    def destroy(self):
+        if self.handle is not None:
+            self._check(self.lib.moe_ctx_destroy(self.handle))
+            self.handle = None
+
+    def close(self):
+        """Drain the stream, then destroy."""
+        if self.handle is not None:
+            self.stream.synchronize()
+            self.destroy()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the C entry points, same names
+    def moe_ctx_status(self) -> int:
+        v = ctypes.c_int32(0)
+        self._check(self.lib.moe_ctx_status(self.handle, ctypes.byref(v)))
+        return int(v.value)
+
+    def moe_ctx_launch_count(self) -> int:
+        return int(self.lib.moe_ctx_launch_count(self.handle))
+
+    def moe_route(self, logits, select_bias, topk_idx, topk_w, T=None):
+        _dev(logits, torch.float32, "logits"); _dev(select_bias, torch.float32, "select_bias")
+        _dev(topk_idx, torch.int32, "topk_idx"); _dev(topk_w, torch.float32, "topk_w")
+        T = logits.shape[0] if T is None else T
+        self._check(self.lib.moe_route(self.handle, _ptr(logits), _ptr(select_bias), T, _ptr(topk_idx), _ptr(topk_w)))
+
+    def moe_dispatch_layout(self, topk_idx, x, counts=None, offsets=None, perm=None, inv_perm=None, T=None):
+        _dev(topk_idx, torch.int32, "topk_idx"); _dev(x, torch.bfloat16, "x")
+        for n, t in (("counts", counts), ("offsets", offsets), ("perm", perm), ("inv_perm", inv_perm)):
+            _dev(t, torch.int32, n)
+        T = topk_idx.shape[0] if T is None else T
+        self._check(self.lib.moe_dispatch_layout(self.handle, _ptr(topk_idx), T, _ptr(x), _ptr(counts), _ptr(offsets),
+                                                 _ptr(perm), _ptr(inv_perm)))
+
+    def moe_grouped_ffn(self, w_gate_up, w_down, x, ws_gate_up=None, ws_down=None, T=None):
+        for n, t in (("w_gate_up", w_gate_up), ("w_down", w_down), ("x", x), ("ws_gate_up", ws_gate_up),
+                     ("ws_down", ws_down)):
+            _dev(t, torch.bfloat16, n)
+        T = x.shape[0] if T is None else T
+        self._check(self.lib.moe_grouped_ffn(self.handle, _ptr(w_gate_up), _ptr(w_down), _ptr(x), _ptr(ws_gate_up),
+                                             _ptr(ws_down), T))
+
+    def moe_combine(self, topk_w, inv_perm, out, T=None):
+        _dev(topk_w, torch.float32, "topk_w"); _dev(inv_perm, torch.int32, "inv_perm"); _dev(out, torch.bfloat16, "out")
+        T = out.shape[0] if T is None else T
+        self._check(self.lib.moe_combine(self.handle, _ptr(topk_w), _ptr(inv_perm), T, _ptr(out)))
+
+    def moe_layer_host(self, logits_host, select_bias, x_host, w_gate_up, w_down, ws_gate_up, ws_down, out_host,
+                       T=None):
+        """logits_host / x_host / out_host are HOST tensors (pinned recommended); the rest are device tensors."""
+        for n, t in (("logits_host", logits_host), ("x_host", x_host), ("out_host", out_host)):
+            if t.is_cuda:
+                raise ValueError(f"{n} must be a host tensor")
+        T = x_host.shape[0] if T is None else T
+        self._check(self.lib.moe_layer_host(self.handle, _ptr(logits_host), _ptr(select_bias), _ptr(x_host), T,
+                                            _ptr(w_gate_up), _ptr(w_down), _ptr(ws_gate_up), _ptr(ws_down),
+                                            _ptr(out_host)))
+
+    def moe_ctx_debug_ptrs(self) -> dict:
+        """Views (no copies) of the workspace buffers of the step in progress / last finished step."""
+        ptrs = [ctypes.c_void_p() for _ in range(6)]
+        self._check(self.lib.moe_ctx_debug_ptrs(self.handle, *[ctypes.byref(p) for p in ptrs]))
+        c = self.cfg
+        N = c.max_tokens * c.top_k
+        base = self.workspace.data_ptr()
+
+        def view(p, rows, cols, dtype):
+            if not p.value or rows * cols == 0:
+                return None
+            esz = torch.empty(0, dtype=dtype).element_size()
+            off = p.value - base
+            return self.workspace[off:off + rows * cols * esz].view(dtype).view(rows, cols)
+
+        return {"x_perm": view(ptrs[0], N, c.hidden, torch.bfloat16), "act": view(ptrs[1], N, c.inter, torch.bfloat16),
+                "y_perm": view(ptrs[2], N, c.hidden, torch.bfloat16),
+                "y_shared": view(ptrs[3], c.max_tokens, c.hidden, torch.bfloat16) if c.n_shared else None,
+                "counts": view(ptrs[4], 1, c.n_experts, torch.int32), "offsets": view(ptrs[5], 1, c.n_experts + 1, torch.int32)}
+
+    # -- convenience: one whole step on device tensors (calls the four entry points in order)
+    def layer(self, x, logits, select_bias, w_gate_up, w_down, ws_gate_up=None, ws_down=None, out=None, bufs=None):
+        T, k, E = x.shape[0], self.cfg.top_k, self.cfg.n_experts
+        if bufs is None:
+            bufs = alloc_step_buffers(T, k, E, x.device)
+        if out is None:
+            out = torch.empty(T, self.cfg.hidden, dtype=torch.bfloat16, device=x.device)
+        self.moe_route(logits, select_bias, bufs["topk_idx"], bufs["topk_w"], T=T)
+        self.moe_dispatch_layout(bufs["topk_idx"], x, bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"],
+                                 T=T)
+        self.moe_grouped_ffn(w_gate_up, w_down, x, ws_gate_up, ws_down, T=T)
+        self.moe_combine(bufs["topk_w"], bufs["inv_perm"], out, T=T)
+        return out, bufs
+
+
+def alloc_step_buffers(T: int, k: int, E: int, device) -> dict:
+    """Caller-owned per-step arrays of the routing and layout stages."""
+    n = max(T * k, 4)
+    return {"topk_idx": torch.empty(n, dtype=torch.int32, device=device)[:T * k].view(T, k),
+            "topk_w": torch.empty(n, dtype=torch.float32, device=device)[:T * k].view(T, k),
+            "counts": torch.empty(E, dtype=torch.int32, device=device),
+            "offsets": torch.empty(E + 1, dtype=torch.int32, device=device),
+            "perm": torch.empty(n, dtype=torch.int32, device=device)[:T * k],
+            "inv_perm": torch.empty(n, dtype=torch.int32, device=device)[:T * k]}

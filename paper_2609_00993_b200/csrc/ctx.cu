@@ -1,0 +1,461 @@
+// C ABI (include/moe_pd.h): phase contexts, workspace carving, host-side validation, call ordering.
+// All compute is in the kernels behind kernels.h; this file only validates, carves and enqueues.
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "../../include/moe_pd.h"
+#include "kernels.h"
+
+namespace {
+
+enum StepState { ST_IDLE = 0, ST_ROUTED = 1, ST_LAID_OUT = 2, ST_LAYOUT_ONLY = 3, ST_FFN_DONE = 4 };
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// One buffer set: everything the kernels of one step write.
+struct BufferSet {
+  char* x_perm;      // bf16 [N,H]
+  char* act;         // bf16 [N,I]
+  char* y_perm;      // bf16 [N,H]
+  char* act_shared;  // bf16 [T,Is]
+  char* y_shared;    // bf16 [T,H]
+  int32_t* counts;   // [E]
+  int32_t* offsets;  // [E+1]
+  int32_t* perm;     // [N]
+  int32_t* inv_perm; // [N]
+  int32_t* topk_idx; // [N]   (host-input path)
+  float* topk_w;     // [N]
+  float* logits;     // [T,E] staging (host-input path)
+  char* x_stage;     // bf16 [T,H]
+  char* out_stage;   // bf16 [T,H]
+  int32_t* scan;     // layout scratch
+};
+
+struct Layout {
+  size_t set_bytes;    // bytes of one buffer set
+  size_t total_bytes;  // status block + all sets
+  int n_sets;
+};
+
+constexpr size_t kStatusBlock = 256;
+
+// Walks the carve of one buffer set; with base == nullptr it only measures.
+size_t carve_set(const moe_config& c, char* base, BufferSet* out) {
+  const size_t T = (size_t)c.max_tokens, N = T * (size_t)c.top_k, H = (size_t)c.hidden, I = (size_t)c.inter;
+  const size_t E = (size_t)c.n_experts, Is = c.n_shared ? (size_t)c.shared_inter : 0;
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> char* {
+    char* p = base ? base + off : nullptr;
+    off += align_up(bytes ? bytes : 1, 256);
+    return p;
+  };
+  BufferSet b;
+  b.x_perm = take(N * H * 2);
+  b.act = take(N * I * 2);
+  b.y_perm = take(N * H * 2);
+  b.act_shared = take(T * Is * 2);
+  b.y_shared = take(c.n_shared ? T * H * 2 : 0);
+  b.counts = reinterpret_cast<int32_t*>(take(E * 4));
+  b.offsets = reinterpret_cast<int32_t*>(take((E + 1) * 4));
+  b.perm = reinterpret_cast<int32_t*>(take(N * 4));
+  b.inv_perm = reinterpret_cast<int32_t*>(take(N * 4));
+  b.topk_idx = reinterpret_cast<int32_t*>(take(N * 4));
+  b.topk_w = reinterpret_cast<float*>(take(N * 4));
+  b.logits = reinterpret_cast<float*>(take(T * E * 4));
+  b.x_stage = take(T * H * 2);
+  b.out_stage = take(T * H * 2);
+  b.scan = reinterpret_cast<int32_t*>(take(moe::layout_scratch_ints((int64_t)N, (int)E) * 4));
+  if (out) *out = b;
+  return off;
+}
+
+const char* validate_config(const moe_config* c) {
+  if (!c) return "config is NULL";
+  if (c->hidden <= 0 || c->hidden % 64) return "hidden must be a positive multiple of 64";
+  if (c->inter <= 0 || c->inter % 64) return "inter must be a positive multiple of 64";
+  if (c->n_experts < 1 || c->n_experts > 1024) return "n_experts must be in 1..1024";
+  if (c->top_k < 1 || c->top_k > 32 || c->top_k > c->n_experts) return "top_k must be in 1..min(n_experts,32)";
+  if (c->n_shared < 0 || c->n_shared > 1) return "n_shared must be 0 or 1";
+  if (c->n_shared && (c->shared_inter <= 0 || c->shared_inter % 64)) return "shared_inter must be a positive multiple of 64";
+  if (c->max_tokens < 1) return "max_tokens must be >= 1";
+  if ((int64_t)c->max_tokens * c->top_k > (int64_t)1 << 30) return "max_tokens * top_k too large";
+  if (c->phase != MOE_PHASE_PREFILL && c->phase != MOE_PHASE_DECODE) return "phase must be MOE_PHASE_PREFILL or MOE_PHASE_DECODE";
+  if (c->sm_budget < 0) return "sm_budget must be >= 0";
+  if (c->gemm_variant < MOE_GEMM_AUTO || c->gemm_variant > MOE_GEMM_VALIDATION) return "unknown gemm_variant";
+  if (!(c->routed_scale == c->routed_scale)) return "routed_scale is NaN";
+  return nullptr;
+}
+
+Layout measure(const moe_config& c) {
+  Layout l;
+  l.n_sets = (c.phase == MOE_PHASE_DECODE) ? 2 : 1;
+  l.set_bytes = carve_set(c, nullptr, nullptr);
+  l.total_bytes = kStatusBlock + l.set_bytes * (size_t)l.n_sets;
+  return l;
+}
+
+thread_local char g_create_error[256] = "";
+
+}  // namespace
+
+struct moe_ctx {
+  moe_config cfg;
+  cudaStream_t stream;
+  char* ws;
+  size_t ws_bytes;
+  int device;
+  int n_sms;
+  int* status;  // device status word (first int of the status block)
+  BufferSet sets[2];
+  int n_sets;
+  int cur;  // double-buffer index (always 0 for a PREFILL context)
+  StepState state;
+  int T;  // tokens of the step in progress
+  // arrays of the step in progress (the caller's or the context's own)
+  int32_t* counts;
+  int32_t* offsets;
+  int32_t* perm;
+  int32_t* inv_perm;
+  cudaEvent_t done;  // recorded after the last enqueue of every call
+  int64_t launches;
+  char err[256];
+};
+
+namespace {
+
+std::mutex g_registry_mutex;
+std::vector<moe_ctx*> g_registry;
+
+moe_status fail(moe_ctx* ctx, moe_status st, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(ctx ? ctx->err : g_create_error, 256, fmt, ap);
+  va_end(ap);
+  return st;
+}
+
+moe_status cuda_fail(moe_ctx* ctx, cudaError_t e, const char* what) {
+  return fail(ctx, e == cudaErrorNotSupported ? MOE_ERR_UNSUPPORTED : MOE_ERR_CUDA, "%s: %s", what,
+              cudaGetErrorString(e));
+}
+
+bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+struct DeviceGuard {
+  int prev = -1;
+  explicit DeviceGuard(int dev) {
+    cudaGetDevice(&prev);
+    if (prev != dev) cudaSetDevice(dev);
+    else prev = -1;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+void mark(moe_ctx* ctx, int n) {
+  ctx->launches += n;
+  cudaEventRecord(ctx->done, ctx->stream);
+}
+
+int gemm_ctas(const moe_ctx* ctx) {
+  return (ctx->cfg.sm_budget > 0 && ctx->cfg.sm_budget < ctx->n_sms) ? ctx->cfg.sm_budget : ctx->n_sms;
+}
+
+// Token tile of the small-M variant: the smallest power of two >= T, within [16, 128].
+int small_m_tile(int T) {
+  int t = 16;
+  while (t < T && t < 128) t <<= 1;
+  return t;
+}
+
+cudaError_t run_gemm(moe_ctx* ctx, const moe::GemmProblem& p, int T, int* n) {
+  int variant = ctx->cfg.gemm_variant;
+  if (variant == MOE_GEMM_AUTO) variant = (ctx->cfg.phase == MOE_PHASE_DECODE) ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M;
+  if (variant == MOE_GEMM_VALIDATION) return moe::launch_gemm_validation(p, ctx->stream, n);
+  const bool swap = (variant == MOE_GEMM_SMALL_M);
+  return moe::launch_gemm_tc(p, swap, swap ? small_m_tile(T) : 128, gemm_ctas(ctx), ctx->status, ctx->stream, n);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* moe_version(void) { return "moe_pd 0.1 (sm_100a)"; }
+
+size_t moe_ctx_workspace_bytes(const moe_config* cfg) {
+  if (validate_config(cfg)) return 0;
+  return measure(*cfg).total_bytes;
+}
+
+moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                          moe_ctx** out) {
+  if (!out) return fail(nullptr, MOE_ERR_INVALID_ARG, "out is NULL");
+  *out = nullptr;
+  if (const char* why = validate_config(cfg)) return fail(nullptr, MOE_ERR_INVALID_ARG, "%s", why);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return fail(nullptr, MOE_ERR_INVALID_ARG, "workspace must be a 256-byte aligned device pointer");
+  const Layout l = measure(*cfg);
+  if (workspace_bytes < l.total_bytes)
+    return fail(nullptr, MOE_ERR_CAPACITY, "workspace has %zu bytes, %zu needed", workspace_bytes, l.total_bytes);
+
+  cudaPointerAttributes attr;
+  cudaError_t e = cudaPointerGetAttributes(&attr, workspace);
+  if (e != cudaSuccess || attr.type != cudaMemoryTypeDevice) {
+    (void)cudaGetLastError();
+    return fail(nullptr, MOE_ERR_INVALID_ARG, "workspace is not device memory");
+  }
+  const char* why = nullptr;
+  if (cfg->gemm_variant != MOE_GEMM_VALIDATION && !moe::gemm_tc_init(&why))
+    return fail(nullptr, MOE_ERR_UNSUPPORTED, "%s", why ? why : "tensor-map encoding unavailable");
+
+  moe_ctx* ctx = new (std::nothrow) moe_ctx();
+  if (!ctx) return fail(nullptr, MOE_ERR_CUDA, "host allocation failed");
+  ctx->cfg = *cfg;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  ctx->ws = static_cast<char*>(workspace);
+  ctx->ws_bytes = l.total_bytes;
+  ctx->device = attr.device;
+  ctx->n_sets = l.n_sets;
+  ctx->cur = 0;
+  ctx->state = ST_IDLE;
+  ctx->T = 0;
+  ctx->launches = 0;
+  ctx->err[0] = 0;
+  ctx->status = reinterpret_cast<int*>(ctx->ws);
+  for (int s = 0; s < l.n_sets; ++s) carve_set(*cfg, ctx->ws + kStatusBlock + (size_t)s * l.set_bytes, &ctx->sets[s]);
+
+  {
+    // Isolation is validated at construction: no two live contexts may share a mutable byte, and a
+    // stream serves contexts of one phase only.
+    std::lock_guard<std::mutex> lock(g_registry_mutex);
+    for (const moe_ctx* o : g_registry) {
+      if (o->device == ctx->device && ctx->ws < o->ws + o->ws_bytes && o->ws < ctx->ws + ctx->ws_bytes) {
+        delete ctx;
+        return fail(nullptr, MOE_ERR_STATE, "workspace overlaps the workspace of a live context");
+      }
+      if (o->device == ctx->device && o->stream == ctx->stream && o->cfg.phase != ctx->cfg.phase) {
+        delete ctx;
+        return fail(nullptr, MOE_ERR_STATE, "stream is already bound to a live context of the other phase");
+      }
+    }
+    g_registry.push_back(ctx);
+  }
+
+  DeviceGuard guard(ctx->device);
+  int sms = 0;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->done, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws, 0, kStatusBlock, ctx->stream);
+  if (e == cudaSuccess) e = cudaEventRecord(ctx->done, ctx->stream);
+  if (e != cudaSuccess) {
+    std::lock_guard<std::mutex> lock(g_registry_mutex);
+    for (size_t i = 0; i < g_registry.size(); ++i)
+      if (g_registry[i] == ctx) g_registry.erase(g_registry.begin() + i);
+    moe_status st = cuda_fail(nullptr, e, "context set-up");
+    delete ctx;
+    return st;
+  }
+  ctx->n_sms = sms;
+  *out = ctx;
+  return MOE_OK;
+}
+
+moe_status moe_ctx_destroy(moe_ctx* ctx) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaError_t q = cudaEventQuery(ctx->done);
+  if (q == cudaErrorNotReady) return fail(ctx, MOE_ERR_STATE, "work is still in flight on the context's stream");
+  if (q != cudaSuccess) (void)cudaGetLastError();
+  {
+    std::lock_guard<std::mutex> lock(g_registry_mutex);
+    for (size_t i = 0; i < g_registry.size(); ++i)
+      if (g_registry[i] == ctx) {
+        g_registry.erase(g_registry.begin() + i);
+        break;
+      }
+  }
+  cudaEventDestroy(ctx->done);
+  delete ctx;
+  return MOE_OK;
+}
+
+moe_status moe_ctx_status(moe_ctx* ctx, int32_t* device_status) {
+  if (!ctx || !device_status) return MOE_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  int32_t v = 0;
+  cudaError_t e = cudaMemcpyAsync(&v, ctx->status, sizeof v, cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, sizeof(int), ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_ctx_status");
+  *device_status = v;
+  return MOE_OK;
+}
+
+const char* moe_last_error(const moe_ctx* ctx) { return ctx ? ctx->err : g_create_error; }
+
+int64_t moe_ctx_launch_count(const moe_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+moe_status moe_route(moe_ctx* ctx, const float* logits, const float* select_bias, int32_t T, int32_t* topk_idx,
+                     float* topk_w) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->state != ST_IDLE && ctx->state != ST_ROUTED)
+    return fail(ctx, MOE_ERR_STATE, "moe_route called in the middle of a step");
+  if (T < 0) return fail(ctx, MOE_ERR_INVALID_ARG, "T < 0");
+  if (T > ctx->cfg.max_tokens) return fail(ctx, MOE_ERR_CAPACITY, "T = %d exceeds max_tokens = %d", T, ctx->cfg.max_tokens);
+  if (T > 0 && (!logits || !topk_idx || !topk_w)) return fail(ctx, MOE_ERR_INVALID_ARG, "NULL pointer");
+  if (misaligned(logits) || misaligned(select_bias) || misaligned(topk_idx) || misaligned(topk_w))
+    return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+  DeviceGuard guard(ctx->device);
+  int n = 0;
+  cudaError_t e = moe::launch_route(logits, select_bias, T, ctx->cfg.n_experts, ctx->cfg.top_k, ctx->cfg.routed_scale,
+                                    topk_idx, topk_w, ctx->stream, &n);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_route");
+  ctx->state = ST_ROUTED;
+  mark(ctx, n);
+  return MOE_OK;
+}
+
+moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T, const void* x, int32_t* counts,
+                               int32_t* offsets, int32_t* perm, int32_t* inv_perm) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->state != ST_IDLE && ctx->state != ST_ROUTED && ctx->state != ST_LAYOUT_ONLY)
+    return fail(ctx, MOE_ERR_STATE, "moe_dispatch_layout called in the middle of a step");
+  if (T < 0) return fail(ctx, MOE_ERR_INVALID_ARG, "T < 0");
+  if (T > ctx->cfg.max_tokens) return fail(ctx, MOE_ERR_CAPACITY, "T = %d exceeds max_tokens = %d", T, ctx->cfg.max_tokens);
+  if (T > 0 && !topk_idx) return fail(ctx, MOE_ERR_INVALID_ARG, "topk_idx is NULL");
+  if (misaligned(topk_idx) || misaligned(x) || misaligned(counts) || misaligned(offsets) || misaligned(perm) ||
+      misaligned(inv_perm))
+    return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+  DeviceGuard guard(ctx->device);
+  BufferSet& b = ctx->sets[ctx->cur];
+  ctx->counts = counts ? counts : b.counts;
+  ctx->offsets = offsets ? offsets : b.offsets;
+  ctx->perm = perm ? perm : b.perm;
+  ctx->inv_perm = inv_perm ? inv_perm : b.inv_perm;
+  int n = 0;
+  cudaError_t e = moe::launch_layout(topk_idx, (int64_t)T * ctx->cfg.top_k, ctx->cfg.n_experts, ctx->counts,
+                                     ctx->offsets, ctx->perm, ctx->inv_perm, b.scan, ctx->status, ctx->stream, &n);
+  if (e == cudaSuccess && x != nullptr)
+    e = moe::launch_permute(x, ctx->inv_perm, b.x_perm, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->stream, &n);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_dispatch_layout");
+  ctx->T = T;
+  ctx->state = x ? ST_LAID_OUT : ST_LAYOUT_ONLY;
+  mark(ctx, n);
+  return MOE_OK;
+}
+
+moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_down, const void* x,
+                           const void* ws_gate_up, const void* ws_down, int32_t T) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->state != ST_LAID_OUT)
+    return fail(ctx, MOE_ERR_STATE, "moe_grouped_ffn needs a moe_dispatch_layout with x in the same step");
+  if (T != ctx->T) return fail(ctx, MOE_ERR_INVALID_ARG, "T = %d differs from the layout's T = %d", T, ctx->T);
+  if (!w_gate_up || !w_down) return fail(ctx, MOE_ERR_INVALID_ARG, "routed weights are NULL");
+  const bool shared = ctx->cfg.n_shared != 0;
+  if (shared && (!ws_gate_up || !ws_down || (!x && T > 0)))
+    return fail(ctx, MOE_ERR_INVALID_ARG, "the shared expert needs ws_gate_up, ws_down and x");
+  if (misaligned(w_gate_up) || misaligned(w_down) || misaligned(x) || misaligned(ws_gate_up) || misaligned(ws_down))
+    return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+  DeviceGuard guard(ctx->device);
+  BufferSet& b = ctx->sets[ctx->cur];
+  const moe_config& c = ctx->cfg;
+  const int64_t N = (int64_t)T * c.top_k, Ncap = (int64_t)c.max_tokens * c.top_k;
+  int n = 0;
+  cudaError_t e = cudaSuccess;
+  if (T > 0) {
+    moe::GemmProblem g1{b.x_perm, w_gate_up, b.act, ctx->offsets, 0, Ncap, N, c.n_experts, c.inter, c.hidden, true};
+    e = run_gemm(ctx, g1, T, &n);
+    if (e == cudaSuccess) {
+      moe::GemmProblem g2{b.act, w_down, b.y_perm, ctx->offsets, 0, Ncap, N, c.n_experts, c.hidden, c.inter, false};
+      e = run_gemm(ctx, g2, T, &n);
+    }
+    if (e == cudaSuccess && shared) {
+      moe::GemmProblem s1{x, ws_gate_up, b.act_shared, nullptr, T, T, T, 1, c.shared_inter, c.hidden, true};
+      e = run_gemm(ctx, s1, T, &n);
+      if (e == cudaSuccess) {
+        moe::GemmProblem s2{b.act_shared, ws_down, b.y_shared, nullptr, T, T, T, 1, c.hidden, c.shared_inter, false};
+        e = run_gemm(ctx, s2, T, &n);
+      }
+    }
+  }
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_grouped_ffn");
+  ctx->state = ST_FFN_DONE;
+  mark(ctx, n);
+  return MOE_OK;
+}
+
+moe_status moe_combine(moe_ctx* ctx, const float* topk_w, const int32_t* inv_perm, int32_t T, void* out) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->state != ST_FFN_DONE) return fail(ctx, MOE_ERR_STATE, "moe_combine needs moe_grouped_ffn in the same step");
+  if (T != ctx->T) return fail(ctx, MOE_ERR_INVALID_ARG, "T = %d differs from the layout's T = %d", T, ctx->T);
+  if (T > 0 && (!topk_w || !out)) return fail(ctx, MOE_ERR_INVALID_ARG, "NULL pointer");
+  if (misaligned(topk_w) || misaligned(inv_perm) || misaligned(out))
+    return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+  DeviceGuard guard(ctx->device);
+  BufferSet& b = ctx->sets[ctx->cur];
+  int n = 0;
+  cudaError_t e = moe::launch_combine(b.y_perm, ctx->cfg.n_shared ? b.y_shared : nullptr,
+                                      inv_perm ? inv_perm : ctx->inv_perm, topk_w, out, T, ctx->cfg.top_k,
+                                      ctx->cfg.hidden, ctx->stream, &n);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_combine");
+  ctx->state = ST_IDLE;
+  if (ctx->n_sets == 2) ctx->cur ^= 1;  // D: the next step works in the other buffer set
+  mark(ctx, n);
+  return MOE_OK;
+}
+
+moe_status moe_layer_host(moe_ctx* ctx, const float* logits_host, const float* select_bias, const void* x_host,
+                          int32_t T, const void* w_gate_up, const void* w_down, const void* ws_gate_up,
+                          const void* ws_down, void* out_host) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->state != ST_IDLE) return fail(ctx, MOE_ERR_STATE, "moe_layer_host called in the middle of a step");
+  if (T < 0) return fail(ctx, MOE_ERR_INVALID_ARG, "T < 0");
+  if (T > ctx->cfg.max_tokens) return fail(ctx, MOE_ERR_CAPACITY, "T = %d exceeds max_tokens = %d", T, ctx->cfg.max_tokens);
+  if (T > 0 && (!logits_host || !x_host || !out_host)) return fail(ctx, MOE_ERR_INVALID_ARG, "NULL host pointer");
+  DeviceGuard guard(ctx->device);
+  BufferSet& b = ctx->sets[ctx->cur];
+  const moe_config& c = ctx->cfg;
+  const size_t x_bytes = (size_t)T * c.hidden * 2;
+  cudaError_t e = cudaSuccess;
+  if (T > 0) {
+    e = cudaMemcpyAsync(b.logits, logits_host, (size_t)T * c.n_experts * 4, cudaMemcpyHostToDevice, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(b.x_stage, x_host, x_bytes, cudaMemcpyHostToDevice, ctx->stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "host-to-device copy");
+  }
+  moe_status st = moe_route(ctx, b.logits, select_bias, T, b.topk_idx, b.topk_w);
+  if (st == MOE_OK) st = moe_dispatch_layout(ctx, b.topk_idx, T, b.x_stage, nullptr, nullptr, nullptr, nullptr);
+  if (st == MOE_OK) st = moe_grouped_ffn(ctx, w_gate_up, w_down, b.x_stage, ws_gate_up, ws_down, T);
+  if (st == MOE_OK) st = moe_combine(ctx, b.topk_w, nullptr, T, b.out_stage);
+  if (st != MOE_OK) {
+    ctx->state = ST_IDLE;
+    return st;
+  }
+  if (T > 0) e = cudaMemcpyAsync(out_host, b.out_stage, x_bytes, cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "device-to-host copy");
+  return MOE_OK;
+}
+
+moe_status moe_ctx_debug_ptrs(moe_ctx* ctx, void** x_perm, void** act, void** y_perm, void** y_shared,
+                              int32_t** counts, int32_t** offsets) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  // after moe_combine a DECODE context has already flipped; report the set the last step used
+  const int set = (ctx->n_sets == 2 && ctx->state == ST_IDLE) ? (ctx->cur ^ 1) : ctx->cur;
+  BufferSet& b = ctx->sets[set];
+  if (x_perm) *x_perm = b.x_perm;
+  if (act) *act = b.act;
+  if (y_perm) *y_perm = b.y_perm;
+  if (y_shared) *y_shared = b.y_shared;
+  if (counts) *counts = b.counts;
+  if (offsets) *offsets = b.offsets;
+  return MOE_OK;
+}
+
+}  // extern "C"

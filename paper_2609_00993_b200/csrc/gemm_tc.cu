@@ -1,0 +1,536 @@
+// Stages a6-a8: grouped expert GEMM on the 5th-generation tensor cores (sm_100a).
+//
+//   operands   bf16, K-major, staged in shared memory by TMA (128-byte swizzle), 64 K-elements per stage
+//   math       tcgen05.mma (kind::f16, M=128) issued by one thread, fp32 accumulators in TMEM
+//   epilogue   tcgen05.ld -> registers -> (SwiGLU) -> bf16 -> global, overlapped with the next tile's MMAs
+//              through two TMEM accumulator stages
+//   schedule   persistent CTAs walk the tile list (expert, row tile, feature tile); the list is derived
+//              on the device from the expert offsets, so no host synchronisation is needed
+//
+// Two variants of the same kernel:
+//   large-M (prefill)  tokens fill the MMA M dimension (128 rows); a stage's weight tile is 256 rows
+//                      (gated: 128 gate rows + the matching 128 up rows), one N=256 MMA per 16 K-elements.
+//   small-M (decode)   swap-AB: 128 weight rows fill M, the expert's tokens sit in N (16..128, chosen per
+//                      tile from the expert's row count), two MMAs per 16 K-elements (one per weight box).
+//                      Each weight byte is read once: the variant is HBM-bound by design.
+// An expert's row tile may run past the end of its segment: TMA needs no alignment on the row coordinate, so
+// segments are NOT padded; rows that belong to the next expert are computed and simply not stored.
+//
+// Warp roles (192 threads): warps 0-3 epilogue (TMEM lanes 32w..32w+31), warp 4 TMA producer, warp 5 MMA
+// issuer and TMEM owner.  Every mbarrier wait is bounded: on expiry the kernel records a timeout in the
+// status word, raises a CTA-wide abort flag, lets copies in flight land, frees its TMEM and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+
+namespace moe {
+namespace {
+
+constexpr int kBlockK = 64;          // K elements per pipeline stage (128 bytes: one swizzle row)
+constexpr int kUmmaK = 16;           // K elements per tcgen05.mma
+constexpr int kWBoxRows = 128;       // weight rows per TMA box
+constexpr int kWBoxBytes = kWBoxRows * kBlockK * 2;  // 16 KB
+constexpr int kThreads = 192;
+constexpr int kEpilogueWarps = 4;
+constexpr int kProducerWarp = 4;
+constexpr int kMmaWarp = 5;
+constexpr int kMaxStages = 8;
+constexpr int kSmemBudget = 227 * 1024;
+constexpr uint32_t kSpinLimit = 1u << 22;
+
+struct TcParams {
+  const int32_t* offsets;  // [E+1] or nullptr (single group of fixed_rows rows)
+  int32_t fixed_rows;
+  int32_t E;
+  int32_t n_feat;          // output features (I for the gated pass, H for the down pass)
+  int32_t K;
+  __nv_bfloat16* out;      // [rows, n_feat]
+  int32_t row_tile;        // tokens per tile: 128 (large-M) or 16..128 (small-M)
+  int32_t n_stages;
+  int32_t x_tile_bytes;    // row_tile * 128
+  int* status;
+};
+
+// ---------------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Bounded wait.  Returns false if the limit ran out or another role of this CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (i >= 256u) {
+      if ((i & 255u) == 0u && *abort_flag) return false;
+      __nanosleep(64);
+    }
+  }
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, both operands K-major bf16, fp32 accumulate.
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The mbarrier gets one arrival when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows written by TMA with the 128-byte swizzle;
+// 8-row groups are 1024 bytes apart (stride byte offset), the leading byte offset is unused for this layout.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+         (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, dense, M x N.
+__device__ __forceinline__ uint32_t umma_idesc(uint32_t M, uint32_t N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+struct Tile {
+  int e, row0, rows, ft;
+};
+
+// tile -> (expert, first row, valid rows, feature tile).  prefix[e] = row tiles of experts < e.
+__device__ __forceinline__ Tile decode_tile(int tile, int n_ft, int E, const int* prefix, const int* seg,
+                                            int row_tile) {
+  const int rt = tile / n_ft;
+  int lo = 0, hi = E;  // largest e in [0,E) with prefix[e] <= rt
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (prefix[mid] <= rt) lo = mid; else hi = mid;
+  }
+  Tile t;
+  t.e = lo;
+  t.ft = tile - rt * n_ft;
+  const int mt = rt - prefix[lo];
+  t.row0 = seg[lo] + mt * row_tile;
+  t.rows = min(row_tile, seg[lo + 1] - t.row0);
+  return t;
+}
+
+// ------------------------------------------------------------------------------------- the kernel
+template <bool SWAP, bool GATED>
+__global__ void __launch_bounds__(kThreads, 1)
+grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                       const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // carve: [stages: W box0 | W box1 | X tile] | barriers | tmem slot | abort | prefix[E+1] | seg[E+1]
+  const uint32_t raw_addr = smem_u32(smem_raw);
+  const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
+  uint8_t* base = smem_raw + (base_addr - raw_addr);
+  const int stage_bytes = 2 * kWBoxBytes + p.x_tile_bytes;
+  uint8_t* after = base + (size_t)p.n_stages * stage_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(after);  // full[S], empty[S], tmem_full[2], tmem_empty[2]
+  const uint32_t bar_full = smem_u32(bars);
+  const uint32_t bar_empty = bar_full + 8u * p.n_stages;
+  const uint32_t bar_tfull = bar_empty + 8u * p.n_stages;
+  const uint32_t bar_tempty = bar_tfull + 16u;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* prefix = reinterpret_cast<int*>(tmem_slot + 2);
+  int* seg = prefix + (p.E + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int kFeatPerTile = GATED ? 128 : 256;
+  const int n_ft = (p.n_feat + kFeatPerTile - 1) / kFeatPerTile;
+  const int num_kb = (p.K + kBlockK - 1) / kBlockK;
+  const uint32_t acc_cols = SWAP ? 2u * (uint32_t)p.row_tile : 256u;  // TMEM columns per accumulator stage
+  uint32_t tmem_cols = 32;
+  while (tmem_cols < 2u * acc_cols) tmem_cols <<= 1;
+
+  // ---- set-up: tile list, barriers, TMEM
+  if (warp == 0) {
+    int carry = 0;
+    for (int b = 0; b < p.E; b += 32) {
+      const int e = b + lane;
+      int beg = 0, cnt = 0;
+      if (e < p.E) {
+        beg = p.offsets ? p.offsets[e] : 0;
+        cnt = p.offsets ? p.offsets[e + 1] - beg : p.fixed_rows;
+        if (cnt < 0) cnt = 0;
+        seg[e] = beg;
+        if (e == p.E - 1) seg[p.E] = beg + cnt;
+      }
+      const int tiles = (cnt + p.row_tile - 1) / p.row_tile;
+      int incl = tiles;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += n;
+      }
+      if (e < p.E) prefix[e] = carry + incl - tiles;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) prefix[p.E] = carry;
+  }
+  if (threadIdx.x == 32) {
+    for (int s = 0; s < p.n_stages; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8u * a, 1);
+      mbar_init(bar_tempty + 8u * a, kEpilogueWarps);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int total_tiles = prefix[p.E] * n_ft;
+
+  if (warp == kProducerWarp) {
+    // ================================================================= TMA producer (one lane)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, p.row_tile);
+        const int w_row0 = t.ft * kFeatPerTile;
+        const int w_row1 = GATED ? p.n_feat + t.ft * kFeatPerTile : w_row0 + kWBoxRows;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const uint32_t s = it % (uint32_t)p.n_stages, ph = (it / (uint32_t)p.n_stages) & 1u;
+          if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t full = bar_full + 8u * s;
+          const uint32_t st = base_addr + s * (uint32_t)stage_bytes;
+          mbar_expect_tx(full, (uint32_t)stage_bytes);
+          tma_load_3d(st, &map_w, full, kb * kBlockK, w_row0, t.e);
+          tma_load_3d(st + kWBoxBytes, &map_w, full, kb * kBlockK, w_row1, t.e);
+          tma_load_2d(st + 2 * kWBoxBytes, &map_x, full, kb * kBlockK, t.row0);
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicCAS(p.status, kStOk, kStTimeout);
+      }
+    }
+  } else if (warp == kMmaWarp) {
+    // ================================================================= MMA issuer (one lane)
+    if (lane == 0) {
+      uint32_t it = 0, tile_iter = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_iter) {
+        const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, p.row_tile);
+        const uint32_t as = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
+        if (!mbar_wait(bar_tempty + 8u * as, aph ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d0 = tmem_base + as * acc_cols;
+        // small-M: the MMA N covers only the rows this tile really has, rounded up to 16
+        const uint32_t n_swap = (uint32_t)min(p.row_tile, (t.rows + 15) & ~15);
+        const uint32_t idesc = SWAP ? umma_idesc(128, n_swap) : umma_idesc(128, 256);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const uint32_t s = it % (uint32_t)p.n_stages, ph = (it / (uint32_t)p.n_stages) & 1u;
+          if (!mbar_wait(bar_full + 8u * s, ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t st = base_addr + s * (uint32_t)stage_bytes;
+          const uint64_t dw0 = umma_smem_desc(st);
+          const uint64_t dw1 = umma_smem_desc(st + kWBoxBytes);
+          const uint64_t dx = umma_smem_desc(st + 2 * kWBoxBytes);
+#pragma unroll
+          for (int kk = 0; kk < kBlockK / kUmmaK; ++kk) {
+            const uint64_t adv = (uint64_t)((kk * kUmmaK * 2) >> 4);  // +32 bytes per K step, in 16-byte units
+            const uint32_t acc = (kb | kk) != 0 ? 1u : 0u;
+            if (SWAP) {
+              umma_bf16(d0, dw0 + adv, dx + adv, idesc, acc);
+              umma_bf16(d0 + (uint32_t)p.row_tile, dw1 + adv, dx + adv, idesc, acc);
+            } else {
+              umma_bf16(d0, dx + adv, dw0 + adv, idesc, acc);  // the two weight boxes are contiguous: N = 256
+            }
+          }
+          umma_commit(bar_empty + 8u * s);  // the stage is free once these MMAs have read it
+        }
+        if (ok) umma_commit(bar_tfull + 8u * as);  // accumulator complete
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicCAS(p.status, kStOk, kStTimeout);
+      }
+    }
+  } else {
+    // ================================================================= epilogue (warps 0-3)
+    uint32_t tile_iter = 0;
+    bool ok = true;
+    const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_iter) {
+      const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, p.row_tile);
+      const uint32_t as = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
+      if (!mbar_wait(bar_tfull + 8u * as, aph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t d0 = tmem_base + as * acc_cols + lane_base;
+      if (SWAP) {
+        // lane = weight row (output feature), column = token
+        const int fl = warp * 32 + lane;
+        const int f_a = t.ft * kFeatPerTile + fl;                 // box 0 feature
+        const int f_b = f_a + kWBoxRows;                          // box 1 feature (down pass only)
+        for (int c = 0; c < t.rows; c += 16) {
+          uint32_t ra[16], rb[16];
+          tmem_ld16(d0 + (uint32_t)c, ra);
+          tmem_ld16(d0 + (uint32_t)(p.row_tile + c), rb);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            if (c + i < t.rows) {
+              __nv_bfloat16* orow = p.out + (size_t)(t.row0 + c + i) * p.n_feat;
+              const float a = __uint_as_float(ra[i]), b = __uint_as_float(rb[i]);
+              if (GATED) {
+                if (f_a < p.n_feat) orow[f_a] = __float2bfloat16_rn(silu_mul(a, b));
+              } else {
+                if (f_a < p.n_feat) orow[f_a] = __float2bfloat16_rn(a);
+                if (f_b < p.n_feat) orow[f_b] = __float2bfloat16_rn(b);
+              }
+            }
+          }
+        }
+      } else {
+        // lane = token row, column = output feature
+        const int r = warp * 32 + lane;
+        const bool row_ok = r < t.rows;
+        __nv_bfloat16* orow = p.out + (size_t)(t.row0 + r) * p.n_feat + (size_t)t.ft * kFeatPerTile;
+        constexpr int kChunks = kFeatPerTile / 32;
+        for (int c = 0; c < kChunks; ++c) {
+          const int f0 = t.ft * kFeatPerTile + c * 32;
+          if (f0 >= p.n_feat) break;  // uniform across the CTA
+          uint32_t ra[32];
+          uint32_t packed[16];
+          tmem_ld32(d0 + (uint32_t)(c * 32), ra);
+          if (GATED) {
+            uint32_t rb[32];
+            tmem_ld32(d0 + (uint32_t)(128 + c * 32), rb);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              packed[i] = pack_bf16(silu_mul(__uint_as_float(ra[2 * i]), __uint_as_float(rb[2 * i])),
+                                    silu_mul(__uint_as_float(ra[2 * i + 1]), __uint_as_float(rb[2 * i + 1])));
+          } else {
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) packed[i] = pack_bf16(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1]));
+          }
+          if (row_ok) {
+            uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              if (f0 + q * 8 < p.n_feat)
+                dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8u * as);
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      atomicCAS(p.status, kStOk, kStTimeout);
+    }
+  }
+
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // give copies still in flight time to land in this CTA's shared memory before it is released
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == kMmaWarp) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, tmem_cols);
+  }
+}
+
+// --------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+const char* g_init_error = nullptr;
+
+bool encode_map(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                const uint32_t* box) {
+  cuuint64_t gdim[3];
+  cuuint64_t gstr[2];
+  cuuint32_t bdim[3];
+  cuuint32_t estr[3] = {1, 1, 1};
+  for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bdim[i] = box[i]; }
+  for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
+  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr,
+                        bdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <bool SWAP, bool GATED>
+cudaError_t launch_variant(const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& prm, int grid, size_t smem,
+                           cudaStream_t stream) {
+  auto kern = grouped_gemm_tc_kernel<SWAP, GATED>;
+  cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  kern<<<grid, kThreads, smem, stream>>>(mx, mw, prm);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool gemm_tc_init(const char** why) {
+  if (g_encode != nullptr) return true;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t err = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (err != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess) {
+    g_init_error = "cuTensorMapEncodeTiled is not available from the installed driver";
+    if (why) *why = g_init_error;
+    (void)cudaGetLastError();
+    return false;
+  }
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return true;
+}
+
+cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int max_ctas, int* status,
+                           cudaStream_t stream, int* n_launches) {
+  if (p.rows_bound <= 0) return cudaSuccess;
+  if (g_encode == nullptr && !gemm_tc_init(nullptr)) return cudaErrorNotSupported;
+  if (p.K % 8 != 0 || p.n_feat % 8 != 0 || p.E < 1 || p.E > 1024) return cudaErrorNotSupported;
+  if (!swap_ab) row_tile = 128;
+  if (row_tile < 16 || row_tile > 128 || (row_tile & (row_tile - 1)) != 0) return cudaErrorNotSupported;
+  if (p.rows_bound > 0x7fffffffLL / 2) return cudaErrorNotSupported;
+
+  const int groups = p.offsets ? p.E : 1;
+  const uint64_t w_rows = (uint64_t)(p.gated ? 2 : 1) * (uint64_t)p.n_feat;
+  CUtensorMap mx, mw;
+  {
+    const uint64_t dims[2] = {(uint64_t)p.K, (uint64_t)p.rows_bound};
+    const uint64_t str[1] = {(uint64_t)p.K * 2};
+    const uint32_t box[2] = {(uint32_t)kBlockK, (uint32_t)row_tile};
+    if (!encode_map(&mx, p.A, 2, dims, str, box)) return cudaErrorInvalidValue;
+  }
+  {
+    const uint64_t dims[3] = {(uint64_t)p.K, w_rows, (uint64_t)groups};
+    const uint64_t str[2] = {(uint64_t)p.K * 2, w_rows * (uint64_t)p.K * 2};
+    const uint32_t box[3] = {(uint32_t)kBlockK, (uint32_t)kWBoxRows, 1u};
+    if (!encode_map(&mw, p.W, 3, dims, str, box)) return cudaErrorInvalidValue;
+  }
+
+  TcParams prm;
+  prm.offsets = p.offsets;
+  prm.fixed_rows = p.fixed_rows;
+  prm.E = groups;
+  prm.n_feat = p.n_feat;
+  prm.K = p.K;
+  prm.out = static_cast<__nv_bfloat16*>(p.out);
+  prm.row_tile = row_tile;
+  prm.x_tile_bytes = row_tile * kBlockK * 2;
+  prm.status = status;
+  const int stage_bytes = 2 * kWBoxBytes + prm.x_tile_bytes;
+  const size_t tail = (2 * kMaxStages + 4) * sizeof(uint64_t) + 2 * sizeof(uint32_t) + 2 * (size_t)(groups + 1) * sizeof(int);
+  int stages = (int)((kSmemBudget - 1024 - (int)tail) / stage_bytes);
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) return cudaErrorNotSupported;
+  prm.n_stages = stages;
+  const size_t smem = 1024 + (size_t)stages * stage_bytes + tail;
+
+  const int feat_per_tile = p.gated ? 128 : 256;
+  const int64_t n_ft = (p.n_feat + feat_per_tile - 1) / feat_per_tile;
+  const int64_t row_tiles = p.rows_bound / row_tile + (groups < p.rows_bound ? groups : p.rows_bound);
+  int64_t tiles = row_tiles * n_ft;
+  int grid = (int)(tiles < (int64_t)max_ctas ? tiles : (int64_t)max_ctas);
+  if (grid < 1) grid = 1;
+
+  cudaError_t err;
+  if (swap_ab) err = p.gated ? launch_variant<true, true>(mx, mw, prm, grid, smem, stream)
+                             : launch_variant<true, false>(mx, mw, prm, grid, smem, stream);
+  else err = p.gated ? launch_variant<false, true>(mx, mw, prm, grid, smem, stream)
+                     : launch_variant<false, false>(mx, mw, prm, grid, smem, stream);
+  if (err == cudaSuccess && n_launches) *n_launches += 1;
+  return err;
+}
+
+}  // namespace moe

@@ -1,0 +1,64 @@
+// Internal launcher interface between the C-ABI layer (ctx.cu) and the kernels.
+// Every launcher enqueues on `stream`, never synchronises, and returns the CUDA error of the launch.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace moe {
+
+// Device status codes (same values as moe_status in the public header).
+constexpr int kStOk = 0;
+constexpr int kStTimeout = 6;
+constexpr int kStBadIndex = 7;
+
+// ---- a1 route ------------------------------------------------------------------------------
+cudaError_t launch_route(const float* logits, const float* bias, int T, int E, int k, float scale, int32_t* idx,
+                         float* w, cudaStream_t stream, int* n_launches);
+
+// ---- a2-a4 layout --------------------------------------------------------------------------
+// Slots per warp-owned chunk in the multi-CTA path, and the scratch it needs.
+constexpr int kLayoutChunk = 1024;
+inline size_t layout_scratch_ints(int64_t n_slots, int E) {
+  int64_t chunks = (n_slots + kLayoutChunk - 1) / kLayoutChunk;
+  return (size_t)(chunks > 0 ? chunks : 1) * (size_t)E;
+}
+cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32_t* counts, int32_t* offsets,
+                          int32_t* perm, int32_t* inv_perm, int32_t* scratch, int* status, cudaStream_t stream,
+                          int* n_launches);
+
+// ---- a5 permute, a9 combine ----------------------------------------------------------------
+cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm, int T, int k, int H,
+                           cudaStream_t stream, int* n_launches);
+cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32_t* inv_perm, const float* topk_w,
+                           void* out, int T, int k, int H, cudaStream_t stream, int* n_launches);
+
+// ---- a6-a8 grouped GEMM --------------------------------------------------------------------
+// One grouped GEMM pass:  out[r, :] = epilogue( A[r, :] . W[e]^T )  for r in expert e's segment.
+//   gated:     W[e] is [2*n_feat, K]; out[r,i] = silu(A.W[e,i]) * (A.W[e,n_feat+i]),  i < n_feat
+//   not gated: W[e] is [n_feat, K];   out[r,c] = A.W[e,c]
+// offsets == nullptr means a single group of `fixed_rows` rows (the shared expert).
+struct GemmProblem {
+  const void* A;           // bf16 [rows_cap, K]
+  const void* W;           // bf16 [E, (gated?2:1)*n_feat, K]
+  void* out;               // bf16 [rows_cap, n_feat]
+  const int32_t* offsets;  // [E+1] device, or nullptr
+  int32_t fixed_rows;      // rows when offsets == nullptr
+  int64_t rows_cap;        // rows addressable in A / out (capacity of the buffers)
+  int64_t rows_bound;      // upper bound on the rows actually routed this call (T*k or T)
+  int32_t E;
+  int32_t n_feat;
+  int32_t K;
+  bool gated;
+};
+
+cudaError_t launch_gemm_validation(const GemmProblem& p, cudaStream_t stream, int* n_launches);
+
+// Tensor-core path (tcgen05 + TMEM + TMA).  `swap_ab` selects the small-M variant; `row_tile` is the
+// token tile (128 for large-M; 16..128 for small-M); `max_ctas` caps the persistent grid.
+// Returns cudaErrorNotSupported for shapes it does not handle.
+cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int max_ctas, int* status,
+                           cudaStream_t stream, int* n_launches);
+// One-time driver entry-point lookup for tensor-map encoding; returns false (with a reason) if unavailable.
+bool gemm_tc_init(const char** why);
+
+}  // namespace moe

@@ -1,0 +1,246 @@
+// Stages a2-a4: per-expert counts, exclusive scan, stable token-to-expert permutation.
+//
+// The permutation must be bit-exact and run-to-run identical, so no slot is claimed with a global
+// atomic.  The flat slots are cut into warp-owned chunks; a warp walks its chunk 32 slots at a time
+// and ranks equal experts inside a step with __match_any_sync, which keeps ascending slot order.
+//   small N (decode, low latency): ONE CTA does count -> scan -> place in shared memory, one launch.
+//   large N (prefill):             count per chunk -> scan over chunks and experts -> place per chunk.
+#include "kernels.h"
+
+namespace moe {
+namespace {
+
+constexpr int kFusedWarps = 32;           // single-CTA path: 32 warps
+constexpr int kFusedMaxSlotsPerWarp = 512;  // -> up to 16384 slots in one CTA
+constexpr int kChunkWarpsPerBlock = 4;    // multi-CTA path: warps (= chunks) per CTA
+
+__device__ __forceinline__ void flag_status(int* status, int code) {
+  if (status != nullptr) atomicCAS(status, kStOk, code);
+}
+
+// Counts one chunk [f0, f1) into hist[0..E) (shared memory, zeroed by the caller).
+__device__ __forceinline__ void count_chunk(const int32_t* __restrict__ topk_idx, int64_t f0, int64_t f1, int E,
+                                            int* hist, int* status) {
+  const int lane = threadIdx.x & 31;
+  for (int64_t f = f0 + lane; f < f1; f += 32) {
+    const int e = topk_idx[f];
+    if (e >= 0 && e < E) atomicAdd(&hist[e], 1);  // integer adds commute: the count is order-independent
+    else flag_status(status, kStBadIndex);
+  }
+}
+
+// Places one chunk.  run[e] holds the destination of the chunk's next slot of expert e.
+__device__ __forceinline__ void place_chunk(const int32_t* __restrict__ topk_idx, int64_t f0, int64_t f1, int E,
+                                            int* run, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
+  const int lane = threadIdx.x & 31;
+  const unsigned lt_mask = (1u << lane) - 1u;
+  for (int64_t base = f0; base < f1; base += 32) {
+    const int64_t f = base + lane;
+    int e = -1;
+    if (f < f1) e = topk_idx[f];
+    const bool valid = (e >= 0 && e < E);
+    const int keyv = valid ? e : (E + lane);  // invalid lanes never group with anyone
+    const unsigned peers = __match_any_sync(0xffffffffu, keyv);
+    int p = -1;
+    if (valid) p = run[e] + __popc(peers & lt_mask);
+    __syncwarp();
+    if (valid && (peers & lt_mask) == 0u) run[e] += __popc(peers);  // the lowest lane of a group advances it
+    __syncwarp();
+    if (f < f1) {
+      inv_perm[f] = p;
+      if (valid) perm[p] = (int32_t)f;
+    }
+  }
+}
+
+// Block-wide exclusive scan of counts[0..E) -> offsets[0..E]; E <= 1024, blockDim.x a multiple of 32 and >= E...
+// handled in rounds of blockDim.x so that any E works.  `warp_sums` is 33 ints of shared scratch.
+__device__ void block_exclusive_scan(const int* counts_sh, int E, int32_t* __restrict__ offsets_out, int* offsets_sh,
+                                     int* warp_sums) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  int carry = 0;
+  for (int base = 0; base < E; base += blockDim.x) {
+    const int e = base + threadIdx.x;
+    const int v = (e < E) ? counts_sh[e] : 0;
+    int incl = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += n;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int ws = (lane < nwarps) ? warp_sums[lane] : 0;
+      int wincl = ws;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, wincl, off);
+        if (lane >= off) wincl += n;
+      }
+      if (lane < nwarps) warp_sums[lane] = wincl - ws;  // exclusive prefix of the warp totals
+      if (lane == 31) warp_sums[32] = wincl;            // total of this round
+    }
+    __syncthreads();
+    const int excl = carry + warp_sums[warp] + incl - v;
+    if (e < E) {
+      offsets_sh[e] = excl;
+      if (offsets_out != nullptr) offsets_out[e] = excl;
+    }
+    carry += warp_sums[32];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    offsets_sh[E] = carry;
+    if (offsets_out != nullptr) offsets_out[E] = carry;
+  }
+  __syncthreads();
+}
+
+// ---- single-CTA path: count, scan and place in one launch -------------------------------------
+// shared memory: hist[kFusedWarps][E] | offsets_sh[E+1] | counts_sh[E] | warp_sums[33]
+__global__ void __launch_bounds__(kFusedWarps * 32)
+layout_fused_kernel(const int32_t* __restrict__ topk_idx, int n_slots, int E, int slots_per_warp,
+                    int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ perm,
+                    int32_t* __restrict__ inv_perm, int* status) {
+  extern __shared__ int sh[];
+  int* hist = sh;
+  int* offsets_sh = hist + kFusedWarps * E;
+  int* counts_sh = offsets_sh + (E + 1);
+  int* warp_sums = counts_sh + E;
+  const int warp = threadIdx.x >> 5;
+
+  for (int i = threadIdx.x; i < kFusedWarps * E; i += blockDim.x) hist[i] = 0;
+  __syncthreads();
+  const int64_t f0 = min((int64_t)warp * slots_per_warp, (int64_t)n_slots);
+  const int64_t f1 = min(f0 + slots_per_warp, (int64_t)n_slots);
+  count_chunk(topk_idx, f0, f1, E, hist + warp * E, status);
+  __syncthreads();
+  // per expert: exclusive prefix over the warps' chunks, total into counts
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    int sum = 0;
+    for (int wv = 0; wv < kFusedWarps; ++wv) {
+      const int c = hist[wv * E + e];
+      hist[wv * E + e] = sum;
+      sum += c;
+    }
+    counts_sh[e] = sum;
+    counts[e] = sum;
+  }
+  __syncthreads();
+  block_exclusive_scan(counts_sh, E, offsets, offsets_sh, warp_sums);
+  int* run = hist + warp * E;
+  for (int e = threadIdx.x & 31; e < E; e += 32) run[e] += offsets_sh[e];
+  __syncwarp();
+  place_chunk(topk_idx, f0, f1, E, run, perm, inv_perm);
+}
+
+// ---- multi-CTA path ------------------------------------------------------------------------------
+// (1) per-chunk histograms: chunk_counts[chunk][e]
+__global__ void __launch_bounds__(kChunkWarpsPerBlock * 32)
+layout_count_kernel(const int32_t* __restrict__ topk_idx, int64_t n_slots, int E, int n_chunks,
+                    int32_t* __restrict__ chunk_counts, int* status) {
+  extern __shared__ int sh[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk = blockIdx.x * kChunkWarpsPerBlock + warp;
+  int* hist = sh + warp * E;
+  for (int e = lane; e < E; e += 32) hist[e] = 0;
+  __syncwarp();
+  if (chunk >= n_chunks) return;
+  const int64_t f0 = (int64_t)chunk * kLayoutChunk;
+  const int64_t f1 = min(f0 + kLayoutChunk, n_slots);
+  count_chunk(topk_idx, f0, f1, E, hist, status);
+  __syncwarp();
+  for (int e = lane; e < E; e += 32) chunk_counts[(size_t)chunk * E + e] = hist[e];
+}
+
+// (2) one CTA: per expert an exclusive prefix over chunks (in place), totals -> counts, then the
+//     exclusive scan over experts -> offsets.
+__global__ void __launch_bounds__(1024)
+layout_scan_kernel(int32_t* __restrict__ chunk_counts, int n_chunks, int E, int32_t* __restrict__ counts,
+                   int32_t* __restrict__ offsets) {
+  extern __shared__ int sh[];
+  int* counts_sh = sh;
+  int* offsets_sh = counts_sh + E;
+  int* warp_sums = offsets_sh + (E + 1);
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    int sum = 0;
+    for (int c = 0; c < n_chunks; ++c) {
+      const int v = chunk_counts[(size_t)c * E + e];
+      chunk_counts[(size_t)c * E + e] = sum;
+      sum += v;
+    }
+    counts_sh[e] = sum;
+    counts[e] = sum;
+  }
+  __syncthreads();
+  block_exclusive_scan(counts_sh, E, offsets, offsets_sh, warp_sums);
+}
+
+// (3) place each chunk at offsets[e] + (prefix of earlier chunks)[e]
+__global__ void __launch_bounds__(kChunkWarpsPerBlock * 32)
+layout_place_kernel(const int32_t* __restrict__ topk_idx, int64_t n_slots, int E, int n_chunks,
+                    const int32_t* __restrict__ chunk_prefix, const int32_t* __restrict__ offsets,
+                    int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
+  extern __shared__ int sh[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk = blockIdx.x * kChunkWarpsPerBlock + warp;
+  if (chunk >= n_chunks) return;
+  int* run = sh + warp * E;
+  for (int e = lane; e < E; e += 32) run[e] = offsets[e] + chunk_prefix[(size_t)chunk * E + e];
+  __syncwarp();
+  const int64_t f0 = (int64_t)chunk * kLayoutChunk;
+  const int64_t f1 = min(f0 + kLayoutChunk, n_slots);
+  place_chunk(topk_idx, f0, f1, E, run, perm, inv_perm);
+}
+
+__global__ void layout_empty_kernel(int E, int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+  for (int e = threadIdx.x; e <= E; e += blockDim.x) {
+    if (e < E) counts[e] = 0;
+    offsets[e] = 0;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32_t* counts, int32_t* offsets,
+                          int32_t* perm, int32_t* inv_perm, int32_t* scratch, int* status, cudaStream_t stream,
+                          int* n_launches) {
+  cudaError_t err;
+  if (n_slots <= 0) {
+    layout_empty_kernel<<<1, 256, 0, stream>>>(E, counts, offsets);
+    err = cudaGetLastError();
+    if (err == cudaSuccess && n_launches) *n_launches += 1;
+    return err;
+  }
+  const size_t fused_smem = ((size_t)kFusedWarps * E + (E + 1) + E + 33) * sizeof(int);
+  if (n_slots <= (int64_t)kFusedWarps * kFusedMaxSlotsPerWarp && fused_smem <= 200 * 1024) {
+    int spw = (int)((n_slots + kFusedWarps - 1) / kFusedWarps);
+    spw = (spw + 31) / 32 * 32;
+    if (fused_smem > 48 * 1024) {
+      err = cudaFuncSetAttribute(layout_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused_smem);
+      if (err != cudaSuccess) return err;
+    }
+    layout_fused_kernel<<<1, kFusedWarps * 32, fused_smem, stream>>>(topk_idx, (int)n_slots, E, spw, counts, offsets,
+                                                                     perm, inv_perm, status);
+    err = cudaGetLastError();
+    if (err == cudaSuccess && n_launches) *n_launches += 1;
+    return err;
+  }
+  const int n_chunks = (int)((n_slots + kLayoutChunk - 1) / kLayoutChunk);
+  const int blocks = (n_chunks + kChunkWarpsPerBlock - 1) / kChunkWarpsPerBlock;
+  const size_t chunk_smem = (size_t)kChunkWarpsPerBlock * E * sizeof(int);
+  layout_count_kernel<<<blocks, kChunkWarpsPerBlock * 32, chunk_smem, stream>>>(topk_idx, n_slots, E, n_chunks,
+                                                                                scratch, status);
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  const size_t scan_smem = ((size_t)E + (E + 1) + 33) * sizeof(int);
+  layout_scan_kernel<<<1, 1024, scan_smem, stream>>>(scratch, n_chunks, E, counts, offsets);
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  layout_place_kernel<<<blocks, kChunkWarpsPerBlock * 32, chunk_smem, stream>>>(topk_idx, n_slots, E, n_chunks,
+                                                                                scratch, offsets, perm, inv_perm);
+  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  if (n_launches) *n_launches += 3;
+  return cudaSuccess;
+}
+
+}  // namespace moe

@@ -1,0 +1,148 @@
+"""Phase contexts: ownership, isolation, call order and host-side error paths (no GPU is ever faulted)."""
+import ctypes
+
+import pytest
+import torch
+
+from paper_2609_00993_b200 import binding as B
+from paper_2609_00993_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _cfg(phase=B.MOE_PHASE_PREFILL, max_tokens=32, **kw):
+    return B.make_config(256, 8, 2, 128, kw.pop("shared_inter", 0), max_tokens, phase, **kw)
+
+
+def test_workspaces_of_live_contexts_may_not_overlap():
+    cfg = _cfg()
+    n = B.moe_ctx_workspace_bytes(cfg)
+    ws = torch.empty(2 * n + 512, dtype=torch.uint8, device=DEV)
+    a = B.MoeContext(cfg, workspace=ws[:n])
+    with pytest.raises(B.MoeError) as ei:
+        B.MoeContext(cfg, workspace=ws[256:256 + n])
+    assert ei.value.status == B.MOE_ERR_STATE
+    off = (n + 255) // 256 * 256
+    b = B.MoeContext(cfg, workspace=ws[off:off + n])  # disjoint range: fine
+    a.close(); b.close()
+    c = B.MoeContext(cfg, workspace=ws[256:256 + n])  # the range is free again after destroy
+    c.close()
+
+
+def test_a_stream_serves_one_phase_only():
+    s = torch.cuda.Stream()
+    p = B.MoeContext(_cfg(B.MOE_PHASE_PREFILL), stream=s)
+    with pytest.raises(B.MoeError) as ei:
+        B.MoeContext(_cfg(B.MOE_PHASE_DECODE), stream=s)
+    assert ei.value.status == B.MOE_ERR_STATE
+    p.close()
+
+
+def test_decode_context_holds_two_buffer_sets():
+    assert B.moe_ctx_workspace_bytes(_cfg(B.MOE_PHASE_DECODE)) > 1.9 * B.moe_ctx_workspace_bytes(_cfg()) - 4096
+    ctx = B.MoeContext(_cfg(B.MOE_PHASE_DECODE))
+    shape = wl.LayerShape("t", T=32, H=256, E=8, k=2, I=128)
+    w, a = wl.make_weights(shape, 1, DEV), wl.make_activations(shape, 2, DEV)
+    torch.cuda.synchronize()
+    ctx.layer(a["x"], a["logits"], None, w["w_gate_up"], w["w_down"])
+    p1 = ctx.moe_ctx_debug_ptrs()["y_perm"].data_ptr()
+    ctx.layer(a["x"], a["logits"], None, w["w_gate_up"], w["w_down"])
+    p2 = ctx.moe_ctx_debug_ptrs()["y_perm"].data_ptr()
+    ctx.layer(a["x"], a["logits"], None, w["w_gate_up"], w["w_down"])
+    p3 = ctx.moe_ctx_debug_ptrs()["y_perm"].data_ptr()
+    assert p1 != p2 and p1 == p3  # the double-buffer index flips per step; addresses are stable
+    ctx.close()
+
+
+def test_call_order_and_argument_errors():
+    ctx = B.MoeContext(_cfg())
+    shape = wl.LayerShape("t", T=32, H=256, E=8, k=2, I=128)
+    w, a = wl.make_weights(shape, 1, DEV), wl.make_activations(shape, 2, DEV)
+    bufs = B.alloc_step_buffers(32, 2, 8, DEV)
+    out = torch.empty(32, 256, dtype=torch.bfloat16, device=DEV)
+    torch.cuda.synchronize()
+
+    def status_of(fn):
+        with pytest.raises(B.MoeError) as ei:
+            fn()
+        return ei.value.status
+
+    assert status_of(lambda: ctx.moe_combine(bufs["topk_w"], bufs["inv_perm"], out)) == B.MOE_ERR_STATE
+    assert status_of(lambda: ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"])) == B.MOE_ERR_STATE
+    big = torch.zeros(64, 8, device=DEV)
+    assert status_of(lambda: ctx.moe_route(big, None, bufs["topk_idx"], bufs["topk_w"])) == B.MOE_ERR_CAPACITY
+    assert status_of(lambda: ctx.moe_route(a["logits"].view(-1)[1:257].view(32, 8), None, bufs["topk_idx"], bufs["topk_w"])) \
+        == B.MOE_ERR_INVALID_ARG  # misaligned pointer
+    ctx.moe_route(a["logits"], None, bufs["topk_idx"], bufs["topk_w"])
+    ctx.moe_dispatch_layout(bufs["topk_idx"], None)  # layout only
+    assert status_of(lambda: ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"])) == B.MOE_ERR_STATE
+    ctx.moe_dispatch_layout(bufs["topk_idx"], a["x"])
+    assert status_of(lambda: ctx.moe_route(a["logits"], None, bufs["topk_idx"], bufs["topk_w"])) == B.MOE_ERR_STATE
+    assert status_of(lambda: ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"], T=16)) == B.MOE_ERR_INVALID_ARG
+    ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"])
+    ctx.moe_combine(bufs["topk_w"], None, out)
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_OK
+    assert ctx.moe_ctx_launch_count() >= 5
+    ctx.close()
+
+
+def test_create_rejects_bad_configurations():
+    for bad in (B.make_config(100, 8, 2, 128, 0, 4), B.make_config(256, 8, 9, 128, 0, 4),
+                B.make_config(256, 2000, 2, 128, 0, 4), B.make_config(256, 8, 2, 128, 0, 0)):
+        assert B.moe_ctx_workspace_bytes(bad) == 0
+        with pytest.raises(B.MoeError):
+            B.MoeContext(bad)
+    cfg = _cfg()
+    small = torch.empty(1024, dtype=torch.uint8, device=DEV)
+    lib = B.load_library()
+    h = ctypes.c_void_p()
+    st = lib.moe_ctx_create(ctypes.byref(cfg), ctypes.c_void_p(small.data_ptr()), small.numel(), None, ctypes.byref(h))
+    assert st == B.MOE_ERR_CAPACITY and not h.value
+
+
+def test_destroy_refuses_while_work_is_in_flight():
+    """An abandoned operation retires its buffers only at a quiescent point."""
+    shape = wl.C3.with_tokens(4096)
+    cfg = B.make_config(shape.H, shape.E, shape.k, shape.I, 0, shape.T, B.MOE_PHASE_PREFILL, 0, B.MOE_GEMM_VALIDATION)
+    s = torch.cuda.Stream()
+    ctx = B.MoeContext(cfg, stream=s)
+    w, a = wl.make_weights(shape, 1, DEV), wl.make_activations(shape, 2, DEV)
+    torch.cuda.synchronize()
+    for _ in range(3):
+        ctx.layer(a["x"], a["logits"], None, w["w_gate_up"], w["w_down"])  # the slow validation GEMM keeps the stream busy
+    with pytest.raises(B.MoeError) as ei:
+        ctx.destroy()
+    assert ei.value.status == B.MOE_ERR_STATE
+    s.synchronize()
+    ctx.destroy()
+
+
+def test_prefill_traffic_cannot_disturb_a_decode_step():
+    """P runs between D's layout and D's combine; D's results are bit-identical to D alone."""
+    shape = wl.LayerShape("t", T=64, H=512, E=16, k=4, I=256, shared_I=128)
+    pshape = shape.with_tokens(1024)
+    w = wl.make_weights(shape, 1, DEV)
+    ad, ap = wl.make_activations(shape, 2, DEV), wl.make_activations(pshape, 3, DEV)
+    sp, sd = torch.cuda.Stream(), torch.cuda.Stream()
+    d = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 64, B.MOE_PHASE_DECODE), stream=sd)
+    p = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 1024, B.MOE_PHASE_PREFILL), stream=sp)
+    torch.cuda.synchronize()
+    alone, bufs_alone = d.layer(ad["x"], ad["logits"], None, w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+    torch.cuda.synchronize()
+    d.layer(ad["x"], ad["logits"], None, w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])  # back to buffer set 0
+    torch.cuda.synchronize()
+    bufs = B.alloc_step_buffers(64, 4, 16, DEV)
+    out = torch.empty(64, 512, dtype=torch.bfloat16, device=DEV)
+    d.moe_route(ad["logits"], None, bufs["topk_idx"], bufs["topk_w"])
+    d.moe_dispatch_layout(bufs["topk_idx"], ad["x"], bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"])
+    for _ in range(3):
+        p.layer(ap["x"], ap["logits"], None, w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+    d.moe_grouped_ffn(w["w_gate_up"], w["w_down"], ad["x"], w["ws_gate_up"], w["ws_down"])
+    p.layer(ap["x"], ap["logits"], None, w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+    d.moe_combine(bufs["topk_w"], bufs["inv_perm"], out)
+    torch.cuda.synchronize()
+    assert torch.equal(out, alone)
+    assert torch.equal(bufs["perm"], bufs_alone["perm"])
+    p.close(); d.close()

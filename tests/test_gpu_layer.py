@@ -1,0 +1,162 @@
+"""Whole-layer parity on the five workloads, in the launch configuration the benchmark times.
+
+Integer outputs (routing indices, counts, offsets, permutation) are compared in full and bit-exactly.
+The bf16 layer output is compared with the oracle's unrounded result: in full where the oracle finishes in
+seconds (C1), else on sampled tokens computed one by one from the dense definition.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import (check_layer, check_topk_w, np_f32, np_i32, oracle_tokens_from_device, sample_tokens)
+from paper_2609_00993_b200 import binding as B
+from paper_2609_00993_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _ctx_for(shape, phase, max_tokens=None, sm_budget=0, stream=None):
+    cfg = B.make_config(shape.H, shape.E, shape.k, shape.I, shape.shared_I, max_tokens or shape.T, phase, sm_budget)
+    return B.MoeContext(cfg, stream=stream)
+
+
+def _check_integers(bufs, logits, bias, shape, T):
+    ridx, rw = oracle.route(np_f32(logits), None if bias is None else np_f32(bias), shape.k)
+    assert np.array_equal(np_i32(bufs["topk_idx"]), ridx), "topk_idx"
+    check_topk_w(bufs["topk_w"], rw)
+    counts, offsets, perm, inv = oracle.layout(ridx.reshape(-1), shape.E)
+    assert np.array_equal(np_i32(bufs["counts"]), counts), "counts"
+    assert np.array_equal(np_i32(bufs["offsets"]), offsets), "offsets"
+    assert np.array_equal(np_i32(bufs["perm"]), perm), "perm"
+    assert np.array_equal(np_i32(bufs["inv_perm"]), inv), "inv_perm"
+    assert counts.sum() == T * shape.k
+    return counts, offsets, perm
+
+
+def _step(ctx, a, w):
+    T = a["x"].shape[0]
+    bufs = B.alloc_step_buffers(T, ctx.cfg.top_k, ctx.cfg.n_experts, DEV)
+    torch.cuda.synchronize()
+    out, _ = ctx.layer(a["x"], a["logits"], a["bias"], w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"],
+                       bufs=bufs)
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_OK
+    return out, bufs
+
+
+@pytest.fixture(scope="module")
+def v3_weights():
+    """DeepSeek-V3-shaped layer weights (22.6 GB on the device), shared by the C2, C4 and C5 cases."""
+    w = wl.make_weights(wl.C2, seed=2, device=DEV)
+    yield w
+    del w
+    torch.cuda.empty_cache()
+
+
+def test_c1_tiny_prefill_full_comparison():
+    shape = wl.C1
+    w = wl.make_weights(shape, 1, DEV)
+    a = wl.make_activations(shape, 1, DEV)
+    ctx = _ctx_for(shape, B.MOE_PHASE_PREFILL)
+    out, bufs = _step(ctx, a, w)
+    _check_integers(bufs, a["logits"], a["bias"], shape, shape.T)
+    ref = oracle.layer(wl.bits(a["x"]), np_f32(a["logits"]), None, shape.k, wl.bits(w["w_gate_up"]), wl.bits(w["w_down"]))
+    check_layer(out, ref["out"], literal=True, label="C1")
+    # the same step through the host-buffer entry point
+    out_h = torch.empty(shape.T, shape.H, dtype=torch.bfloat16).pin_memory()
+    ctx.moe_layer_host(a["logits"].cpu().pin_memory(), None, a["x"].cpu().pin_memory(), w["w_gate_up"], w["w_down"],
+                       None, None, out_h)
+    assert torch.equal(out_h, out.cpu())
+    ctx.close()
+
+
+def test_c3_prefill_qwen3_shaped():
+    shape = wl.C3
+    w = wl.make_weights(shape, 3, DEV)
+    a = wl.make_activations(shape, 3, DEV)
+    ctx = _ctx_for(shape, B.MOE_PHASE_PREFILL)
+    out, bufs = _step(ctx, a, w)
+    counts, offsets, perm = _check_integers(bufs, a["logits"], a["bias"], shape, shape.T)
+    toks = sample_tokens(shape.T, counts, offsets, perm, shape.k, 48, seed=3)
+    ref, mag = oracle_tokens_from_device(a["x"], bufs["topk_idx"], bufs["topk_w"], w, toks)
+    check_layer(out[toks], ref, mag, literal=True, label="C3")
+    # variable-length prefill: the same context takes one call per prompt chunk (eager variable-length P)
+    lens = wl.prefill_chunk_lengths(shape.T, seed=3)
+    start = 0
+    for n in lens[:3]:
+        sub = {"x": a["x"][start:start + n].contiguous(), "logits": a["logits"][start:start + n].contiguous(), "bias": None}
+        o2, _ = _step(ctx, sub, w)
+        assert torch.equal(o2, out[start:start + n]), "a token's output must not depend on its batch"
+        start += n
+    ctx.close()
+
+
+def test_c2_decode_v3_shaped(v3_weights):
+    shape = wl.C2
+    a = wl.make_activations(shape, 2, DEV)
+    ctx = _ctx_for(shape, B.MOE_PHASE_DECODE)
+    out, bufs = _step(ctx, a, v3_weights)
+    counts, offsets, perm = _check_integers(bufs, a["logits"], a["bias"], shape, shape.T)
+    toks = sample_tokens(shape.T, counts, offsets, perm, shape.k, 12, seed=2)
+    ref, mag = oracle_tokens_from_device(a["x"], bufs["topk_idx"], bufs["topk_w"], v3_weights, toks)
+    check_layer(out[toks], ref, mag, literal=False, label="C2")
+    # a second step lands in the other buffer set of the D context and gives the same bits
+    out2, _ = _step(ctx, a, v3_weights)
+    assert torch.equal(out, out2)
+    ctx.close()
+
+
+def test_c4_prefill_and_decode_contexts_concurrently(v3_weights):
+    """A P batch on stream P and a D batch on stream D, each with its own context: results equal the
+    ones each phase gives alone (bitwise), and match the oracle on sampled tokens."""
+    sp, sd = torch.cuda.Stream(), torch.cuda.Stream()
+    ctx_p = _ctx_for(wl.C4_P, B.MOE_PHASE_PREFILL, stream=sp)
+    ctx_d = _ctx_for(wl.C4_D, B.MOE_PHASE_DECODE, stream=sd)
+    ap = wl.make_activations(wl.C4_P, 4000, DEV)
+    ad = wl.make_activations(wl.C4_D, 5000, DEV)
+    w = v3_weights
+    bp = B.alloc_step_buffers(wl.C4_P.T, 8, 256, DEV)
+    bd = B.alloc_step_buffers(wl.C4_D.T, 8, 256, DEV)
+    op = torch.empty(wl.C4_P.T, 7168, dtype=torch.bfloat16, device=DEV)
+    od = torch.empty(wl.C4_D.T, 7168, dtype=torch.bfloat16, device=DEV)
+    torch.cuda.synchronize()
+    # alone
+    ctx_p.layer(ap["x"], ap["logits"], ap["bias"], w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"], out=op, bufs=bp)
+    torch.cuda.synchronize()
+    ctx_d.layer(ad["x"], ad["logits"], ad["bias"], w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"], out=od, bufs=bd)
+    torch.cuda.synchronize()
+    op_alone, od_alone = op.clone(), od.clone()
+    perm_d_alone = bd["perm"].clone()
+    op.zero_(); od.zero_()
+    torch.cuda.synchronize()
+    # together: P first so that a P layer is in flight when the D steps start
+    ctx_p.layer(ap["x"], ap["logits"], ap["bias"], w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"], out=op, bufs=bp)
+    for _ in range(2):
+        ctx_d.layer(ad["x"], ad["logits"], ad["bias"], w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"], out=od, bufs=bd)
+    torch.cuda.synchronize()
+    assert ctx_p.moe_ctx_status() == B.MOE_OK and ctx_d.moe_ctx_status() == B.MOE_OK
+    assert torch.equal(op, op_alone) and torch.equal(od, od_alone) and torch.equal(bd["perm"], perm_d_alone)
+    for name, shape, a, bufs, out in (("C4-P", wl.C4_P, ap, bp, op), ("C4-D", wl.C4_D, ad, bd, od)):
+        counts, offsets, perm = _check_integers(bufs, a["logits"], a["bias"], shape, shape.T)
+        toks = sample_tokens(shape.T, counts, offsets, perm, shape.k, 6, seed=4)
+        ref, mag = oracle_tokens_from_device(a["x"], bufs["topk_idx"], bufs["topk_w"], w, toks)
+        check_layer(out[toks], ref, mag, literal=False, label=name)
+    ctx_p.close(); ctx_d.close()
+
+
+@pytest.mark.parametrize("T", [1, 16, 128, 1024, 8192, 32768])
+def test_c5_skewed_routing(v3_weights, T):
+    shape = wl.C5.with_tokens(T)
+    a = wl.make_activations(shape, 6, DEV)
+    phase = B.MOE_PHASE_DECODE if T <= 256 else B.MOE_PHASE_PREFILL
+    ctx = _ctx_for(shape, phase)
+    out, bufs = _step(ctx, a, v3_weights)
+    counts, offsets, perm = _check_integers(bufs, a["logits"], a["bias"], shape, T)
+    toks = sample_tokens(T, counts, offsets, perm, shape.k, 4, seed=T)
+    ref, mag = oracle_tokens_from_device(a["x"], bufs["topk_idx"], bufs["topk_w"], v3_weights, toks)
+    check_layer(out[toks], ref, mag, literal=False, label=f"C5 T={T}")
+    if T >= 128:
+        assert counts.max() * shape.E / counts.sum() > 8, "the Zipf popularity should skew the load"
+    ctx.close()
