@@ -165,11 +165,25 @@ moe_status moe_layer_host(moe_ctx* ctx, const float* logits_host, const float* s
                           int32_t T, const void* w_gate_up, const void* w_down, const void* ws_gate_up,
                           const void* ws_down, void* out_host);
 
-/* Test/inspection only: device pointers into the context's CURRENT buffer set.  Rows
+/* Test/inspection only: device pointers into the buffer set of the step in progress (between steps: of
+ * the step that finished last).  Rows
  * [0, T*k) of x_perm [.,H], act [.,I], y_perm [.,H] and rows [0,T) of y_shared [.,H] are
  * defined after the respective stage.  Any out-pointer may be NULL. */
 moe_status moe_ctx_debug_ptrs(moe_ctx* ctx, void** x_perm, void** act, void** y_perm, void** y_shared,
                               int32_t** counts, int32_t** offsets);
+
+/* Per-stage device timing (measurement aid; off by default).  While enabled, every stage's launches are
+ * bracketed by CUDA events on the context's stream.  moe_ctx_read_profile synchronises the stream, returns
+ * the summed device time and the number of bracketed launches per stage since the last read, and resets.
+ * Stage order: 0 route, 1 layout (counts+scan+permutation), 2 permute rows, 3 routed GEMM1+SwiGLU,
+ * 4 routed GEMM2, 5 shared GEMM1+SwiGLU, 6 shared GEMM2, 7 combine. */
+#define MOE_N_STAGES 8
+typedef struct {
+  double ms[MOE_N_STAGES];
+  int64_t calls[MOE_N_STAGES];
+} moe_stage_times;
+moe_status moe_ctx_set_profiling(moe_ctx* ctx, int32_t enabled);
+moe_status moe_ctx_read_profile(moe_ctx* ctx, moe_stage_times* out);
 
 /* Kernels launched on this context since creation (for launch accounting in benchmarks). */
 int64_t moe_ctx_launch_count(const moe_ctx* ctx);

@@ -27,7 +27,9 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_CAPACITY", 3:
 # every symbol include/moe_pd.h declares
 EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_destroy", "moe_ctx_status",
            "moe_last_error", "moe_route", "moe_dispatch_layout", "moe_grouped_ffn", "moe_combine", "moe_layer_host",
-           "moe_ctx_debug_ptrs", "moe_ctx_launch_count")
+           "moe_ctx_debug_ptrs", "moe_ctx_launch_count", "moe_ctx_set_profiling", "moe_ctx_read_profile")
+
+STAGE_NAMES = ("route", "layout", "permute", "gemm1_swiglu", "gemm2", "shared_gemm1_swiglu", "shared_gemm2", "combine")
 
 
 class moe_config(ctypes.Structure):
@@ -35,6 +37,10 @@ class moe_config(ctypes.Structure):
                 ("inter", ctypes.c_int32), ("n_shared", ctypes.c_int32), ("shared_inter", ctypes.c_int32),
                 ("max_tokens", ctypes.c_int32), ("phase", ctypes.c_int32), ("sm_budget", ctypes.c_int32),
                 ("gemm_variant", ctypes.c_int32), ("routed_scale", ctypes.c_float)]
+
+
+class moe_stage_times(ctypes.Structure):
+    _fields_ = [("ms", ctypes.c_double * 8), ("calls", ctypes.c_int64 * 8)]
 
 
 class MoeError(RuntimeError):
@@ -83,6 +89,10 @@ def load_library() -> ctypes.CDLL:
     lib.moe_ctx_debug_ptrs.argtypes = [vp] + [ctypes.POINTER(vp)] * 6
     lib.moe_ctx_launch_count.restype = i64
     lib.moe_ctx_launch_count.argtypes = [vp]
+    lib.moe_ctx_set_profiling.restype = i32
+    lib.moe_ctx_set_profiling.argtypes = [vp, i32]
+    lib.moe_ctx_read_profile.restype = i32
+    lib.moe_ctx_read_profile.argtypes = [vp, ctypes.POINTER(moe_stage_times)]
     _lib = lib
     return lib
 
@@ -173,6 +183,15 @@ class MoeContext:
 
     def moe_ctx_launch_count(self) -> int:
         return int(self.lib.moe_ctx_launch_count(self.handle))
+
+    def moe_ctx_set_profiling(self, enabled: bool):
+        self._check(self.lib.moe_ctx_set_profiling(self.handle, int(bool(enabled))))
+
+    def moe_ctx_read_profile(self) -> dict:
+        """{stage name: (summed device ms, bracketed launches)} since the last read; synchronises the stream."""
+        t = moe_stage_times()
+        self._check(self.lib.moe_ctx_read_profile(self.handle, ctypes.byref(t)))
+        return {n: (float(t.ms[i]), int(t.calls[i])) for i, n in enumerate(STAGE_NAMES)}
 
     def moe_route(self, logits, select_bias, topk_idx, topk_w, T=None):
         _dev(logits, torch.float32, "logits"); _dev(select_bias, torch.float32, "select_bias")

@@ -124,6 +124,11 @@ struct moe_ctx {
   int32_t* inv_perm;
   cudaEvent_t done;  // recorded after the last enqueue of every call
   int64_t launches;
+  // per-stage timing (off by default): event pairs recorded around each stage's launches
+  bool profiling;
+  struct Span { cudaEvent_t beg, end; int stage; };
+  std::vector<Span> spans;
+  size_t spans_used;
   char err[256];
 };
 
@@ -163,6 +168,26 @@ void mark(moe_ctx* ctx, int n) {
   ctx->launches += n;
   cudaEventRecord(ctx->done, ctx->stream);
 }
+
+// Brackets the launches of one stage with events when profiling is on.
+struct StageTimer {
+  moe_ctx* ctx;
+  moe_ctx::Span* span = nullptr;
+  StageTimer(moe_ctx* c, int stage) : ctx(c) {
+    if (!c->profiling) return;
+    if (c->spans_used == c->spans.size()) {
+      moe_ctx::Span s;
+      if (cudaEventCreate(&s.beg) != cudaSuccess || cudaEventCreate(&s.end) != cudaSuccess) return;
+      c->spans.push_back(s);
+    }
+    span = &c->spans[c->spans_used++];
+    span->stage = stage;
+    cudaEventRecord(span->beg, c->stream);
+  }
+  ~StageTimer() {
+    if (span) cudaEventRecord(span->end, ctx->stream);
+  }
+};
 
 int gemm_ctas(const moe_ctx* ctx) {
   return (ctx->cfg.sm_budget > 0 && ctx->cfg.sm_budget < ctx->n_sms) ? ctx->cfg.sm_budget : ctx->n_sms;
@@ -227,6 +252,8 @@ moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspa
   ctx->state = ST_IDLE;
   ctx->T = 0;
   ctx->launches = 0;
+  ctx->profiling = false;
+  ctx->spans_used = 0;
   ctx->err[0] = 0;
   ctx->status = reinterpret_cast<int*>(ctx->ws);
   for (int s = 0; s < l.n_sets; ++s) carve_set(*cfg, ctx->ws + kStatusBlock + (size_t)s * l.set_bytes, &ctx->sets[s]);
@@ -282,6 +309,10 @@ moe_status moe_ctx_destroy(moe_ctx* ctx) {
       }
   }
   cudaEventDestroy(ctx->done);
+  for (auto& sp : ctx->spans) {
+    cudaEventDestroy(sp.beg);
+    cudaEventDestroy(sp.end);
+  }
   delete ctx;
   return MOE_OK;
 }
@@ -314,8 +345,12 @@ moe_status moe_route(moe_ctx* ctx, const float* logits, const float* select_bias
     return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
   DeviceGuard guard(ctx->device);
   int n = 0;
-  cudaError_t e = moe::launch_route(logits, select_bias, T, ctx->cfg.n_experts, ctx->cfg.top_k, ctx->cfg.routed_scale,
-                                    topk_idx, topk_w, ctx->stream, &n);
+  cudaError_t e;
+  {
+    StageTimer tm(ctx, 0);
+    e = moe::launch_route(logits, select_bias, T, ctx->cfg.n_experts, ctx->cfg.top_k, ctx->cfg.routed_scale, topk_idx,
+                          topk_w, ctx->stream, &n);
+  }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_route");
   ctx->state = ST_ROUTED;
   mark(ctx, n);
@@ -340,10 +375,16 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
   ctx->perm = perm ? perm : b.perm;
   ctx->inv_perm = inv_perm ? inv_perm : b.inv_perm;
   int n = 0;
-  cudaError_t e = moe::launch_layout(topk_idx, (int64_t)T * ctx->cfg.top_k, ctx->cfg.n_experts, ctx->counts,
-                                     ctx->offsets, ctx->perm, ctx->inv_perm, b.scan, ctx->status, ctx->stream, &n);
-  if (e == cudaSuccess && x != nullptr)
+  cudaError_t e;
+  {
+    StageTimer tm(ctx, 1);
+    e = moe::launch_layout(topk_idx, (int64_t)T * ctx->cfg.top_k, ctx->cfg.n_experts, ctx->counts, ctx->offsets,
+                           ctx->perm, ctx->inv_perm, b.scan, ctx->status, ctx->stream, &n);
+  }
+  if (e == cudaSuccess && x != nullptr) {
+    StageTimer tm(ctx, 2);
     e = moe::launch_permute(x, ctx->inv_perm, b.x_perm, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->stream, &n);
+  }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_dispatch_layout");
   ctx->T = T;
   ctx->state = x ? ST_LAID_OUT : ST_LAYOUT_ONLY;
@@ -371,16 +412,24 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
   cudaError_t e = cudaSuccess;
   if (T > 0) {
     moe::GemmProblem g1{b.x_perm, w_gate_up, b.act, ctx->offsets, 0, Ncap, N, c.n_experts, c.inter, c.hidden, true};
-    e = run_gemm(ctx, g1, T, &n);
+    {
+      StageTimer tm(ctx, 3);
+      e = run_gemm(ctx, g1, T, &n);
+    }
     if (e == cudaSuccess) {
       moe::GemmProblem g2{b.act, w_down, b.y_perm, ctx->offsets, 0, Ncap, N, c.n_experts, c.hidden, c.inter, false};
+      StageTimer tm(ctx, 4);
       e = run_gemm(ctx, g2, T, &n);
     }
     if (e == cudaSuccess && shared) {
       moe::GemmProblem s1{x, ws_gate_up, b.act_shared, nullptr, T, T, T, 1, c.shared_inter, c.hidden, true};
-      e = run_gemm(ctx, s1, T, &n);
+      {
+        StageTimer tm(ctx, 5);
+        e = run_gemm(ctx, s1, T, &n);
+      }
       if (e == cudaSuccess) {
         moe::GemmProblem s2{b.act_shared, ws_down, b.y_shared, nullptr, T, T, T, 1, c.hidden, c.shared_inter, false};
+        StageTimer tm(ctx, 6);
         e = run_gemm(ctx, s2, T, &n);
       }
     }
@@ -401,9 +450,12 @@ moe_status moe_combine(moe_ctx* ctx, const float* topk_w, const int32_t* inv_per
   DeviceGuard guard(ctx->device);
   BufferSet& b = ctx->sets[ctx->cur];
   int n = 0;
-  cudaError_t e = moe::launch_combine(b.y_perm, ctx->cfg.n_shared ? b.y_shared : nullptr,
-                                      inv_perm ? inv_perm : ctx->inv_perm, topk_w, out, T, ctx->cfg.top_k,
-                                      ctx->cfg.hidden, ctx->stream, &n);
+  cudaError_t e;
+  {
+    StageTimer tm(ctx, 7);
+    e = moe::launch_combine(b.y_perm, ctx->cfg.n_shared ? b.y_shared : nullptr, inv_perm ? inv_perm : ctx->inv_perm,
+                            topk_w, out, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->stream, &n);
+  }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_combine");
   ctx->state = ST_IDLE;
   if (ctx->n_sets == 2) ctx->cur ^= 1;  // D: the next step works in the other buffer set
@@ -440,6 +492,32 @@ moe_status moe_layer_host(moe_ctx* ctx, const float* logits_host, const float* s
   if (T > 0) e = cudaMemcpyAsync(out_host, b.out_stage, x_bytes, cudaMemcpyDeviceToHost, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "device-to-host copy");
+  return MOE_OK;
+}
+
+moe_status moe_ctx_set_profiling(moe_ctx* ctx, int32_t enabled) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  ctx->profiling = enabled != 0;
+  return MOE_OK;
+}
+
+moe_status moe_ctx_read_profile(moe_ctx* ctx, moe_stage_times* out) {
+  if (!ctx || !out) return MOE_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  memset(out, 0, sizeof *out);
+  cudaError_t e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_ctx_read_profile");
+  for (size_t i = 0; i < ctx->spans_used; ++i) {
+    const moe_ctx::Span& sp = ctx->spans[i];
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, sp.beg, sp.end) == cudaSuccess && sp.stage >= 0 && sp.stage < MOE_N_STAGES) {
+      out->ms[sp.stage] += ms;
+      out->calls[sp.stage] += 1;
+    } else {
+      (void)cudaGetLastError();
+    }
+  }
+  ctx->spans_used = 0;
   return MOE_OK;
 }
 

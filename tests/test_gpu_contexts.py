@@ -72,8 +72,8 @@ def test_call_order_and_argument_errors():
     assert status_of(lambda: ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"])) == B.MOE_ERR_STATE
     big = torch.zeros(64, 8, device=DEV)
     assert status_of(lambda: ctx.moe_route(big, None, bufs["topk_idx"], bufs["topk_w"])) == B.MOE_ERR_CAPACITY
-    assert status_of(lambda: ctx.moe_route(a["logits"].view(-1)[1:257].view(32, 8), None, bufs["topk_idx"], bufs["topk_w"])) \
-        == B.MOE_ERR_INVALID_ARG  # misaligned pointer
+    odd = torch.zeros(32 * 8 + 4, device=DEV)[1:257].view(32, 8)  # 4 bytes past a 16-byte boundary
+    assert status_of(lambda: ctx.moe_route(odd, None, bufs["topk_idx"], bufs["topk_w"])) == B.MOE_ERR_INVALID_ARG
     ctx.moe_route(a["logits"], None, bufs["topk_idx"], bufs["topk_w"])
     ctx.moe_dispatch_layout(bufs["topk_idx"], None)  # layout only
     assert status_of(lambda: ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"])) == B.MOE_ERR_STATE
