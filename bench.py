@@ -340,7 +340,6 @@ def run_ours(args):
     l0 = ctx.moe_ctx_launch_count()
     ms_total = timed(args.steps, step)
     launches = ctx.moe_ctx_launch_count() - l0
-    clocks = sampler.stop() if rank == 0 else None
     ms_per_step = ms_total / args.steps
     value = world * T / (ms_per_step * 1e-3)
 
@@ -349,29 +348,32 @@ def run_ours(args):
     timed(args.steps, step)
     prof = ctx.moe_ctx_read_profile()
     ctx.moe_ctx_set_profiling(False)
+    clocks = sampler.stop() if rank == 0 else None  # sampled over the timed region and its per-kernel repeat
     stage_us = {n: (1e3 * ms / c if c else None) for n, (ms, c) in prof.items()}
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region
-    hx = [a["x"].cpu().pin_memory() for a in acts]
-    hl = [a["logits"].cpu().pin_memory() for a in acts]
-    hout = torch.empty(T, H, dtype=torch.bfloat16).pin_memory()
+    e2e_value = None
+    if not args.quick:
+        hx = [a["x"].cpu().pin_memory() for a in acts]
+        hl = [a["logits"].cpu().pin_memory() for a in acts]
+        hout = torch.empty(T, H, dtype=torch.bfloat16).pin_memory()
 
-    def host_step(i):
-        ctx.moe_layer_host(hl[i % n_in], None, hx[i % n_in], *wargs, hout)
+        def host_step(i):
+            ctx.moe_layer_host(hl[i % n_in], None, hx[i % n_in], *wargs, hout)
 
-    for i in range(max(3, args.warmup)):
-        host_step(i)
-    barrier()
-    t0 = time.perf_counter()
-    for i in range(args.steps):
-        host_step(i)
-    torch.cuda.synchronize(dev)
-    e2e_s = time.perf_counter() - t0
-    if dist is not None:
-        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = world * T * args.steps / e2e_s
+        for i in range(max(3, args.warmup)):
+            host_step(i)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(args.steps):
+            host_step(i)
+        torch.cuda.synchronize(dev)
+        e2e_s = time.perf_counter() - t0
+        if dist is not None:
+            t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        e2e_value = world * T * args.steps / e2e_s
     assert ctx.moe_ctx_status() == B.MOE_OK
 
     if rank != 0:
@@ -408,9 +410,11 @@ def run_ours(args):
     }
 
     # ---- CPU baseline: the oracle on a bounded sample, on this machine's host cores
-    cpu_rate, cpu_dt, cores = oracle_sample_rate(oracle_inputs(shape, args.ref_tokens))
-    cpu_baseline = {"value": cpu_rate, "unit": UNIT, "cores": cores, "kind": "oracle",
-                    "sample": f"all stages on the first {args.ref_tokens} of {T} tokens ({cpu_dt:.1f} s)"}
+    cpu_baseline = None
+    if not args.quick:
+        cpu_rate, cpu_dt, cores = oracle_sample_rate(oracle_inputs(shape, args.ref_tokens))
+        cpu_baseline = {"value": cpu_rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"all stages on the first {args.ref_tokens} of {T} tokens ({cpu_dt:.1f} s)"}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -425,7 +429,7 @@ def run_ours(args):
     ctx.close()
     del w, acts
     torch.cuda.empty_cache()
-    if world == 1 and not args.no_pd:
+    if world == 1 and not args.no_pd and not args.quick:
         try:
             line["decode"] = decode_under_prefill(torch, B, wl, dev, args.pd_iters, 20)
         except Exception as exc:  # the headline number stands even if the P/D section cannot run
@@ -446,6 +450,8 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=4096, help="tokens of the cpu_baseline oracle sample")
     ap.add_argument("--ref-step-tokens", type=int, default=256, help="tokens per step of the reference (oracle) arm")
     ap.add_argument("--no-pd", action="store_true", help="skip the decode-under-prefill section")
+    ap.add_argument("--quick", action="store_true",
+                    help="device-resident timed region only (no e2e, cpu_baseline or decode section): the profiling case")
     ap.add_argument("--pd-iters", type=int, default=200)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":

@@ -157,6 +157,26 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
  * Ends the step; a DECODE context then flips its double-buffer index. */
 moe_status moe_combine(moe_ctx* ctx, const float* topk_w, const int32_t* inv_perm, int32_t T, void* out);
 
+/* The same layout (stages a2-a4, no row movement) for callers that cannot allocate device memory and so
+ * cannot supply a context with a workspace: code that runs inside another framework's memory pool, a
+ * runtime that has handed every byte of the device to its own allocator, or any place where cudaMalloc is
+ * forbidden.  (The paper has no counterpart of this entry point; it exists for such embedders.)
+ * The scratch the large-T path needs lives in a 256 KiB array inside the library image, which each GPU that
+ * loads the library holds until the process exits.  Limit: ceil(T*top_k / 1024) * n_experts <= 65536
+ * (e.g. T*top_k <= 262144 at 256 experts); beyond it the call returns MOE_ERR_CAPACITY and does nothing.
+ * The call allocates nothing and frees nothing.  It works on the device that is current when it is called:
+ * the pointers and the stream must belong to that device.  The first call on each device looks up the
+ * array's device address (a host-side set-up step); make that first call before any stream capture begins.
+ * All calls on one device share the array: two calls whose kernels can overlap on the GPU (different
+ * streams without an ordering between them) race on it -- order them.  Nothing in the array needs clearing
+ * between calls: every cell is written before it is read within a call.
+ * Arguments and results are those of moe_dispatch_layout with x == NULL; all four output arrays are
+ * required (perm and inv_perm may be NULL only when T == 0).  An out-of-range expert index is dropped
+ * (inv_perm[f] = -1); there is no status word to report it to. */
+moe_status moe_dispatch_layout_static(const int32_t* topk_idx, int32_t T, int32_t top_k, int32_t n_experts,
+                                      int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm,
+                                      void* cuda_stream);
+
 /* One whole step with HOST activations: copies logits_host [T,E] fp32 and x_host [T,H] bf16
  * to the device (cudaMemcpyAsync into context-owned staging), runs a1..a9, copies out
  * [T,H] bf16 back to out_host and synchronises the stream before returning.  Pinned host

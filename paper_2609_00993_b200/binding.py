@@ -27,7 +27,8 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_CAPACITY", 3:
 # every symbol include/moe_pd.h declares
 EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_destroy", "moe_ctx_status",
            "moe_last_error", "moe_route", "moe_dispatch_layout", "moe_grouped_ffn", "moe_combine", "moe_layer_host",
-           "moe_ctx_debug_ptrs", "moe_ctx_launch_count", "moe_ctx_set_profiling", "moe_ctx_read_profile")
+           "moe_ctx_debug_ptrs", "moe_ctx_launch_count", "moe_ctx_set_profiling", "moe_ctx_read_profile",
+           "moe_dispatch_layout_static")
 
 STAGE_NAMES = ("route", "layout", "permute", "gemm1_swiglu", "gemm2", "shared_gemm1_swiglu", "shared_gemm2", "combine")
 
@@ -93,6 +94,8 @@ def load_library() -> ctypes.CDLL:
     lib.moe_ctx_set_profiling.argtypes = [vp, i32]
     lib.moe_ctx_read_profile.restype = i32
     lib.moe_ctx_read_profile.argtypes = [vp, ctypes.POINTER(moe_stage_times)]
+    lib.moe_dispatch_layout_static.restype = i32
+    lib.moe_dispatch_layout_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -275,3 +278,17 @@ def alloc_step_buffers(T: int, k: int, E: int, device) -> dict:
             "offsets": torch.empty(E + 1, dtype=torch.int32, device=device),
             "perm": torch.empty(n, dtype=torch.int32, device=device)[:T * k],
             "inv_perm": torch.empty(n, dtype=torch.int32, device=device)[:T * k]}
+
+
+def moe_dispatch_layout_static(topk_idx, n_experts, counts, offsets, perm, inv_perm, stream=None, T=None, top_k=None):
+    """Layout without a context and without any allocation (see the header): for embedders that cannot
+    allocate device memory.  Returns the moe_status code instead of raising, so callers can test limits."""
+    lib = load_library()
+    T = topk_idx.shape[0] if T is None else T
+    top_k = topk_idx.shape[1] if top_k is None else top_k
+    for n, t in (("topk_idx", topk_idx), ("counts", counts), ("offsets", offsets), ("perm", perm), ("inv_perm", inv_perm)):
+        _dev(t, torch.int32, n)
+    s = stream if stream is not None else torch.cuda.current_stream(topk_idx.device)
+    with torch.cuda.device(topk_idx.device):
+        return int(lib.moe_dispatch_layout_static(_ptr(topk_idx), T, top_k, n_experts, _ptr(counts), _ptr(offsets),
+                                                  _ptr(perm), _ptr(inv_perm), ctypes.c_void_p(s.cuda_stream)))

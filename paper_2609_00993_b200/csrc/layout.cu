@@ -5,6 +5,8 @@
 // and ranks equal experts inside a step with __match_any_sync, which keeps ascending slot order.
 //   small N (decode, low latency): ONE CTA does count -> scan -> place in shared memory, one launch.
 //   large N (prefill):             count per chunk -> scan over chunks and experts -> place per chunk.
+#include <mutex>
+
 #include "kernels.h"
 
 namespace moe {
@@ -244,3 +246,61 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
 }
 
 }  // namespace moe
+
+// ------------------------------------------------------------------------------------------------
+// Dispatch layout for callers that cannot allocate.
+//
+// Some hosts of this library are not allowed to obtain device memory at the point where they need a
+// layout: code that lives inside another framework's memory pool and must not disturb it, or a runtime
+// that has handed all device memory to its own allocator and has no cudaMalloc left to call.  They cannot give a context a workspace either.  For
+// them the chunk histograms of the multi-CTA path live in this fixed array instead.  It is part of the
+// loaded module, so every GPU that loads the library holds these 256 KiB until the process exits.
+#include "../../include/moe_pd.h"
+
+namespace {
+
+constexpr int kStaticScratchInts = 64 * 1024;  // 256 KiB: up to ceil(N/1024) * E = 65536 histogram cells
+static __device__ __align__(256) int32_t g_static_layout_scratch[kStaticScratchInts];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+int32_t* g_static_scratch_addr[kMaxDevices] = {};  // device address of the array, per device ordinal
+
+}  // namespace
+
+extern "C" moe_status moe_dispatch_layout_static(const int32_t* topk_idx, int32_t T, int32_t top_k,
+                                                 int32_t n_experts, int32_t* counts, int32_t* offsets,
+                                                 int32_t* perm, int32_t* inv_perm, void* cuda_stream) {
+  if (T < 0 || top_k < 1 || n_experts < 1 || n_experts > 1024) return MOE_ERR_INVALID_ARG;
+  if (!counts || !offsets || (T > 0 && (!topk_idx || !perm || !inv_perm))) return MOE_ERR_INVALID_ARG;
+  const int64_t n_slots = (int64_t)T * top_k;
+  if (n_slots > ((int64_t)1 << 30)) return MOE_ERR_CAPACITY;
+  if (moe::layout_scratch_ints(n_slots, n_experts) > (size_t)kStaticScratchInts) return MOE_ERR_CAPACITY;
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MOE_ERR_CUDA;
+  int32_t* scratch = nullptr;
+  {
+    // Set-up, once per device, with that device current: in host code the array's name is only a
+    // stand-in for the symbol, so ask the runtime for the address the kernels must be given.
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_scratch_addr[dev] == nullptr) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_static_layout_scratch) != cudaSuccess || p == nullptr) {
+        (void)cudaGetLastError();
+        return MOE_ERR_CUDA;
+      }
+      g_static_scratch_addr[dev] = static_cast<int32_t*>(p);
+    }
+    scratch = g_static_scratch_addr[dev];
+  }
+  // Nothing in the scratch has to start at zero: the count kernel writes every histogram cell that the
+  // scan and place kernels read afterwards, so what the previous call left behind is never seen.
+  cudaError_t e = moe::launch_layout(topk_idx, n_slots, n_experts, counts, offsets, perm, inv_perm, scratch,
+                                     /*status=*/nullptr, static_cast<cudaStream_t>(cuda_stream), nullptr);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return MOE_ERR_CUDA;
+  }
+  return MOE_OK;
+}
