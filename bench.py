@@ -239,7 +239,8 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm):
     p_alone_ms = e0.elapsed_time(e1) / n_p
     res["prefill_alone_tokens_per_s"] = wl.C4_P.T / (p_alone_ms * 1e-3)
 
-    # concurrent: keep stream P saturated with P batches while the D steps are timed one by one
+    # (1) concurrent, no segmentation: stream P kept saturated with whole P batches, D steps timed one by one;
+    #     only the stream priority separates the phases
     inflight = []
 
     def feed_p(i):
@@ -251,32 +252,94 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm):
         ev.record(sp)
         inflight.append(ev)
 
+    n_unseg = max(20, iters // 4)
     with torch.cuda.stream(sp):
         pe0 = torch.cuda.Event(enable_timing=True); pe0.record(sp)
-    t_host0 = time.perf_counter()
-    conc = time_d(iters, before=feed_p)
+    conc = time_d(n_unseg, before=feed_p)
     with torch.cuda.stream(sp):
         pe1 = torch.cuda.Event(enable_timing=True); pe1.record(sp)
     torch.cuda.synchronize(dev)
-    conc_wall = time.perf_counter() - t_host0
-    res["concurrent_us"] = {"p50": percentile(conc, 50), "p99": percentile(conc, 99), "max": max(conc)}
-    res["prefill_concurrent_tokens_per_s"] = wl.C4_P.T * iters / (pe0.elapsed_time(pe1) * 1e-3)
-    res["p99_ratio_concurrent_over_alone"] = res["concurrent_us"]["p99"] / res["alone_us"]["p99"]
+    res["concurrent_unsegmented_us"] = {"p50": percentile(conc, 50), "p99": percentile(conc, 99), "max": max(conc),
+                                        "prefill_tokens_per_s": wl.C4_P.T * n_unseg / (pe0.elapsed_time(pe1) * 1e-3)}
+    inflight.clear()
 
-    # serial: P then D on one timeline (D waits for the P batch before it)
+    # (2) segment turnstile: P is cut at safe boundaries (one launch per `span` experts); the host controller
+    #     admits the waiting D step at the first boundary after it became ready and holds P's next segment
+    #     until that D step is done.  Per iteration one P batch and one D step, as in config 4.
+    #     Arrival model (worst case per step): the D batch becomes ready the moment a randomly chosen P
+    #     segment b starts executing, so it waits for the whole of segment b and is admitted at the boundary
+    #     after it.  The start event of the D step is therefore ordered after segment b-1, its kernels after
+    #     segment b, and P's segment b+1 after the D step.
+    import random
+
+    def turnstile_run(span, n_iter, seed=0):
+        rng = random.Random(seed)
+        st = {"target": 0, "i": 0, "prev": None, "evs": []}
+
+        def at_boundary(b, nb):
+            after_b = torch.cuda.Event()
+            after_b.record(sp)
+            if b == st["target"] % nb:
+                with torch.cuda.stream(sd):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    sd.wait_event(st["prev"])   # D becomes ready as segment b starts
+                    e0.record(sd)
+                    sd.wait_event(after_b)      # ... and is admitted at the boundary after it
+                    d_step(st["i"])
+                    e1.record(sd)
+                sp.wait_event(e1)               # P's next segment is released after the D step
+                st["evs"].append((e0, e1))
+            st["prev"] = after_b
+
+        ctx_p.moe_ctx_set_segments(span, at_boundary)
+        torch.cuda.synchronize(dev)
+        with torch.cuda.stream(sp):
+            t0 = torch.cuda.Event(enable_timing=True); t0.record(sp)
+        for i in range(n_iter):
+            st["target"], st["i"] = rng.randrange(1 << 20), i
+            start = torch.cuda.Event()
+            start.record(sp)
+            st["prev"] = start
+            p_step(i)
+            if i % 4 == 3:
+                torch.cuda.synchronize(dev)  # keep the host at most a few batches ahead of the device
+        with torch.cuda.stream(sp):
+            t1 = torch.cuda.Event(enable_timing=True); t1.record(sp)
+        torch.cuda.synchronize(dev)
+        ctx_p.moe_ctx_set_segments(0)
+        us = [1e3 * a.elapsed_time(b) for a, b in st["evs"]]
+        return {"span_experts": span, "d_steps": len(us), "p50": percentile(us, 50), "p99": percentile(us, 99),
+                "max": max(us), "prefill_tokens_per_s": wl.C4_P.T * n_iter / (t0.elapsed_time(t1) * 1e-3),
+                "p99_over_alone": percentile(us, 99) / res["alone_us"]["p99"]}
+
+    turnstile_run(16, 8)  # warm-up
+    res["turnstile"] = [turnstile_run(span, iters if span == 16 else max(20, iters // 4)) for span in (8, 16, 32, 64)]
+    best = [r for r in res["turnstile"] if r["span_experts"] == 16][0]
+    res["concurrent_us"] = {"p50": best["p50"], "p99": best["p99"], "max": best["max"],
+                            "policy": "segment turnstile, 16 experts per P segment"}
+    res["prefill_concurrent_tokens_per_s"] = best["prefill_tokens_per_s"]
+    res["p99_ratio_concurrent_over_alone"] = best["p99_over_alone"]
+
+    # (3) serial: the D batch becomes ready as a whole (unsegmented) P batch starts and waits for all of it
     ser = []
     for i in range(max(8, iters // 10)):
+        start = torch.cuda.Event()
+        start.record(sp)
         p_step(i)
-        sd.wait_stream(sp)
         with torch.cuda.stream(sd):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(sd); d_step(i); e1.record(sd)
+            sd.wait_event(start)
+            e0.record(sd)
+            sd.wait_stream(sp)
+            d_step(i)
+            e1.record(sd)
         sp.wait_stream(sd)
         ser.append((e0, e1))
     torch.cuda.synchronize(dev)
     ser_us = [1e3 * a.elapsed_time(b) for a, b in ser]
     res["serial_us"] = {"p50": percentile(ser_us, 50), "p99": percentile(ser_us, 99),
-                        "d_wait_behind_p_ms": p_alone_ms}
+                        "note": "D ready at the start of an unsegmented P batch, runs after it"}
+    res["prefill_serial_tokens_per_s"] = wl.C4_P.T / ((p_alone_ms + res["alone_us"]["p50"] * 1e-3) * 1e-3)
     res["iterations"] = iters
     res["workload"] = "C4: P T=4096 on stream P || D T=64 on stream D (high priority), DeepSeek-V3-shaped layer"
     ctx_p.close(); ctx_d.close()

@@ -150,6 +150,18 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
 moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_down, const void* x,
                            const void* ws_gate_up, const void* ws_down, int32_t T);
 
+/* Prefill segmentation.  A single P execution spans several D iterations, so the paper divides P into
+ * segments delimited by backend-provided boundaries (Section "In-Place P/D Execution"; the span K of Section
+ * "Prefill Policy Interface").  With experts_per_segment > 0, moe_grouped_ffn enqueues each routed GEMM pass
+ * as one launch per group of that many experts (the shared-expert passes are segments of their own) and
+ * calls `fn(user, i, n)` on the calling host thread right after segment i of n has been enqueued: a safe
+ * point at which the caller's controller may enqueue a D step on another context and order the streams (for
+ * instance make this context's stream wait for an event of the D stream) before the next segment is
+ * enqueued.  The callback must not call into THIS context.  Results are bit-identical to the unsegmented
+ * call.  experts_per_segment = 0 switches segmentation off; fn may be NULL. */
+typedef void (*moe_boundary_fn)(void* user, int32_t boundary, int32_t n_boundaries);
+moe_status moe_ctx_set_segments(moe_ctx* ctx, int32_t experts_per_segment, moe_boundary_fn fn, void* user);
+
 /* Stage a9 -- weighted combine back to token order:
  *   out[t,:] = sum_j topk_w[t,j] * y_perm[inv_perm[t*k+j],:]  (+ y_shared[t,:]),  fp32 sum, bf16 store.
  * topk_w [T,k] fp32; inv_perm [N] int32 or NULL to use the layout of this step kept by the

@@ -28,7 +28,9 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_CAPACITY", 3:
 EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_destroy", "moe_ctx_status",
            "moe_last_error", "moe_route", "moe_dispatch_layout", "moe_grouped_ffn", "moe_combine", "moe_layer_host",
            "moe_ctx_debug_ptrs", "moe_ctx_launch_count", "moe_ctx_set_profiling", "moe_ctx_read_profile",
-           "moe_dispatch_layout_static")
+           "moe_dispatch_layout_static", "moe_ctx_set_segments")
+
+BOUNDARY_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32)
 
 STAGE_NAMES = ("route", "layout", "permute", "gemm1_swiglu", "gemm2", "shared_gemm1_swiglu", "shared_gemm2", "combine")
 
@@ -94,6 +96,8 @@ def load_library() -> ctypes.CDLL:
     lib.moe_ctx_set_profiling.argtypes = [vp, i32]
     lib.moe_ctx_read_profile.restype = i32
     lib.moe_ctx_read_profile.argtypes = [vp, ctypes.POINTER(moe_stage_times)]
+    lib.moe_ctx_set_segments.restype = i32
+    lib.moe_ctx_set_segments.argtypes = [vp, i32, BOUNDARY_FN, vp]
     lib.moe_dispatch_layout_static.restype = i32
     lib.moe_dispatch_layout_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     _lib = lib
@@ -186,6 +190,14 @@ class MoeContext:
 
     def moe_ctx_launch_count(self) -> int:
         return int(self.lib.moe_ctx_launch_count(self.handle))
+
+    def moe_ctx_set_segments(self, experts_per_segment: int, fn=None):
+        """fn(boundary, n_boundaries) is called on the host after each P segment has been enqueued."""
+        if fn is None:
+            self._boundary_cb = ctypes.cast(None, BOUNDARY_FN)
+        else:
+            self._boundary_cb = BOUNDARY_FN(lambda _user, i, n: fn(i, n))  # kept alive by the context
+        self._check(self.lib.moe_ctx_set_segments(self.handle, experts_per_segment, self._boundary_cb, None))
 
     def moe_ctx_set_profiling(self, enabled: bool):
         self._check(self.lib.moe_ctx_set_profiling(self.handle, int(bool(enabled))))

@@ -124,6 +124,10 @@ struct moe_ctx {
   int32_t* inv_perm;
   cudaEvent_t done;  // recorded after the last enqueue of every call
   int64_t launches;
+  // prefill segmentation (off by default)
+  int seg_experts;
+  moe_boundary_fn boundary_fn;
+  void* boundary_user;
   // per-stage timing (off by default): event pairs recorded around each stage's launches
   bool profiling;
   struct Span { cudaEvent_t beg, end; int stage; };
@@ -254,6 +258,9 @@ moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspa
   ctx->launches = 0;
   ctx->profiling = false;
   ctx->spans_used = 0;
+  ctx->seg_experts = 0;
+  ctx->boundary_fn = nullptr;
+  ctx->boundary_user = nullptr;
   ctx->err[0] = 0;
   ctx->status = reinterpret_cast<int*>(ctx->ws);
   for (int s = 0; s < l.n_sets; ++s) carve_set(*cfg, ctx->ws + kStatusBlock + (size_t)s * l.set_bytes, &ctx->sets[s]);
@@ -411,15 +418,31 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
   int n = 0;
   cudaError_t e = cudaSuccess;
   if (T > 0) {
+    // One launch per pass, or one per group of seg_experts experts with a boundary call after each.
+    const int span = (ctx->seg_experts > 0 && ctx->seg_experts < c.n_experts) ? ctx->seg_experts : c.n_experts;
+    const int routed_segs = (c.n_experts + span - 1) / span;
+    const int n_bound = 2 * routed_segs + (shared ? 2 : 0);
+    int bound = 0;
+    auto boundary = [&]() {
+      if (ctx->seg_experts > 0 && ctx->boundary_fn) {
+        cudaEventRecord(ctx->done, ctx->stream);
+        ctx->boundary_fn(ctx->boundary_user, bound, n_bound);
+      }
+      ++bound;
+    };
     moe::GemmProblem g1{b.x_perm, w_gate_up, b.act, ctx->offsets, 0, Ncap, N, c.n_experts, c.inter, c.hidden, true};
-    {
-      StageTimer tm(ctx, 3);
-      e = run_gemm(ctx, g1, T, &n);
-    }
-    if (e == cudaSuccess) {
-      moe::GemmProblem g2{b.act, w_down, b.y_perm, ctx->offsets, 0, Ncap, N, c.n_experts, c.hidden, c.inter, false};
-      StageTimer tm(ctx, 4);
-      e = run_gemm(ctx, g2, T, &n);
+    moe::GemmProblem g2{b.act, w_down, b.y_perm, ctx->offsets, 0, Ncap, N, c.n_experts, c.hidden, c.inter, false};
+    for (int pass = 0; pass < 2 && e == cudaSuccess; ++pass) {
+      moe::GemmProblem& g = pass == 0 ? g1 : g2;
+      for (int e0 = 0; e0 < c.n_experts && e == cudaSuccess; e0 += span) {
+        g.e_begin = e0;
+        g.e_end = e0 + span < c.n_experts ? e0 + span : c.n_experts;
+        {
+          StageTimer tm(ctx, pass == 0 ? 3 : 4);
+          e = run_gemm(ctx, g, T, &n);
+        }
+        if (e == cudaSuccess) boundary();
+      }
     }
     if (e == cudaSuccess && shared) {
       moe::GemmProblem s1{x, ws_gate_up, b.act_shared, nullptr, T, T, T, 1, c.shared_inter, c.hidden, true};
@@ -428,9 +451,13 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
         e = run_gemm(ctx, s1, T, &n);
       }
       if (e == cudaSuccess) {
+        boundary();
         moe::GemmProblem s2{b.act_shared, ws_down, b.y_shared, nullptr, T, T, T, 1, c.hidden, c.shared_inter, false};
-        StageTimer tm(ctx, 6);
-        e = run_gemm(ctx, s2, T, &n);
+        {
+          StageTimer tm(ctx, 6);
+          e = run_gemm(ctx, s2, T, &n);
+        }
+        if (e == cudaSuccess) boundary();
       }
     }
   }
@@ -492,6 +519,16 @@ moe_status moe_layer_host(moe_ctx* ctx, const float* logits_host, const float* s
   if (T > 0) e = cudaMemcpyAsync(out_host, b.out_stage, x_bytes, cudaMemcpyDeviceToHost, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "device-to-host copy");
+  return MOE_OK;
+}
+
+moe_status moe_ctx_set_segments(moe_ctx* ctx, int32_t experts_per_segment, moe_boundary_fn fn, void* user) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (experts_per_segment < 0) return fail(ctx, MOE_ERR_INVALID_ARG, "experts_per_segment < 0");
+  if (ctx->state != ST_IDLE) return fail(ctx, MOE_ERR_STATE, "segmentation can only change between steps");
+  ctx->seg_experts = experts_per_segment;
+  ctx->boundary_fn = fn;
+  ctx->boundary_user = user;
   return MOE_OK;
 }
 

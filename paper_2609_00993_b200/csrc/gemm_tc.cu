@@ -40,9 +40,10 @@ constexpr int kSmemBudget = 227 * 1024;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 struct TcParams {
-  const int32_t* offsets;  // [E+1] or nullptr (single group of fixed_rows rows)
+  const int32_t* offsets;  // [E+1] (already advanced to the first expert of the launch) or nullptr
   int32_t fixed_rows;
-  int32_t E;
+  int32_t E;               // experts covered by this launch
+  int32_t e_base;          // index of the launch's first expert in the weight tensor
   int32_t n_feat;          // output features (I for the gated pass, H for the down pass)
   int32_t K;
   __nv_bfloat16* out;      // [rows, n_feat]
@@ -281,8 +282,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           const uint32_t full = bar_full + 8u * s;
           const uint32_t st = base_addr + s * (uint32_t)stage_bytes;
           mbar_expect_tx(full, (uint32_t)stage_bytes);
-          tma_load_3d(st, &map_w, full, kb * kBlockK, w_row0, t.e);
-          tma_load_3d(st + kWBoxBytes, &map_w, full, kb * kBlockK, w_row1, t.e);
+          tma_load_3d(st, &map_w, full, kb * kBlockK, w_row0, p.e_base + t.e);
+          tma_load_3d(st + kWBoxBytes, &map_w, full, kb * kBlockK, w_row1, p.e_base + t.e);
           tma_load_2d(st + 2 * kWBoxBytes, &map_x, full, kb * kBlockK, t.row0);
         }
       }
@@ -499,10 +500,14 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int
     if (!encode_map(&mw, p.W, 3, dims, str, box)) return cudaErrorInvalidValue;
   }
 
+  const int e_begin = p.offsets ? p.e_begin : 0;
+  const int e_end = (p.offsets && p.e_end >= 0) ? p.e_end : groups;
+  if (e_begin < 0 || e_end > groups || e_begin >= e_end) return cudaErrorInvalidValue;
   TcParams prm;
-  prm.offsets = p.offsets;
+  prm.offsets = p.offsets ? p.offsets + e_begin : nullptr;
   prm.fixed_rows = p.fixed_rows;
-  prm.E = groups;
+  prm.E = e_end - e_begin;
+  prm.e_base = e_begin;
   prm.n_feat = p.n_feat;
   prm.K = p.K;
   prm.out = static_cast<__nv_bfloat16*>(p.out);
@@ -510,7 +515,7 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int
   prm.x_tile_bytes = row_tile * kBlockK * 2;
   prm.status = status;
   const int stage_bytes = 2 * kWBoxBytes + prm.x_tile_bytes;
-  const size_t tail = (2 * kMaxStages + 4) * sizeof(uint64_t) + 2 * sizeof(uint32_t) + 2 * (size_t)(groups + 1) * sizeof(int);
+  const size_t tail = (2 * kMaxStages + 4) * sizeof(uint64_t) + 2 * sizeof(uint32_t) + 2 * (size_t)(prm.E + 1) * sizeof(int);
   int stages = (int)((kSmemBudget - 1024 - (int)tail) / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) return cudaErrorNotSupported;
@@ -519,7 +524,7 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int
 
   const int feat_per_tile = p.gated ? 128 : 256;
   const int64_t n_ft = (p.n_feat + feat_per_tile - 1) / feat_per_tile;
-  const int64_t row_tiles = p.rows_bound / row_tile + (groups < p.rows_bound ? groups : p.rows_bound);
+  const int64_t row_tiles = p.rows_bound / row_tile + (prm.E < p.rows_bound ? prm.E : p.rows_bound);
   int64_t tiles = row_tiles * n_ft;
   int grid = (int)(tiles < (int64_t)max_ctas ? tiles : (int64_t)max_ctas);
   if (grid < 1) grid = 1;

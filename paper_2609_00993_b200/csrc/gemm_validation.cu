@@ -94,9 +94,13 @@ cudaError_t launch_gemm_validation(const GemmProblem& p, cudaStream_t stream, in
   const auto* A = static_cast<const __nv_bfloat16*>(p.A);
   const auto* W = static_cast<const __nv_bfloat16*>(p.W);
   auto* out = static_cast<__nv_bfloat16*>(p.out);
-  const int E = p.offsets ? p.E : 1;
-  if (p.gated) gemm_validation_kernel<true><<<grid, 256, 0, stream>>>(A, W, out, p.offsets, p.fixed_rows, E, p.n_feat, p.K);
-  else gemm_validation_kernel<false><<<grid, 256, 0, stream>>>(A, W, out, p.offsets, p.fixed_rows, E, p.n_feat, p.K);
+  const int e_begin = p.offsets ? p.e_begin : 0;
+  const int e_end = (p.offsets && p.e_end >= 0) ? p.e_end : (int)groups;
+  const int E = e_end - e_begin;  // experts of this launch
+  const int32_t* offs = p.offsets ? p.offsets + e_begin : nullptr;
+  W += (size_t)e_begin * (size_t)(p.gated ? 2 : 1) * p.n_feat * p.K;
+  if (p.gated) gemm_validation_kernel<true><<<grid, 256, 0, stream>>>(A, W, out, offs, p.fixed_rows, E, p.n_feat, p.K);
+  else gemm_validation_kernel<false><<<grid, 256, 0, stream>>>(A, W, out, offs, p.fixed_rows, E, p.n_feat, p.K);
   cudaError_t err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;

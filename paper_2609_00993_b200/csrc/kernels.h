@@ -45,10 +45,12 @@ struct GemmProblem {
   int32_t fixed_rows;      // rows when offsets == nullptr
   int64_t rows_cap;        // rows addressable in A / out (capacity of the buffers)
   int64_t rows_bound;      // upper bound on the rows actually routed this call (T*k or T)
-  int32_t E;
+  int32_t E;               // experts in W and offsets
   int32_t n_feat;
   int32_t K;
   bool gated;
+  int32_t e_begin = 0;     // this launch covers experts [e_begin, e_end) only (a prefill segment);
+  int32_t e_end = -1;      // e_end < 0 means E
 };
 
 cudaError_t launch_gemm_validation(const GemmProblem& p, cudaStream_t stream, int* n_launches);

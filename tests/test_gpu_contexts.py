@@ -146,3 +146,59 @@ def test_prefill_traffic_cannot_disturb_a_decode_step():
     assert torch.equal(out, alone)
     assert torch.equal(bufs["perm"], bufs_alone["perm"])
     p.close(); d.close()
+
+
+def test_prefill_segments_are_bit_identical_and_boundaries_are_monotone():
+    shape = wl.LayerShape("t", T=600, H=512, E=16, k=4, I=256, shared_I=128)
+    w, a = wl.make_weights(shape, 1, DEV), wl.make_activations(shape, 2, DEV)
+    ctx = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 600, B.MOE_PHASE_PREFILL))
+    torch.cuda.synchronize()
+    whole, _ = ctx.layer(a["x"], a["logits"], None, w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+    torch.cuda.synchronize()
+    for span in (1, 5, 16, 64):
+        seen = []
+        ctx.moe_ctx_set_segments(span, lambda i, n: seen.append((i, n)))
+        out, _ = ctx.layer(a["x"], a["logits"], None, w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+        torch.cuda.synchronize()
+        assert torch.equal(out, whole), f"span {span}"
+        segs = -(-16 // min(span, 16))
+        assert seen == [(i, 2 * segs + 2) for i in range(2 * segs + 2)], f"span {span}: {seen}"
+    ctx.moe_ctx_set_segments(0)
+    assert ctx.moe_ctx_status() == B.MOE_OK
+    ctx.close()
+
+
+def test_decode_step_admitted_at_a_prefill_boundary():
+    """The host controller enqueues a D step at a P boundary and holds P's next segment until D is done:
+    both phases give exactly the results they give alone."""
+    shape = wl.LayerShape("t", T=48, H=512, E=16, k=4, I=256, shared_I=128)
+    pshape = shape.with_tokens(2048)
+    w = wl.make_weights(shape, 1, DEV)
+    ad, ap = wl.make_activations(shape, 2, DEV), wl.make_activations(pshape, 3, DEV)
+    sp, sd = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    d = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 48, B.MOE_PHASE_DECODE), stream=sd)
+    p = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 2048, B.MOE_PHASE_PREFILL), stream=sp)
+    wargs = (w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+    torch.cuda.synchronize()
+    d_alone, _ = d.layer(ad["x"], ad["logits"], None, *wargs)
+    p_alone, _ = p.layer(ap["x"], ap["logits"], None, *wargs)
+    torch.cuda.synchronize()
+    d_out = torch.empty_like(d_alone)
+    admitted = []
+
+    def turnstile(i, n):
+        if i % 3 == 0:  # admit one D step at every third boundary
+            d.layer(ad["x"], ad["logits"], None, *wargs, out=d_out)
+            ev = torch.cuda.Event()
+            ev.record(sd)
+            sp.wait_event(ev)  # the next P segment starts after this D step
+            admitted.append(i)
+
+    p.moe_ctx_set_segments(4, turnstile)
+    p_out, _ = p.layer(ap["x"], ap["logits"], None, *wargs)
+    torch.cuda.synchronize()
+    assert len(admitted) == 4 and admitted[0] == 0  # 2 * 4 + 2 = 10 boundaries
+    assert torch.equal(p_out, p_alone) and torch.equal(d_out, d_alone)
+    assert p.moe_ctx_status() == B.MOE_OK and d.moe_ctx_status() == B.MOE_OK
+    p.moe_ctx_set_segments(0)
+    p.close(); d.close()
