@@ -38,6 +38,7 @@ constexpr int kMmaWarp = 5;
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kEpiStagingBytes = kEpilogueWarps * 32 * 128;  // per-warp 32 x 128-byte staging tiles
 
 struct TcParams {
   const int32_t* offsets;  // [E+1] (already advanced to the first expert of the launch) or nullptr
@@ -196,14 +197,16 @@ __device__ __forceinline__ Tile decode_tile(int tile, int n_ft, int E, const int
 template <bool SWAP, bool GATED>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                       const TcParams p) {
+                       const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
-  // carve: [stages: W box0 | W box1 | X tile] | barriers | tmem slot | abort | prefix[E+1] | seg[E+1]
+  // carve: [stages] | epilogue staging (large-M) | barriers | tmem slot | abort | prefix[E+1] | seg[E+1]
+  //   stage: W box0 | W box1 | X tile
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
   uint8_t* base = smem_raw + (base_addr - raw_addr);
   const int stage_bytes = 2 * kWBoxBytes + p.x_tile_bytes;
-  uint8_t* after = base + (size_t)p.n_stages * stage_bytes;
+  uint8_t* epi_smem = base + (size_t)p.n_stages * stage_bytes;  // kEpilogueWarps x 4 KB, large-M only
+  uint8_t* after = epi_smem + (SWAP ? 0 : kEpiStagingBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(after);  // full[S], empty[S], tmem_full[2], tmem_empty[2]
   const uint32_t bar_full = smem_u32(bars);
   const uint32_t bar_empty = bar_full + 8u * p.n_stages;
@@ -215,6 +218,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   int* seg = prefix + (p.E + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int unit = (int)blockIdx.x, n_units = (int)gridDim.x;
+  const int tile_rows = p.row_tile;  // token rows per tile of the list
   constexpr int kFeatPerTile = GATED ? 128 : 256;
   const int n_ft = (p.n_feat + kFeatPerTile - 1) / kFeatPerTile;
   const int num_kb = (p.K + kBlockK - 1) / kBlockK;
@@ -235,7 +240,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         seg[e] = beg;
         if (e == p.E - 1) seg[p.E] = beg + cnt;
       }
-      const int tiles = (cnt + p.row_tile - 1) / p.row_tile;
+      const int tiles = (cnt + tile_rows - 1) / tile_rows;
       int incl = tiles;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
@@ -272,8 +277,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, p.row_tile);
+      for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
+        const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, tile_rows);
         const int w_row0 = t.ft * kFeatPerTile;
         const int w_row1 = GATED ? p.n_feat + t.ft * kFeatPerTile : w_row0 + kWBoxRows;
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
@@ -297,8 +302,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     if (lane == 0) {
       uint32_t it = 0, tile_iter = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_iter) {
-        const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, p.row_tile);
+      for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++tile_iter) {
+        const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, tile_rows);
         const uint32_t as = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
         if (!mbar_wait(bar_tempty + 8u * as, aph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
@@ -339,12 +344,18 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     uint32_t tile_iter = 0;
     bool ok = true;
     const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_iter) {
-      const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, p.row_tile);
+    for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++tile_iter) {
+      const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, tile_rows);
       const uint32_t as = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
+      auto release_acc = [&]() {  // hand the accumulator stage back to the MMA issuer
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty + 8u * as);
+      };
       if (!mbar_wait(bar_tfull + 8u * as, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t d0 = tmem_base + as * acc_cols + lane_base;
+      bool released = false;  // has this warp already handed the accumulator stage back?
       if (SWAP) {
         // lane = weight row (output feature), column = token
         const int fl = warp * 32 + lane;
@@ -370,42 +381,56 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           }
         }
       } else {
-        // lane = token row, column = output feature
-        const int r = warp * 32 + lane;
-        const bool row_ok = r < t.rows;
-        __nv_bfloat16* orow = p.out + (size_t)(t.row0 + r) * p.n_feat + (size_t)t.ft * kFeatPerTile;
-        constexpr int kChunks = kFeatPerTile / 32;
-        for (int c = 0; c < kChunks; ++c) {
-          const int f0 = t.ft * kFeatPerTile + c * 32;
+        // lane = token row, column = output feature.  Two 32-column chunks (128 bytes of a row) at a time go
+        // through a per-warp staging tile in shared memory (16-byte pieces XOR-swizzled by row, conflict-free
+        // both ways), so that every global store instruction writes four whole 128-byte lines instead of
+        // touching 32 different rows.
+        constexpr int kPairs = kFeatPerTile / 64;
+        uint8_t* stage_tile = epi_smem + warp * 4096;  // 32 rows x 128 bytes
+        const int rows_here = t.rows - warp * 32;       // rows of this warp's 32 that are valid (may be <= 0)
+        for (int pc = 0; pc < kPairs; ++pc) {
+          const int f0 = t.ft * kFeatPerTile + pc * 64;
           if (f0 >= p.n_feat) break;  // uniform across the CTA
-          uint32_t ra[32];
-          uint32_t packed[16];
-          tmem_ld32(d0 + (uint32_t)(c * 32), ra);
-          if (GATED) {
-            uint32_t rb[32];
-            tmem_ld32(d0 + (uint32_t)(128 + c * 32), rb);
-            tmem_ld_wait();
+          uint32_t packed[32];
 #pragma unroll
-            for (int i = 0; i < 16; ++i)
-              packed[i] = pack_bf16(silu_mul(__uint_as_float(ra[2 * i]), __uint_as_float(rb[2 * i])),
-                                    silu_mul(__uint_as_float(ra[2 * i + 1]), __uint_as_float(rb[2 * i + 1])));
-          } else {
-            tmem_ld_wait();
+          for (int h = 0; h < 2; ++h) {
+            uint32_t ra[32];
+            tmem_ld32(d0 + (uint32_t)(pc * 64 + h * 32), ra);
+            if (GATED) {
+              uint32_t rb[32];
+              tmem_ld32(d0 + (uint32_t)(128 + pc * 64 + h * 32), rb);
+              tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 16; ++i) packed[i] = pack_bf16(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1]));
+              for (int i = 0; i < 16; ++i)
+                packed[h * 16 + i] = pack_bf16(silu_mul(__uint_as_float(ra[2 * i]), __uint_as_float(rb[2 * i])),
+                                               silu_mul(__uint_as_float(ra[2 * i + 1]), __uint_as_float(rb[2 * i + 1])));
+            } else {
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                packed[h * 16 + i] = pack_bf16(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1]));
+            }
           }
-          if (row_ok) {
-            uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-              if (f0 + q * 8 < p.n_feat)
-                dst[q] = make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+          if (pc == kPairs - 1 || f0 + 64 >= p.n_feat) {
+            release_acc();  // the accumulator has been read completely: hand it back before the stores go out
+            released = true;
           }
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<uint4*>(stage_tile + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+          __syncwarp();
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + (lane >> 3), piece = lane & 7;
+            const uint4 v = *reinterpret_cast<const uint4*>(stage_tile + rr * 128 + ((piece ^ (rr & 7)) << 4));
+            if (rr < rows_here && f0 + piece * 8 < p.n_feat)
+              *reinterpret_cast<uint4*>(p.out + (size_t)(t.row0 + warp * 32 + rr) * p.n_feat + f0 + piece * 8) = v;
+          }
+          __syncwarp();
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty + 8u * as);
+      if (!released) release_acc();
     }
     if (!ok && lane == 0) {
       *abort_flag = 1;
@@ -448,10 +473,9 @@ bool encode_map(CUtensorMap* map, const void* base, int rank, const uint64_t* di
   return r == CUDA_SUCCESS;
 }
 
-template <bool SWAP, bool GATED>
-cudaError_t launch_variant(const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& prm, int grid, size_t smem,
-                           cudaStream_t stream) {
-  auto kern = grouped_gemm_tc_kernel<SWAP, GATED>;
+template <typename Kernel>
+cudaError_t launch_variant(Kernel kern, const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& prm, int grid,
+                           size_t smem, cudaStream_t stream) {
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
   kern<<<grid, kThreads, smem, stream>>>(mx, mw, prm);
@@ -515,7 +539,8 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int
   prm.x_tile_bytes = row_tile * kBlockK * 2;
   prm.status = status;
   const int stage_bytes = 2 * kWBoxBytes + prm.x_tile_bytes;
-  const size_t tail = (2 * kMaxStages + 4) * sizeof(uint64_t) + 2 * sizeof(uint32_t) + 2 * (size_t)(prm.E + 1) * sizeof(int);
+  const size_t tail = (swap_ab ? 0 : kEpiStagingBytes) + (2 * kMaxStages + 4) * sizeof(uint64_t) +
+                      2 * sizeof(uint32_t) + 2 * (size_t)(prm.E + 1) * sizeof(int);
   int stages = (int)((kSmemBudget - 1024 - (int)tail) / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < 2) return cudaErrorNotSupported;
@@ -525,15 +550,15 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int
   const int feat_per_tile = p.gated ? 128 : 256;
   const int64_t n_ft = (p.n_feat + feat_per_tile - 1) / feat_per_tile;
   const int64_t row_tiles = p.rows_bound / row_tile + (prm.E < p.rows_bound ? prm.E : p.rows_bound);
-  int64_t tiles = row_tiles * n_ft;
+  const int64_t tiles = row_tiles * n_ft;
+
   int grid = (int)(tiles < (int64_t)max_ctas ? tiles : (int64_t)max_ctas);
   if (grid < 1) grid = 1;
-
   cudaError_t err;
-  if (swap_ab) err = p.gated ? launch_variant<true, true>(mx, mw, prm, grid, smem, stream)
-                             : launch_variant<true, false>(mx, mw, prm, grid, smem, stream);
-  else err = p.gated ? launch_variant<false, true>(mx, mw, prm, grid, smem, stream)
-                     : launch_variant<false, false>(mx, mw, prm, grid, smem, stream);
+  if (swap_ab) err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true>, mx, mw, prm, grid, smem, stream)
+                             : launch_variant(grouped_gemm_tc_kernel<true, false>, mx, mw, prm, grid, smem, stream);
+  else err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true>, mx, mw, prm, grid, smem, stream)
+                     : launch_variant(grouped_gemm_tc_kernel<false, false>, mx, mw, prm, grid, smem, stream);
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }

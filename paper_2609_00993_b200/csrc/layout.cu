@@ -20,14 +20,26 @@ __device__ __forceinline__ void flag_status(int* status, int code) {
   if (status != nullptr) atomicCAS(status, kStOk, code);
 }
 
+constexpr int kBatch = 8;  // steps of 32 slots whose index loads are issued together (latency hiding)
+
 // Counts one chunk [f0, f1) into hist[0..E) (shared memory, zeroed by the caller).
 __device__ __forceinline__ void count_chunk(const int32_t* __restrict__ topk_idx, int64_t f0, int64_t f1, int E,
                                             int* hist, int* status) {
   const int lane = threadIdx.x & 31;
-  for (int64_t f = f0 + lane; f < f1; f += 32) {
-    const int e = topk_idx[f];
-    if (e >= 0 && e < E) atomicAdd(&hist[e], 1);  // integer adds commute: the count is order-independent
-    else flag_status(status, kStBadIndex);
+  for (int64_t base = f0; base < f1; base += 32 * kBatch) {
+    int ev[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int64_t f = base + 32 * u + lane;
+      ev[u] = (f < f1) ? __ldg(topk_idx + f) : 0;
+    }
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      if (base + 32 * u + lane >= f1) continue;
+      const int e = ev[u];
+      if (e >= 0 && e < E) atomicAdd(&hist[e], 1);  // integer adds commute: the count is order-independent
+      else flag_status(status, kStBadIndex);
+    }
   }
 }
 
@@ -36,21 +48,31 @@ __device__ __forceinline__ void place_chunk(const int32_t* __restrict__ topk_idx
                                             int* run, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
   const int lane = threadIdx.x & 31;
   const unsigned lt_mask = (1u << lane) - 1u;
-  for (int64_t base = f0; base < f1; base += 32) {
-    const int64_t f = base + lane;
-    int e = -1;
-    if (f < f1) e = topk_idx[f];
-    const bool valid = (e >= 0 && e < E);
-    const int keyv = valid ? e : (E + lane);  // invalid lanes never group with anyone
-    const unsigned peers = __match_any_sync(0xffffffffu, keyv);
-    int p = -1;
-    if (valid) p = run[e] + __popc(peers & lt_mask);
-    __syncwarp();
-    if (valid && (peers & lt_mask) == 0u) run[e] += __popc(peers);  // the lowest lane of a group advances it
-    __syncwarp();
-    if (f < f1) {
-      inv_perm[f] = p;
-      if (valid) perm[p] = (int32_t)f;
+  for (int64_t base0 = f0; base0 < f1; base0 += 32 * kBatch) {
+    int ev[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int64_t f = base0 + 32 * u + lane;
+      ev[u] = (f < f1) ? __ldg(topk_idx + f) : -1;
+    }
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      const int64_t base = base0 + 32 * u;
+      if (base >= f1) break;  // uniform across the warp
+      const int64_t f = base + lane;
+      const int e = ev[u];
+      const bool valid = (e >= 0 && e < E);
+      const int keyv = valid ? e : (E + lane);  // invalid lanes never group with anyone
+      const unsigned peers = __match_any_sync(0xffffffffu, keyv);
+      int p = -1;
+      if (valid) p = run[e] + __popc(peers & lt_mask);
+      __syncwarp();
+      if (valid && (peers & lt_mask) == 0u) run[e] += __popc(peers);  // the lowest lane of a group advances it
+      __syncwarp();
+      if (f < f1) {
+        inv_perm[f] = p;
+        if (valid) perm[p] = (int32_t)f;
+      }
     }
   }
 }

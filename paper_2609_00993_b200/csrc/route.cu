@@ -1,7 +1,8 @@
 // Stage a1: top-k routing over given router logits.  One warp per token; each lane keeps
 // ceil(E/32) selection keys in registers (128-bit loads when E is a multiple of 128), and k rounds of
 // a shuffle arg-max on (key descending, expert index ascending) pick the experts.  The routed weights
-// are a max-subtracted softmax over the k selected unbiased logits.
+// are a max-subtracted softmax over the k selected unbiased logits.  The arg-max uses the integer warp
+// reductions (redux.sync) on an order-preserving integer image of the key.
 #include "kernels.h"
 
 namespace moe {
@@ -9,9 +10,12 @@ namespace {
 
 constexpr int kWarpsPerBlock = 8;
 
-// Does candidate (v1, e1) come before (v0, e0) in the selection order?
-__device__ __forceinline__ bool comes_before(float v1, int e1, float v0, int e0) {
-  return (v1 > v0) || (v1 == v0 && e1 < e0);
+// Monotone map from a finite float to an unsigned integer (larger float <=> larger integer), so that the
+// warp arg-max can use the integer redux instructions.  -0.0 has been folded into +0.0 before the call,
+// which keeps the IEEE tie between the two zeros.
+__device__ __forceinline__ unsigned ordered_bits(float v) {
+  const unsigned u = __float_as_uint(v);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
 // VPT: keys per lane (power of two >= ceil(E/32)).  VEC: lanes own runs of 4 consecutive experts.
@@ -27,21 +31,21 @@ route_kernel(const float* __restrict__ logits, const float* __restrict__ bias, i
   // expert owned by this lane's i-th register; increasing in i so that "first wins" keeps the lower index
   auto expert_of = [&](int i) -> int { return VEC ? 128 * (i >> 2) + 4 * lane + (i & 3) : 32 * i + lane; };
 
-  float key[VPT];
+  unsigned key[VPT];  // ordered_bits(logit + bias)
   if constexpr (VEC) {
 #pragma unroll
     for (int q = 0; q < VPT / 4; ++q) {
       const int e0 = 128 * q + 4 * lane;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
       if (e0 < E) {
-        float4 v = *reinterpret_cast<const float4*>(row + e0);
+        v = *reinterpret_cast<const float4*>(row + e0);
         if (bias != nullptr) {
-          float4 b = *reinterpret_cast<const float4*>(bias + e0);
+          const float4 b = *reinterpret_cast<const float4*>(bias + e0);
           v.x = __fadd_rn(v.x, b.x); v.y = __fadd_rn(v.y, b.y); v.z = __fadd_rn(v.z, b.z); v.w = __fadd_rn(v.w, b.w);
         }
-        key[4 * q + 0] = v.x; key[4 * q + 1] = v.y; key[4 * q + 2] = v.z; key[4 * q + 3] = v.w;
-      } else {
-        key[4 * q + 0] = key[4 * q + 1] = key[4 * q + 2] = key[4 * q + 3] = 0.f;
       }
+      key[4 * q + 0] = ordered_bits(v.x + 0.0f); key[4 * q + 1] = ordered_bits(v.y + 0.0f);
+      key[4 * q + 2] = ordered_bits(v.z + 0.0f); key[4 * q + 3] = ordered_bits(v.w + 0.0f);
     }
   } else {
 #pragma unroll
@@ -52,14 +56,14 @@ route_kernel(const float* __restrict__ logits, const float* __restrict__ bias, i
         v = row[e];
         if (bias != nullptr) v = __fadd_rn(v, bias[e]);
       }
-      key[i] = v;
+      key[i] = ordered_bits(v + 0.0f);
     }
   }
 
   unsigned taken = 0u;  // bit i: this lane's i-th key is already selected
   int my_e = 0;         // lane j (< k) ends up holding the j-th selected expert
   for (int j = 0; j < k; ++j) {
-    float bv = 0.f;
+    unsigned bv = 0u;
     int be = 0x7fffffff;
     bool has = false;
 #pragma unroll
@@ -70,20 +74,13 @@ route_kernel(const float* __restrict__ logits, const float* __restrict__ bias, i
         bv = key[i]; be = e; has = true;
       }
     }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-      const int oe = __shfl_xor_sync(0xffffffffu, be, off);
-      const bool oh = __shfl_xor_sync(0xffffffffu, (int)has, off) != 0;
-      if (oh && (!has || comes_before(ov, oe, bv, be))) {
-        bv = ov; be = oe; has = true;
-      }
-    }
-    be = __shfl_sync(0xffffffffu, be, 0);  // one answer for the warp even if the order was not total (NaN)
-    const int owner = VEC ? ((be & 127) >> 2) : (be & 31);
-    const int slot = VEC ? (4 * (be >> 7) + (be & 3)) : (be >> 5);
+    // warp arg-max on (key descending, expert index ascending): largest key, then the lowest index holding it
+    const unsigned top = __reduce_max_sync(0xffffffffu, has ? bv : 0u);
+    const int win = (int)__reduce_min_sync(0xffffffffu, (unsigned)((has && bv == top) ? be : 0x7fffffff));
+    const int owner = VEC ? ((win & 127) >> 2) : (win & 31);
+    const int slot = VEC ? (4 * (win >> 7) + (win & 3)) : (win >> 5);
     if (lane == owner) taken |= (1u << slot);
-    if (lane == j) my_e = be;
+    if (lane == j) my_e = win;
   }
 
   const bool active = lane < k;

@@ -10,7 +10,7 @@ namespace {
 
 constexpr int kPermuteThreads = 256;
 constexpr int kPermuteVecPerThread = 4;  // 16-byte vectors held in registers per pass
-constexpr int kCombineThreads = 128;
+constexpr int kCombineThreads = 256;
 
 // x_perm[inv_perm[t*k+j], :] = x[t, :]  for j < k.  One CTA walks tokens; a token's row is loaded once
 // into registers and stored to its k destinations.
@@ -51,41 +51,67 @@ __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4& v, floa
 }
 
 // out[t,:] = sum_j w[t,j] * y_perm[inv_perm[t*k+j],:] (+ y_shared[t,:]); ascending j, then the shared row.
-// grid = (T, ceil(H8 / kCombineThreads)).  KU is the unroll width of the gather.
+// Persistent CTAs walk (token, 256-vector column block) items; a thread owns one 16-byte vector of the
+// output row, keeps the k gathered loads in flight together, and fetches the next item's row indices and
+// weights before it consumes the current rows, so the index -> row dependency is off the critical path.
+// KU is the unroll width of the gather (k <= KU handled in one pass).
 template <int KU>
 __global__ void __launch_bounds__(kCombineThreads)
 combine_kernel(const uint4* __restrict__ y_perm, const uint4* __restrict__ y_shared,
                const int32_t* __restrict__ inv_perm, const float* __restrict__ topk_w, uint4* __restrict__ out, int T,
-               int k, int H8) {
-  const int t = blockIdx.x;
-  const int v = blockIdx.y * kCombineThreads + threadIdx.x;
-  if (v >= H8) return;
-  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  for (int j0 = 0; j0 < k; j0 += KU) {
-    uint4 val[KU];
-    float wj[KU];
+               int k, int H8, int col_blocks) {
+  const long long n_items = (long long)T * col_blocks;
+  long long item = blockIdx.x;
+  if (item >= n_items) return;
+  int pj[KU];
+  float wj[KU];
+  auto load_meta = [&](long long it) {
+    const int t = (int)(it / col_blocks);
 #pragma unroll
     for (int u = 0; u < KU; ++u) {
-      const int j = j0 + u;
+      pj[u] = -1;
       wj[u] = 0.f;
-      val[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (j < k) {
-        const int p = __ldg(inv_perm + (size_t)t * k + j);
-        if (p >= 0) {
-          wj[u] = __ldg(topk_w + (size_t)t * k + j);
-          val[u] = __ldg(y_perm + (size_t)p * H8 + v);
-        }
+      if (u < k) {
+        pj[u] = __ldg(inv_perm + (size_t)t * k + u);
+        wj[u] = __ldg(topk_w + (size_t)t * k + u);
       }
     }
+  };
+  load_meta(item);
+  while (item < n_items) {
+    const int t = (int)(item / col_blocks);
+    const int v = (int)(item % col_blocks) * kCombineThreads + threadIdx.x;
+    const bool in = v < H8;
+    uint4 val[KU];
+    float wc[KU];
 #pragma unroll
-    for (int u = 0; u < KU; ++u) fma_bf16x8(acc, val[u], wj[u]);
+    for (int u = 0; u < KU; ++u) {
+      wc[u] = pj[u] >= 0 ? wj[u] : 0.f;
+      val[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (in && pj[u] >= 0) val[u] = __ldg(y_perm + (size_t)pj[u] * H8 + v);
+    }
+    uint4 sh = make_uint4(0u, 0u, 0u, 0u);
+    if (in && y_shared != nullptr) sh = __ldg(y_shared + (size_t)t * H8 + v);
+    const long long next = item + gridDim.x;
+    if (next < n_items) load_meta(next);  // issued while the rows above are still in flight
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int u = 0; u < KU; ++u) fma_bf16x8(acc, val[u], wc[u]);
+    // experts beyond KU (k > KU): plain second pass
+    for (int j = KU; j < k; ++j) {
+      const int pr = __ldg(inv_perm + (size_t)t * k + j);
+      if (in && pr >= 0) fma_bf16x8(acc, __ldg(y_perm + (size_t)pr * H8 + v), __ldg(topk_w + (size_t)t * k + j));
+    }
+    if (y_shared != nullptr) fma_bf16x8(acc, sh, 1.0f);
+    if (in) {
+      uint4 o;
+      __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) oh[q] = __floats2bfloat162_rn(acc[2 * q], acc[2 * q + 1]);
+      out[(size_t)t * H8 + v] = o;
+    }
+    item = next;
   }
-  if (y_shared != nullptr) fma_bf16x8(acc, __ldg(y_shared + (size_t)t * H8 + v), 1.0f);
-  uint4 o;
-  __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
-#pragma unroll
-  for (int q = 0; q < 4; ++q) oh[q] = __floats2bfloat162_rn(acc[2 * q], acc[2 * q + 1]);
-  out[(size_t)t * H8 + v] = o;
 }
 
 }  // namespace
@@ -106,13 +132,23 @@ cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32
                            void* out, int T, int k, int H, cudaStream_t stream, int* n_launches) {
   if (T <= 0) return cudaSuccess;
   const int H8 = H / 8;
-  dim3 grid(T, (H8 + kCombineThreads - 1) / kCombineThreads);
+  const int col_blocks = (H8 + kCombineThreads - 1) / kCombineThreads;
+  const long long n_items = (long long)T * col_blocks;
   const uint4* yp = static_cast<const uint4*>(y_perm);
   const uint4* ys = static_cast<const uint4*>(y_shared);
   uint4* o = static_cast<uint4*>(out);
-  if (k >= 8) combine_kernel<8><<<grid, kCombineThreads, 0, stream>>>(yp, ys, inv_perm, topk_w, o, T, k, H8);
-  else if (k >= 4) combine_kernel<4><<<grid, kCombineThreads, 0, stream>>>(yp, ys, inv_perm, topk_w, o, T, k, H8);
-  else combine_kernel<2><<<grid, kCombineThreads, 0, stream>>>(yp, ys, inv_perm, topk_w, o, T, k, H8);
+  auto launch = [&](auto kern) {
+    int dev = 0, sms = 148, per_sm = 2;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kCombineThreads, 0);
+    const long long cap = (long long)sms * (per_sm > 0 ? per_sm : 1);  // one resident wave of persistent CTAs
+    const int grid = (int)(n_items < cap ? n_items : cap);
+    kern<<<grid, kCombineThreads, 0, stream>>>(yp, ys, inv_perm, topk_w, o, T, k, H8, col_blocks);
+  };
+  if (k > 4) launch(combine_kernel<8>);
+  else if (k > 2) launch(combine_kernel<4>);
+  else launch(combine_kernel<2>);
   cudaError_t err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
