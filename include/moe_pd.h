@@ -174,8 +174,8 @@ moe_status moe_combine(moe_ctx* ctx, const float* topk_w, const int32_t* inv_per
  * runtime that has handed every byte of the device to its own allocator, or any place where cudaMalloc is
  * forbidden.  (The paper has no counterpart of this entry point; it exists for such embedders.)
  * The scratch the large-T path needs lives in a 256 KiB array inside the library image, which each GPU that
- * loads the library holds until the process exits.  Limit: ceil(T*top_k / 1024) * n_experts <= 65536
- * (e.g. T*top_k <= 262144 at 256 experts); beyond it the call returns MOE_ERR_CAPACITY and does nothing.
+ * loads the library holds until the process exits.  Limit: ceil(T*top_k / 256) * n_experts <= 65536
+ * (e.g. T*top_k <= 65536 at 256 experts); beyond it the call returns MOE_ERR_CAPACITY and does nothing.
  * The call allocates nothing and frees nothing.  It works on the device that is current when it is called:
  * the pointers and the stream must belong to that device.  The first call on each device looks up the
  * array's device address (a host-side set-up step); make that first call before any stream capture begins.

@@ -390,7 +390,8 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
   }
   if (e == cudaSuccess && x != nullptr) {
     StageTimer tm(ctx, 2);
-    e = moe::launch_permute(x, ctx->inv_perm, b.x_perm, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->stream, &n);
+    e = moe::launch_permute(x, ctx->inv_perm, b.x_perm, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->status, ctx->stream,
+                            &n);
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_dispatch_layout");
   ctx->T = T;
@@ -481,7 +482,7 @@ moe_status moe_combine(moe_ctx* ctx, const float* topk_w, const int32_t* inv_per
   {
     StageTimer tm(ctx, 7);
     e = moe::launch_combine(b.y_perm, ctx->cfg.n_shared ? b.y_shared : nullptr, inv_perm ? inv_perm : ctx->inv_perm,
-                            topk_w, out, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->stream, &n);
+                            topk_w, out, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->status, ctx->stream, &n);
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_combine");
   ctx->state = ST_IDLE;

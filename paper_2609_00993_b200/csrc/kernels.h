@@ -17,7 +17,7 @@ cudaError_t launch_route(const float* logits, const float* bias, int T, int E, i
 
 // ---- a2-a4 layout --------------------------------------------------------------------------
 // Slots per warp-owned chunk in the multi-CTA path, and the scratch it needs.
-constexpr int kLayoutChunk = 1024;
+constexpr int kLayoutChunk = 256;
 inline size_t layout_scratch_ints(int64_t n_slots, int E) {
   int64_t chunks = (n_slots + kLayoutChunk - 1) / kLayoutChunk;
   return (size_t)(chunks > 0 ? chunks : 1) * (size_t)E;
@@ -27,10 +27,10 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
                           int* n_launches);
 
 // ---- a5 permute, a9 combine ----------------------------------------------------------------
-cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm, int T, int k, int H,
+cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm, int T, int k, int H, int* status,
                            cudaStream_t stream, int* n_launches);
 cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32_t* inv_perm, const float* topk_w,
-                           void* out, int T, int k, int H, cudaStream_t stream, int* n_launches);
+                           void* out, int T, int k, int H, int* status, cudaStream_t stream, int* n_launches);
 
 // ---- a6-a8 grouped GEMM --------------------------------------------------------------------
 // One grouped GEMM pass:  out[r, :] = epilogue( A[r, :] . W[e]^T )  for r in expert e's segment.

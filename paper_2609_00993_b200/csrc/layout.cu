@@ -179,23 +179,51 @@ layout_count_kernel(const int32_t* __restrict__ topk_idx, int64_t n_slots, int E
 }
 
 // (2) one CTA: per expert an exclusive prefix over chunks (in place), totals -> counts, then the
-//     exclusive scan over experts -> offsets.
+//     exclusive scan over experts -> offsets.  The 1024 threads form `parts` x Epad: a thread owns one
+//     expert and one contiguous run of chunks, so the walk over chunks is `parts` times shorter, and its
+//     loads go out in batches of kBatch before the dependent stores.
+//     shared memory: partial[parts][Epad] | counts_sh[E] | offsets_sh[E+1] | warp_sums[33]
 __global__ void __launch_bounds__(1024)
-layout_scan_kernel(int32_t* __restrict__ chunk_counts, int n_chunks, int E, int32_t* __restrict__ counts,
-                   int32_t* __restrict__ offsets) {
+layout_scan_kernel(int32_t* __restrict__ chunk_counts, int n_chunks, int E, int Epad, int parts,
+                   int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
   extern __shared__ int sh[];
-  int* counts_sh = sh;
+  int* partial = sh;
+  int* counts_sh = partial + parts * Epad;
   int* offsets_sh = counts_sh + E;
   int* warp_sums = offsets_sh + (E + 1);
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    int sum = 0;
-    for (int c = 0; c < n_chunks; ++c) {
-      const int v = chunk_counts[(size_t)c * E + e];
-      chunk_counts[(size_t)c * E + e] = sum;
-      sum += v;
+  const int part = threadIdx.x / Epad, e = threadIdx.x % Epad;
+  const bool active = part < parts && e < E;
+  const int per = (n_chunks + parts - 1) / parts;
+  const int c0 = min(part * per, n_chunks), c1 = min(c0 + per, n_chunks);
+  int sum = 0;
+  if (active) {
+    for (int cb = c0; cb < c1; cb += kBatch) {
+      int v[kBatch];
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) v[u] = (cb + u < c1) ? chunk_counts[(size_t)(cb + u) * E + e] : 0;
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) sum += v[u];
     }
-    counts_sh[e] = sum;
-    counts[e] = sum;
+  }
+  if (part < parts) partial[part * Epad + e] = sum;
+  __syncthreads();
+  if (active) {
+    int run = 0;
+    for (int q = 0; q < part; ++q) run += partial[q * Epad + e];
+    if (part == parts - 1) {
+      counts_sh[e] = run + sum;
+      counts[e] = run + sum;
+    }
+    for (int cb = c0; cb < c1; cb += kBatch) {
+      int v[kBatch];
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) v[u] = (cb + u < c1) ? chunk_counts[(size_t)(cb + u) * E + e] : 0;
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        if (cb + u < c1) chunk_counts[(size_t)(cb + u) * E + e] = run;
+        run += v[u];
+      }
+    }
   }
   __syncthreads();
   block_exclusive_scan(counts_sh, E, offsets, offsets_sh, warp_sums);
@@ -257,8 +285,12 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
   layout_count_kernel<<<blocks, kChunkWarpsPerBlock * 32, chunk_smem, stream>>>(topk_idx, n_slots, E, n_chunks,
                                                                                 scratch, status);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
-  const size_t scan_smem = ((size_t)E + (E + 1) + 33) * sizeof(int);
-  layout_scan_kernel<<<1, 1024, scan_smem, stream>>>(scratch, n_chunks, E, counts, offsets);
+  const int Epad = (E + 31) / 32 * 32;
+  int parts = 1024 / Epad;
+  if (parts > n_chunks) parts = n_chunks;
+  if (parts < 1) parts = 1;
+  const size_t scan_smem = ((size_t)parts * Epad + E + (E + 1) + 33) * sizeof(int);
+  layout_scan_kernel<<<1, 1024, scan_smem, stream>>>(scratch, n_chunks, E, Epad, parts, counts, offsets);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
   layout_place_kernel<<<blocks, kChunkWarpsPerBlock * 32, chunk_smem, stream>>>(topk_idx, n_slots, E, n_chunks,
                                                                                 scratch, offsets, perm, inv_perm);
@@ -281,7 +313,7 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
 
 namespace {
 
-constexpr int kStaticScratchInts = 64 * 1024;  // 256 KiB: up to ceil(N/1024) * E = 65536 histogram cells
+constexpr int kStaticScratchInts = 64 * 1024;  // 256 KiB: up to ceil(N/256) * E = 65536 histogram cells
 static __device__ __align__(256) int32_t g_static_layout_scratch[kStaticScratchInts];
 
 constexpr int kMaxDevices = 64;

@@ -1,6 +1,12 @@
-// Stage a5 (routed row movement) and stage a9 (weighted combine).  Both are pure HBM streaming:
-// every access is a 128-bit vector, a row is read once and written k times (permute) or k rows are
-// gathered, summed in fp32 and written once (combine).
+// Stage a5 (routed row movement) and stage a9 (weighted combine).  Both are pure HBM streaming, so both move
+// rows with bulk asynchronous copies (cp.async.bulk) through shared-memory slots: a copy of several KB is one
+// instruction, completion is tracked by mbarriers (loads) and bulk groups (stores), and many tens of KB per SM
+// stay in flight without costing registers or issue slots.
+//   permute  one warp per CTA walks (token, row chunk) items: the chunk is loaded once into a slot and stored
+//            from there to its k destination rows.
+//   combine  a producer warp gathers the k (+ shared) row chunks of an item into a slot, four consumer warps
+//            sum them in fp32 in ascending expert order, round once to bf16 and store.  Deterministic.
+// Every mbarrier wait is bounded; on expiry the kernel records a timeout in the status word and stops.
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -8,37 +14,114 @@
 namespace moe {
 namespace {
 
-constexpr int kPermuteThreads = 256;
-constexpr int kPermuteVecPerThread = 4;  // 16-byte vectors held in registers per pass
-constexpr int kCombineThreads = 256;
+constexpr uint32_t kSpinLimit = 1u << 22;
 
-// x_perm[inv_perm[t*k+j], :] = x[t, :]  for j < k.  One CTA walks tokens; a token's row is loaded once
-// into registers and stored to its k destinations.
-__global__ void __launch_bounds__(kPermuteThreads)
-permute_rows_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ inv_perm, uint4* __restrict__ x_perm,
-                    int T, int k, int H8) {
-  for (int t = blockIdx.x; t < T; t += gridDim.x) {
-    const uint4* src = x + (size_t)t * H8;
-    for (int v0 = 0; v0 < H8; v0 += kPermuteThreads * kPermuteVecPerThread) {
-      uint4 val[kPermuteVecPerThread];
-#pragma unroll
-      for (int u = 0; u < kPermuteVecPerThread; ++u) {
-        const int v = v0 + u * kPermuteThreads + threadIdx.x;
-        if (v < H8) val[u] = __ldg(src + v);
-      }
-      for (int j = 0; j < k; ++j) {
-        const int p = __ldg(inv_perm + (size_t)t * k + j);
-        if (p < 0) continue;  // dropped slot (expert index was out of range)
-        uint4* dst = x_perm + (size_t)p * H8;
-#pragma unroll
-        for (int u = 0; u < kPermuteVecPerThread; ++u) {
-          const int v = v0 + u * kPermuteThreads + threadIdx.x;
-          if (v < H8) dst[v] = val[u];
-        }
-      }
-    }
-  }
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if (i >= 256u) __nanosleep(64);
+  }
+  return false;
+}
+// global -> shared, `bytes` a multiple of 16, both addresses 16-byte aligned; completes on the mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+// shared -> global, tracked by the issuing thread's bulk groups
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src_smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void flag_timeout(int* status) {
+  if (status != nullptr) atomicCAS(status, kStOk, kStTimeout);
+}
+
+// ------------------------------------------------------------------------------------------- a5 permute
+constexpr int kPermuteSlots = 4;
+constexpr int kPermuteChunkCols = 4096;  // bf16 columns per item: at most 8 KB per slot
+
+// x_perm[inv_perm[t*k+j], c0:c1] = x[t, c0:c1] for j < k.  One warp per CTA; lane j stores destination j.
+// dynamic shared memory: kPermuteSlots slots of slot_bytes | full[kPermuteSlots]
+__global__ void __launch_bounds__(32)
+permute_rows_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ inv_perm,
+                    __nv_bfloat16* __restrict__ x_perm, int T, int k, int H, int col_blocks, int slot_bytes,
+                    int* status) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const uint32_t slots = smem_u32(smem);
+  const uint32_t bar_full = slots + (uint32_t)(kPermuteSlots * slot_bytes);
+  const int lane = threadIdx.x;
+  const long long n_items = (long long)T * col_blocks;
+  if (lane == 0) {
+    for (int s = 0; s < kPermuteSlots; ++s) mbar_init(bar_full + 8u * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncwarp();
+
+  auto item_of = [&](long long n) { return (long long)blockIdx.x + n * gridDim.x; };
+  auto issue_load = [&](long long n) {  // lane 0 only
+    const long long it = item_of(n);
+    if (it >= n_items) return;
+    const int t = (int)(it / col_blocks), c0 = (int)(it % col_blocks) * kPermuteChunkCols;
+    const uint32_t bytes = (uint32_t)(min(kPermuteChunkCols, H - c0) * 2);
+    const uint32_t s = (uint32_t)(n % kPermuteSlots);
+    mbar_expect_tx(bar_full + 8u * s, bytes);
+    bulk_load(slots + s * (uint32_t)slot_bytes, x + (size_t)t * H + c0, bytes, bar_full + 8u * s);
+  };
+
+  if (lane == 0)
+    for (int n = 0; n < kPermuteSlots; ++n) issue_load(n);
+  bool ok = true;
+  for (long long n = 0; item_of(n) < n_items; ++n) {
+    const long long it = item_of(n);
+    const int t = (int)(it / col_blocks), c0 = (int)(it % col_blocks) * kPermuteChunkCols;
+    const uint32_t bytes = (uint32_t)(min(kPermuteChunkCols, H - c0) * 2);
+    const uint32_t s = (uint32_t)(n % kPermuteSlots), ph = (uint32_t)((n / kPermuteSlots) & 1);
+    int dst_row = -1;
+    if (lane < k) dst_row = __ldg(inv_perm + (size_t)t * k + lane);  // in flight while the row chunk arrives
+    ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8u * s, ph));
+    if (!ok) break;
+    if (dst_row >= 0) bulk_store(x_perm + (size_t)dst_row * H + c0, slots + s * (uint32_t)slot_bytes, bytes);
+    bulk_commit();
+    // the slot used one item ago may be refilled once every lane's stores from it have read shared memory
+    bulk_wait_read<1>();
+    __syncwarp();
+    if (lane == 0 && n >= 1) issue_load(n - 1 + kPermuteSlots);
+  }
+  bulk_wait_read<0>();
+  if (!ok && lane == 0) flag_timeout(status);
+}
+
+// ------------------------------------------------------------------------------------------- a9 combine
+constexpr int kCombineChunkCols = 1024;  // bf16 columns per item: 2 KB per gathered row chunk
+constexpr int kCombineConsumers = 128;   // one 16-byte vector (8 columns) per consumer thread
+constexpr int kCombineThreads = kCombineConsumers + 32;
+constexpr int kCombineMaxStages = 4;
 
 __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4& v, float w) {
   const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
@@ -50,106 +133,143 @@ __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4& v, floa
   }
 }
 
-// out[t,:] = sum_j w[t,j] * y_perm[inv_perm[t*k+j],:] (+ y_shared[t,:]); ascending j, then the shared row.
-// Persistent CTAs walk (token, 256-vector column block) items; a thread owns one 16-byte vector of the
-// output row, keeps the k gathered loads in flight together, and fetches the next item's row indices and
-// weights before it consumes the current rows, so the index -> row dependency is off the critical path.
-// KU is the unroll width of the gather (k <= KU handled in one pass).
-template <int KU>
+// out[t, c0:c1] = sum_j w[t,j] * y_perm[inv_perm[t*k+j], c0:c1] (+ y_shared[t, c0:c1]); ascending j, then shared.
+// dynamic shared memory, per stage: (k+1) row chunks of chunk_bytes | k weights | valid mask; then barriers.
+// Producer lane j gathers row j; lane 0 also fetches the shared row.
 __global__ void __launch_bounds__(kCombineThreads)
-combine_kernel(const uint4* __restrict__ y_perm, const uint4* __restrict__ y_shared,
-               const int32_t* __restrict__ inv_perm, const float* __restrict__ topk_w, uint4* __restrict__ out, int T,
-               int k, int H8, int col_blocks) {
+combine_kernel(const __nv_bfloat16* __restrict__ y_perm, const __nv_bfloat16* __restrict__ y_shared,
+               const int32_t* __restrict__ inv_perm, const float* __restrict__ topk_w, __nv_bfloat16* __restrict__ out,
+               int T, int k, int H, int col_blocks, int chunk_bytes, int stage_bytes, int n_stages, int* status) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const uint32_t base = smem_u32(smem);
+  const uint32_t bar_full = base + (uint32_t)(n_stages * stage_bytes);
+  const uint32_t bar_empty = bar_full + 8u * n_stages;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int meta_off = (k + 1) * chunk_bytes;  // weights (k floats), then the valid mask
   const long long n_items = (long long)T * col_blocks;
-  long long item = blockIdx.x;
-  if (item >= n_items) return;
-  int pj[KU];
-  float wj[KU];
-  auto load_meta = [&](long long it) {
-    const int t = (int)(it / col_blocks);
-#pragma unroll
-    for (int u = 0; u < KU; ++u) {
-      pj[u] = -1;
-      wj[u] = 0.f;
-      if (u < k) {
-        pj[u] = __ldg(inv_perm + (size_t)t * k + u);
-        wj[u] = __ldg(topk_w + (size_t)t * k + u);
-      }
+  const bool shared = y_shared != nullptr;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < n_stages; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, kCombineConsumers / 32);
     }
-  };
-  load_meta(item);
-  while (item < n_items) {
-    const int t = (int)(item / col_blocks);
-    const int v = (int)(item % col_blocks) * kCombineThreads + threadIdx.x;
-    const bool in = v < H8;
-    uint4 val[KU];
-    float wc[KU];
-#pragma unroll
-    for (int u = 0; u < KU; ++u) {
-      wc[u] = pj[u] >= 0 ? wj[u] : 0.f;
-      val[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (in && pj[u] >= 0) val[u] = __ldg(y_perm + (size_t)pj[u] * H8 + v);
-    }
-    uint4 sh = make_uint4(0u, 0u, 0u, 0u);
-    if (in && y_shared != nullptr) sh = __ldg(y_shared + (size_t)t * H8 + v);
-    const long long next = item + gridDim.x;
-    if (next < n_items) load_meta(next);  // issued while the rows above are still in flight
-    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int u = 0; u < KU; ++u) fma_bf16x8(acc, val[u], wc[u]);
-    // experts beyond KU (k > KU): plain second pass
-    for (int j = KU; j < k; ++j) {
-      const int pr = __ldg(inv_perm + (size_t)t * k + j);
-      if (in && pr >= 0) fma_bf16x8(acc, __ldg(y_perm + (size_t)pr * H8 + v), __ldg(topk_w + (size_t)t * k + j));
-    }
-    if (y_shared != nullptr) fma_bf16x8(acc, sh, 1.0f);
-    if (in) {
-      uint4 o;
-      __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) oh[q] = __floats2bfloat162_rn(acc[2 * q], acc[2 * q + 1]);
-      out[(size_t)t * H8 + v] = o;
-    }
-    item = next;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  __syncthreads();
+
+  if (warp == kCombineConsumers / 32) {
+    // ============================================================ producer warp: lane j gathers row j
+    bool ok = true;
+    long long n = 0;
+    for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++n) {
+      const int t = (int)(it / col_blocks), c0 = (int)(it % col_blocks) * kCombineChunkCols;
+      const uint32_t bytes = (uint32_t)(min(kCombineChunkCols, H - c0) * 2);
+      const uint32_t s = (uint32_t)(n % n_stages), ph = (uint32_t)((n / n_stages) & 1);
+      int row = -1;
+      float wv = 0.f;
+      if (lane < k) {
+        row = __ldg(inv_perm + (size_t)t * k + lane);
+        wv = __ldg(topk_w + (size_t)t * k + lane);
+      }
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8u * s, ph ^ 1u));
+      if (!ok) break;
+      uint8_t* st = smem + (size_t)s * stage_bytes;
+      const unsigned valid = __ballot_sync(0xffffffffu, row >= 0);
+      if (lane < k) reinterpret_cast<float*>(st + meta_off)[lane] = wv;
+      if (lane == 0) *reinterpret_cast<unsigned*>(st + meta_off + 4 * k) = valid;
+      __syncwarp();
+      const uint32_t full = bar_full + 8u * s;
+      if (lane == 0) mbar_expect_tx(full, (uint32_t)(__popc(valid) + (shared ? 1 : 0)) * bytes);
+      __syncwarp();
+      const uint32_t dst = base + s * (uint32_t)stage_bytes;
+      if (row >= 0) bulk_load(dst + (uint32_t)(lane * chunk_bytes), y_perm + (size_t)row * H + c0, bytes, full);
+      if (shared && lane == 0) bulk_load(dst + (uint32_t)(k * chunk_bytes), y_shared + (size_t)t * H + c0, bytes, full);
+    }
+    if (!ok && lane == 0) flag_timeout(status);
+  } else {
+    // ============================================================ consumer warps: one 16-byte vector each
+    bool ok = true;
+    long long n = 0;
+    const int v = threadIdx.x;
+    for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++n) {
+      const int t = (int)(it / col_blocks), c0 = (int)(it % col_blocks) * kCombineChunkCols;
+      const int cols = min(kCombineChunkCols, H - c0);
+      const uint32_t s = (uint32_t)(n % n_stages), ph = (uint32_t)((n / n_stages) & 1);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8u * s, ph));
+      if (!ok) break;
+      const uint8_t* st = smem + (size_t)s * stage_bytes;
+      const float* wts = reinterpret_cast<const float*>(st + meta_off);
+      const unsigned valid = *reinterpret_cast<const unsigned*>(st + meta_off + 4 * k);
+      if (v * 8 < cols) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int j = 0; j < k; ++j)
+          if ((valid >> j) & 1u)
+            fma_bf16x8(acc, *reinterpret_cast<const uint4*>(st + (size_t)j * chunk_bytes + v * 16), wts[j]);
+        if (shared) fma_bf16x8(acc, *reinterpret_cast<const uint4*>(st + (size_t)k * chunk_bytes + v * 16), 1.0f);
+        uint4 o;
+        __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) oh[q] = __floats2bfloat162_rn(acc[2 * q], acc[2 * q + 1]);
+        *reinterpret_cast<uint4*>(out + (size_t)t * H + c0 + v * 8) = o;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_empty + 8u * s);
+    }
+    if (!ok && lane == 0) flag_timeout(status);
+  }
+}
+
+int resident_ctas(const void* kern, int threads, size_t smem) {
+  int dev = 0, sms = 148, per_sm = 1;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
+  return sms * (per_sm > 0 ? per_sm : 1);
 }
 
 }  // namespace
 
-cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm, int T, int k, int H,
+cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm, int T, int k, int H, int* status,
                            cudaStream_t stream, int* n_launches) {
   if (T <= 0) return cudaSuccess;
-  const int H8 = H / 8;
-  const int blocks = T < 148 * 8 ? T : 148 * 8;
-  permute_rows_kernel<<<blocks, kPermuteThreads, 0, stream>>>(static_cast<const uint4*>(x), inv_perm,
-                                                              static_cast<uint4*>(x_perm), T, k, H8);
-  cudaError_t err = cudaGetLastError();
+  if (k > 32) return cudaErrorNotSupported;  // one storing lane per destination
+  const int col_blocks = (H + kPermuteChunkCols - 1) / kPermuteChunkCols;
+  const int slot_bytes = (H < kPermuteChunkCols ? H : kPermuteChunkCols) * 2;
+  const size_t smem = (size_t)kPermuteSlots * slot_bytes + 8 * kPermuteSlots;
+  cudaError_t err = cudaFuncSetAttribute(permute_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
+  const long long n_items = (long long)T * col_blocks;
+  const long long cap = resident_ctas(reinterpret_cast<const void*>(permute_rows_kernel), 32, smem);
+  const int grid = (int)(n_items < cap ? n_items : cap);
+  permute_rows_kernel<<<grid, 32, smem, stream>>>(static_cast<const __nv_bfloat16*>(x), inv_perm,
+                                                  static_cast<__nv_bfloat16*>(x_perm), T, k, H, col_blocks, slot_bytes,
+                                                  status);
+  err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }
 
 cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32_t* inv_perm, const float* topk_w,
-                           void* out, int T, int k, int H, cudaStream_t stream, int* n_launches) {
+                           void* out, int T, int k, int H, int* status, cudaStream_t stream, int* n_launches) {
   if (T <= 0) return cudaSuccess;
-  const int H8 = H / 8;
-  const int col_blocks = (H8 + kCombineThreads - 1) / kCombineThreads;
+  if (k > 32) return cudaErrorNotSupported;  // one gathering lane per row
+  const int col_blocks = (H + kCombineChunkCols - 1) / kCombineChunkCols;
+  const int chunk_bytes = (H < kCombineChunkCols ? H : kCombineChunkCols) * 2;
+  const int stage_bytes = ((k + 1) * chunk_bytes + 4 * k + 4 + 127) / 128 * 128;
+  int stages = (64 * 1024) / stage_bytes;  // about 64 KB of slots per CTA, three CTAs per SM
+  if (stages > kCombineMaxStages) stages = kCombineMaxStages;
+  if (stages < 2) stages = 2;
+  const size_t smem = (size_t)stages * stage_bytes + 16 * stages;
+  cudaError_t err = cudaFuncSetAttribute(combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (err != cudaSuccess) return err;
   const long long n_items = (long long)T * col_blocks;
-  const uint4* yp = static_cast<const uint4*>(y_perm);
-  const uint4* ys = static_cast<const uint4*>(y_shared);
-  uint4* o = static_cast<uint4*>(out);
-  auto launch = [&](auto kern) {
-    int dev = 0, sms = 148, per_sm = 2;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kCombineThreads, 0);
-    const long long cap = (long long)sms * (per_sm > 0 ? per_sm : 1);  // one resident wave of persistent CTAs
-    const int grid = (int)(n_items < cap ? n_items : cap);
-    kern<<<grid, kCombineThreads, 0, stream>>>(yp, ys, inv_perm, topk_w, o, T, k, H8, col_blocks);
-  };
-  if (k > 4) launch(combine_kernel<8>);
-  else if (k > 2) launch(combine_kernel<4>);
-  else launch(combine_kernel<2>);
-  cudaError_t err = cudaGetLastError();
+  const long long cap = resident_ctas(reinterpret_cast<const void*>(combine_kernel), kCombineThreads, smem);
+  const int grid = (int)(n_items < cap ? n_items : cap);
+  combine_kernel<<<grid, kCombineThreads, smem, stream>>>(
+      static_cast<const __nv_bfloat16*>(y_perm), static_cast<const __nv_bfloat16*>(y_shared), inv_perm, topk_w,
+      static_cast<__nv_bfloat16*>(out), T, k, H, col_blocks, chunk_bytes, stage_bytes, stages, status);
+  err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }
