@@ -208,7 +208,9 @@ moe_status moe_ctx_debug_ptrs(moe_ctx* ctx, void** x_perm, void** act, void** y_
  * bracketed by CUDA events on the context's stream.  moe_ctx_read_profile synchronises the stream, returns
  * the summed device time and the number of bracketed launches per stage since the last read, and resets.
  * Stage order: 0 route, 1 layout (counts+scan+permutation), 2 permute rows, 3 routed GEMM1+SwiGLU,
- * 4 routed GEMM2, 5 shared GEMM1+SwiGLU, 6 shared GEMM2, 7 combine. */
+ * 4 routed GEMM2, 5 shared GEMM1+SwiGLU, 6 shared GEMM2, 7 combine.  Without prefill segmentation the shared
+ * expert's passes ride in the routed launches, so their time is part of stages 3 and 4 and stages 5 and 6
+ * stay empty. */
 #define MOE_N_STAGES 8
 typedef struct {
   double ms[MOE_N_STAGES];

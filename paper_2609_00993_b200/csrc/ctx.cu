@@ -204,12 +204,26 @@ int small_m_tile(int T) {
   return t;
 }
 
-cudaError_t run_gemm(moe_ctx* ctx, const moe::GemmProblem& p, int T, int* n) {
-  int variant = ctx->cfg.gemm_variant;
-  if (variant == MOE_GEMM_AUTO) variant = (ctx->cfg.phase == MOE_PHASE_DECODE) ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M;
-  if (variant == MOE_GEMM_VALIDATION) return moe::launch_gemm_validation(p, ctx->stream, n);
+int gemm_variant_of(const moe_ctx* ctx) {
+  const int v = ctx->cfg.gemm_variant;
+  return v != MOE_GEMM_AUTO ? v : (ctx->cfg.phase == MOE_PHASE_DECODE ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M);
+}
+
+// `dense` (the shared expert's pass, or nullptr) rides in the same launch on the tensor-core path.
+cudaError_t run_gemm(moe_ctx* ctx, const moe::GemmProblem& p, const moe::GemmDenseGroup* dense, int T, int* n) {
+  const int variant = gemm_variant_of(ctx);
+  if (variant == MOE_GEMM_VALIDATION) {
+    cudaError_t e = moe::launch_gemm_validation(p, ctx->stream, n);
+    if (e == cudaSuccess && dense != nullptr) {
+      moe::GemmProblem d{dense->A, dense->W, dense->out, nullptr, dense->rows, dense->rows, dense->rows, 1,
+                         dense->n_feat, dense->K, p.gated};
+      e = moe::launch_gemm_validation(d, ctx->stream, n);
+    }
+    return e;
+  }
   const bool swap = (variant == MOE_GEMM_SMALL_M);
-  return moe::launch_gemm_tc(p, swap, swap ? small_m_tile(T) : 128, gemm_ctas(ctx), ctx->status, ctx->stream, n);
+  return moe::launch_gemm_tc(p, dense, swap, swap ? small_m_tile(T) : 128, gemm_ctas(ctx), ctx->status, ctx->stream,
+                             n);
 }
 
 }  // namespace
@@ -433,6 +447,11 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
     };
     moe::GemmProblem g1{b.x_perm, w_gate_up, b.act, ctx->offsets, 0, Ncap, N, c.n_experts, c.inter, c.hidden, true};
     moe::GemmProblem g2{b.act, w_down, b.y_perm, ctx->offsets, 0, Ncap, N, c.n_experts, c.hidden, c.inter, false};
+    moe::GemmDenseGroup s1{x, ws_gate_up, b.act_shared, T, c.shared_inter, c.hidden};
+    moe::GemmDenseGroup s2{b.act_shared, ws_down, b.y_shared, T, c.hidden, c.shared_inter};
+    // Unsegmented: the shared expert's two passes ride in the routed launches (two launches in all).
+    // Segmented: they are segments of their own, after the routed ones.
+    const bool fuse_shared = shared && ctx->seg_experts == 0;
     for (int pass = 0; pass < 2 && e == cudaSuccess; ++pass) {
       moe::GemmProblem& g = pass == 0 ? g1 : g2;
       for (int e0 = 0; e0 < c.n_experts && e == cudaSuccess; e0 += span) {
@@ -440,23 +459,23 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
         g.e_end = e0 + span < c.n_experts ? e0 + span : c.n_experts;
         {
           StageTimer tm(ctx, pass == 0 ? 3 : 4);
-          e = run_gemm(ctx, g, T, &n);
+          e = run_gemm(ctx, g, fuse_shared ? (pass == 0 ? &s1 : &s2) : nullptr, T, &n);
         }
         if (e == cudaSuccess) boundary();
       }
     }
-    if (e == cudaSuccess && shared) {
-      moe::GemmProblem s1{x, ws_gate_up, b.act_shared, nullptr, T, T, T, 1, c.shared_inter, c.hidden, true};
+    if (e == cudaSuccess && shared && !fuse_shared) {
+      moe::GemmProblem d1{s1.A, s1.W, s1.out, nullptr, T, T, T, 1, s1.n_feat, s1.K, true};
       {
         StageTimer tm(ctx, 5);
-        e = run_gemm(ctx, s1, T, &n);
+        e = run_gemm(ctx, d1, nullptr, T, &n);
       }
       if (e == cudaSuccess) {
         boundary();
-        moe::GemmProblem s2{b.act_shared, ws_down, b.y_shared, nullptr, T, T, T, 1, c.hidden, c.shared_inter, false};
+        moe::GemmProblem d2{s2.A, s2.W, s2.out, nullptr, T, T, T, 1, s2.n_feat, s2.K, false};
         {
           StageTimer tm(ctx, 6);
-          e = run_gemm(ctx, s2, T, &n);
+          e = run_gemm(ctx, d2, nullptr, T, &n);
         }
         if (e == cudaSuccess) boundary();
       }

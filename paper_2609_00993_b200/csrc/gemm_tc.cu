@@ -52,6 +52,11 @@ struct TcParams {
   int32_t n_stages;
   int32_t x_tile_bytes;    // row_tile * 128
   int* status;
+  // optional dense group (shared expert) computed by the same launch; rows2 == 0: none
+  int32_t rows2;
+  int32_t n_feat2;
+  int32_t K2;
+  __nv_bfloat16* out2;
 };
 
 // ---------------------------------------------------------------------------------- PTX wrappers
@@ -173,23 +178,36 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 struct Tile {
   int e, row0, rows, ft;
+  bool dense;  // a tile of the dense group
 };
 
-// tile -> (expert, first row, valid rows, feature tile).  prefix[e] = row tiles of experts < e.
-__device__ __forceinline__ Tile decode_tile(int tile, int n_ft, int E, const int* prefix, const int* seg,
-                                            int row_tile) {
+// tile -> (expert, first row, valid rows, feature tile).  The dense group's tiles come first (row tile major),
+// then the experts': prefix[e] = row tiles of experts < e.
+__device__ __forceinline__ Tile decode_tile(int tile, int dense_tiles, int n_ft2, int rows2, int n_ft, int E,
+                                            const int* prefix, const int* seg, int row_tile) {
+  Tile t;
+  if (tile < dense_tiles) {
+    const int rt = tile / n_ft2;
+    t.e = 0;
+    t.ft = tile - rt * n_ft2;
+    t.row0 = rt * row_tile;
+    t.rows = min(row_tile, rows2 - t.row0);
+    t.dense = true;
+    return t;
+  }
+  tile -= dense_tiles;
   const int rt = tile / n_ft;
   int lo = 0, hi = E;  // largest e in [0,E) with prefix[e] <= rt
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
     if (prefix[mid] <= rt) lo = mid; else hi = mid;
   }
-  Tile t;
   t.e = lo;
   t.ft = tile - rt * n_ft;
   const int mt = rt - prefix[lo];
   t.row0 = seg[lo] + mt * row_tile;
   t.rows = min(row_tile, seg[lo + 1] - t.row0);
+  t.dense = false;
   return t;
 }
 
@@ -197,6 +215,7 @@ __device__ __forceinline__ Tile decode_tile(int tile, int n_ft, int E, const int
 template <bool SWAP, bool GATED>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                       const __grid_constant__ CUtensorMap map_x2, const __grid_constant__ CUtensorMap map_w2,
                        const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   // carve: [stages] | epilogue staging (large-M) | barriers | tmem slot | abort | prefix[E+1] | seg[E+1]
@@ -222,7 +241,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   const int tile_rows = p.row_tile;  // token rows per tile of the list
   constexpr int kFeatPerTile = GATED ? 128 : 256;
   const int n_ft = (p.n_feat + kFeatPerTile - 1) / kFeatPerTile;
-  const int num_kb = (p.K + kBlockK - 1) / kBlockK;
+  const int num_kb1 = (p.K + kBlockK - 1) / kBlockK, num_kb2 = (p.K2 + kBlockK - 1) / kBlockK;
+  const int n_ft2 = (p.n_feat2 + kFeatPerTile - 1) / kFeatPerTile;
+  const int dense_tiles = p.rows2 > 0 ? ((p.rows2 + p.row_tile - 1) / p.row_tile) * n_ft2 : 0;
   const uint32_t acc_cols = SWAP ? 2u * (uint32_t)p.row_tile : 256u;  // TMEM columns per accumulator stage
   uint32_t tmem_cols = 32;
   while (tmem_cols < 2u * acc_cols) tmem_cols <<= 1;
@@ -270,7 +291,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int total_tiles = prefix[p.E] * n_ft;
+  const int total_tiles = dense_tiles + prefix[p.E] * n_ft;
 
   if (warp == kProducerWarp) {
     // ================================================================= TMA producer (one lane)
@@ -278,18 +299,22 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       uint32_t it = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
-        const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, tile_rows);
+        const Tile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, seg, tile_rows);
         const int w_row0 = t.ft * kFeatPerTile;
-        const int w_row1 = GATED ? p.n_feat + t.ft * kFeatPerTile : w_row0 + kWBoxRows;
+        const int w_row1 = GATED ? (t.dense ? p.n_feat2 : p.n_feat) + t.ft * kFeatPerTile : w_row0 + kWBoxRows;
+        const CUtensorMap* mw = t.dense ? &map_w2 : &map_w;
+        const CUtensorMap* mx = t.dense ? &map_x2 : &map_x;
+        const int w_e = t.dense ? 0 : p.e_base + t.e;
+        const int num_kb = t.dense ? num_kb2 : num_kb1;
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const uint32_t s = it % (uint32_t)p.n_stages, ph = (it / (uint32_t)p.n_stages) & 1u;
           if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t full = bar_full + 8u * s;
           const uint32_t st = base_addr + s * (uint32_t)stage_bytes;
           mbar_expect_tx(full, (uint32_t)stage_bytes);
-          tma_load_3d(st, &map_w, full, kb * kBlockK, w_row0, p.e_base + t.e);
-          tma_load_3d(st + kWBoxBytes, &map_w, full, kb * kBlockK, w_row1, p.e_base + t.e);
-          tma_load_2d(st + 2 * kWBoxBytes, &map_x, full, kb * kBlockK, t.row0);
+          tma_load_3d(st, mw, full, kb * kBlockK, w_row0, w_e);
+          tma_load_3d(st + kWBoxBytes, mw, full, kb * kBlockK, w_row1, w_e);
+          tma_load_2d(st + 2 * kWBoxBytes, mx, full, kb * kBlockK, t.row0);
         }
       }
       if (!ok) {
@@ -303,7 +328,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       uint32_t it = 0, tile_iter = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++tile_iter) {
-        const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, tile_rows);
+        const Tile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, seg, tile_rows);
         const uint32_t as = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
         if (!mbar_wait(bar_tempty + 8u * as, aph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
@@ -311,6 +336,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         // small-M: the MMA N covers only the rows this tile really has, rounded up to 16
         const uint32_t n_swap = (uint32_t)min(p.row_tile, (t.rows + 15) & ~15);
         const uint32_t idesc = SWAP ? umma_idesc(128, n_swap) : umma_idesc(128, 256);
+        const int num_kb = t.dense ? num_kb2 : num_kb1;
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const uint32_t s = it % (uint32_t)p.n_stages, ph = (it / (uint32_t)p.n_stages) & 1u;
           if (!mbar_wait(bar_full + 8u * s, ph, abort_flag)) { ok = false; break; }
@@ -345,7 +371,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     bool ok = true;
     const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
     for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++tile_iter) {
-      const Tile t = decode_tile(tile, n_ft, p.E, prefix, seg, tile_rows);
+      const Tile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, seg, tile_rows);
       const uint32_t as = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
       auto release_acc = [&]() {  // hand the accumulator stage back to the MMA issuer
         tc_fence_before();
@@ -355,6 +381,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       if (!mbar_wait(bar_tfull + 8u * as, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t d0 = tmem_base + as * acc_cols + lane_base;
+      __nv_bfloat16* const out = t.dense ? p.out2 : p.out;
+      const int n_feat = t.dense ? p.n_feat2 : p.n_feat;
       bool released = false;  // has this warp already handed the accumulator stage back?
       if (SWAP) {
         // lane = weight row (output feature), column = token
@@ -369,13 +397,13 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             if (c + i < t.rows) {
-              __nv_bfloat16* orow = p.out + (size_t)(t.row0 + c + i) * p.n_feat;
+              __nv_bfloat16* orow = out + (size_t)(t.row0 + c + i) * n_feat;
               const float a = __uint_as_float(ra[i]), b = __uint_as_float(rb[i]);
               if (GATED) {
-                if (f_a < p.n_feat) orow[f_a] = __float2bfloat16_rn(silu_mul(a, b));
+                if (f_a < n_feat) orow[f_a] = __float2bfloat16_rn(silu_mul(a, b));
               } else {
-                if (f_a < p.n_feat) orow[f_a] = __float2bfloat16_rn(a);
-                if (f_b < p.n_feat) orow[f_b] = __float2bfloat16_rn(b);
+                if (f_a < n_feat) orow[f_a] = __float2bfloat16_rn(a);
+                if (f_b < n_feat) orow[f_b] = __float2bfloat16_rn(b);
               }
             }
           }
@@ -390,7 +418,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         const int rows_here = t.rows - warp * 32;       // rows of this warp's 32 that are valid (may be <= 0)
         for (int pc = 0; pc < kPairs; ++pc) {
           const int f0 = t.ft * kFeatPerTile + pc * 64;
-          if (f0 >= p.n_feat) break;  // uniform across the CTA
+          if (f0 >= n_feat) break;  // uniform across the CTA
           uint32_t packed[32];
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
@@ -411,7 +439,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
                 packed[h * 16 + i] = pack_bf16(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1]));
             }
           }
-          if (pc == kPairs - 1 || f0 + 64 >= p.n_feat) {
+          if (pc == kPairs - 1 || f0 + 64 >= n_feat) {
             release_acc();  // the accumulator has been read completely: hand it back before the stores go out
             released = true;
           }
@@ -424,8 +452,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           for (int it = 0; it < 8; ++it) {
             const int rr = it * 4 + (lane >> 3), piece = lane & 7;
             const uint4 v = *reinterpret_cast<const uint4*>(stage_tile + rr * 128 + ((piece ^ (rr & 7)) << 4));
-            if (rr < rows_here && f0 + piece * 8 < p.n_feat)
-              *reinterpret_cast<uint4*>(p.out + (size_t)(t.row0 + warp * 32 + rr) * p.n_feat + f0 + piece * 8) = v;
+            if (rr < rows_here && f0 + piece * 8 < n_feat)
+              *reinterpret_cast<uint4*>(out + (size_t)(t.row0 + warp * 32 + rr) * n_feat + f0 + piece * 8) = v;
           }
           __syncwarp();
         }
@@ -474,11 +502,11 @@ bool encode_map(CUtensorMap* map, const void* base, int rank, const uint64_t* di
 }
 
 template <typename Kernel>
-cudaError_t launch_variant(Kernel kern, const CUtensorMap& mx, const CUtensorMap& mw, const TcParams& prm, int grid,
-                           size_t smem, cudaStream_t stream) {
+cudaError_t launch_variant(Kernel kern, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& mx2,
+                           const CUtensorMap& mw2, const TcParams& prm, int grid, size_t smem, cudaStream_t stream) {
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
-  kern<<<grid, kThreads, smem, stream>>>(mx, mw, prm);
+  kern<<<grid, kThreads, smem, stream>>>(mx, mw, mx2, mw2, prm);
   return cudaGetLastError();
 }
 
@@ -499,9 +527,12 @@ bool gemm_tc_init(const char** why) {
   return true;
 }
 
-cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int max_ctas, int* status,
-                           cudaStream_t stream, int* n_launches) {
-  if (p.rows_bound <= 0) return cudaSuccess;
+cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bool swap_ab, int row_tile,
+                           int max_ctas, int* status, cudaStream_t stream, int* n_launches) {
+  if (dense != nullptr && dense->rows <= 0) dense = nullptr;
+  if (p.rows_bound <= 0 && dense == nullptr) return cudaSuccess;
+  if (p.rows_bound <= 0) return cudaErrorInvalidValue;  // a dense group never comes without its routed pass
+  if (dense != nullptr && (dense->K % 8 != 0 || dense->n_feat % 8 != 0)) return cudaErrorNotSupported;
   if (g_encode == nullptr && !gemm_tc_init(nullptr)) return cudaErrorNotSupported;
   if (p.K % 8 != 0 || p.n_feat % 8 != 0 || p.E < 1 || p.E > 1024) return cudaErrorNotSupported;
   if (!swap_ab) row_tile = 128;
@@ -527,7 +558,23 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int
   const int e_begin = p.offsets ? p.e_begin : 0;
   const int e_end = (p.offsets && p.e_end >= 0) ? p.e_end : groups;
   if (e_begin < 0 || e_end > groups || e_begin >= e_end) return cudaErrorInvalidValue;
+  CUtensorMap mx2 = mx, mw2 = mw;
+  if (dense != nullptr) {
+    const uint64_t w2_rows = (uint64_t)(p.gated ? 2 : 1) * (uint64_t)dense->n_feat;
+    const uint64_t dx[2] = {(uint64_t)dense->K, (uint64_t)dense->rows};
+    const uint64_t sx[1] = {(uint64_t)dense->K * 2};
+    const uint32_t bx[2] = {(uint32_t)kBlockK, (uint32_t)row_tile};
+    if (!encode_map(&mx2, dense->A, 2, dx, sx, bx)) return cudaErrorInvalidValue;
+    const uint64_t dw[3] = {(uint64_t)dense->K, w2_rows, 1};
+    const uint64_t sw[2] = {(uint64_t)dense->K * 2, w2_rows * (uint64_t)dense->K * 2};
+    const uint32_t bw[3] = {(uint32_t)kBlockK, (uint32_t)kWBoxRows, 1u};
+    if (!encode_map(&mw2, dense->W, 3, dw, sw, bw)) return cudaErrorInvalidValue;
+  }
   TcParams prm;
+  prm.rows2 = dense ? dense->rows : 0;
+  prm.n_feat2 = dense ? dense->n_feat : 8;
+  prm.K2 = dense ? dense->K : 8;
+  prm.out2 = dense ? static_cast<__nv_bfloat16*>(dense->out) : nullptr;
   prm.offsets = p.offsets ? p.offsets + e_begin : nullptr;
   prm.fixed_rows = p.fixed_rows;
   prm.E = e_end - e_begin;
@@ -550,15 +597,17 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int
   const int feat_per_tile = p.gated ? 128 : 256;
   const int64_t n_ft = (p.n_feat + feat_per_tile - 1) / feat_per_tile;
   const int64_t row_tiles = p.rows_bound / row_tile + (prm.E < p.rows_bound ? prm.E : p.rows_bound);
-  const int64_t tiles = row_tiles * n_ft;
+  int64_t tiles = row_tiles * n_ft;
+  if (dense != nullptr)
+    tiles += (int64_t)((dense->rows + row_tile - 1) / row_tile) * ((dense->n_feat + feat_per_tile - 1) / feat_per_tile);
 
   int grid = (int)(tiles < (int64_t)max_ctas ? tiles : (int64_t)max_ctas);
   if (grid < 1) grid = 1;
   cudaError_t err;
-  if (swap_ab) err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true>, mx, mw, prm, grid, smem, stream)
-                             : launch_variant(grouped_gemm_tc_kernel<true, false>, mx, mw, prm, grid, smem, stream);
-  else err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true>, mx, mw, prm, grid, smem, stream)
-                     : launch_variant(grouped_gemm_tc_kernel<false, false>, mx, mw, prm, grid, smem, stream);
+  if (swap_ab) err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true>, mx, mw, mx2, mw2, prm, grid, smem, stream)
+                             : launch_variant(grouped_gemm_tc_kernel<true, false>, mx, mw, mx2, mw2, prm, grid, smem, stream);
+  else err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true>, mx, mw, mx2, mw2, prm, grid, smem, stream)
+                     : launch_variant(grouped_gemm_tc_kernel<false, false>, mx, mw, mx2, mw2, prm, grid, smem, stream);
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }

@@ -53,13 +53,25 @@ struct GemmProblem {
   int32_t e_end = -1;      // e_end < 0 means E
 };
 
+// A dense group (the shared expert) that rides in the same launch as a grouped problem: its tiles are added
+// to the tile list, so a pass that would fill only a few CTAs by itself shares the persistent grid.
+struct GemmDenseGroup {
+  const void* A;    // bf16 [rows, K]
+  const void* W;    // bf16 [(gated?2:1)*n_feat, K]
+  void* out;        // bf16 [rows, n_feat]
+  int32_t rows;
+  int32_t n_feat;
+  int32_t K;
+};
+
 cudaError_t launch_gemm_validation(const GemmProblem& p, cudaStream_t stream, int* n_launches);
 
 // Tensor-core path (tcgen05 + TMEM + TMA).  `swap_ab` selects the small-M variant; `row_tile` is the
 // token tile (128 for large-M; 16..128 for small-M); `max_ctas` caps the persistent grid.
 // Returns cudaErrorNotSupported for shapes it does not handle.
-cudaError_t launch_gemm_tc(const GemmProblem& p, bool swap_ab, int row_tile, int max_ctas, int* status,
-                           cudaStream_t stream, int* n_launches);
+// `dense` (optional) is computed in the same launch with the same `gated` epilogue.
+cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bool swap_ab, int row_tile,
+                           int max_ctas, int* status, cudaStream_t stream, int* n_launches);
 // One-time driver entry-point lookup for tensor-map encoding; returns false (with a reason) if unavailable.
 bool gemm_tc_init(const char** why);
 
