@@ -452,6 +452,25 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None  # sampled over the timed region and its per-kernel repeat
     stage_us = {n: (1e3 * ms / c if c else None) for n, (ms, c) in prof.items()}
 
+    # ---- variant: GEMM1 gathers its rows from x while it runs (no x_perm is written or re-read)
+    fused = None
+    if not args.quick:
+        ctx_g = B.MoeContext(B.make_config(H, E, k, I, shape.shared_I, T, B.MOE_PHASE_PREFILL, row_gather=1),
+                             stream=stream, device=dev)
+
+        def step_g(i):
+            a = acts[i % n_in]
+            ctx_g.layer(a["x"], a["logits"], a["bias"], *wargs, out=out, bufs=bufs)
+
+        with torch.cuda.stream(stream):
+            for i in range(args.warmup):
+                step_g(i)
+        ms_g = timed(args.steps, step_g) / args.steps
+        assert ctx_g.moe_ctx_status() == B.MOE_OK
+        ctx_g.close()
+        fused = {"ms_per_step": ms_g, "value": whole_job_rate(T, world, ms_g * 1e-3), "unit": UNIT,
+                 "note": "row_gather=1: stage a5 fused into GEMM1 (cp.async row gather), x_perm not materialised"}
+
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region
     e2e_value = None
     if not args.quick:
@@ -529,7 +548,7 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": T * E * 4 + T * H * 2,
                     "d2h_bytes_per_step": T * H * 2},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu_baseline,
-            "stages": stages}
+            "stages": stages, "fused_row_gather": fused}
     ctx.close()
     del w, acts
     torch.cuda.empty_cache()

@@ -77,6 +77,10 @@ typedef struct {
                            context may occupy (the analogue of the paper's separate
                            communication-SM budgets per phase)                          */
   int32_t gemm_variant; /* moe_gemm_variant                                             */
+  int32_t row_gather;   /* 0: moe_dispatch_layout writes x_perm (stage a5 is its own kernel).
+                           1: with the large-M GEMM variant, GEMM1 gathers its rows from x
+                              through perm while it runs; x_perm is not written, and x must
+                              be passed to moe_grouped_ffn.  Ignored by the other variants. */
   float routed_scale;   /* multiplies the routed weights; 1.0f unless the model says so */
 } moe_config;
 
@@ -146,7 +150,8 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
  * act, y_perm and y_shared are stored as bf16 (round to nearest even) in the workspace.
  * w_gate_up [E,2I,H] bf16 (rows 0..I-1 gate, I..2I-1 up), w_down [E,H,I] bf16,
  * ws_gate_up [2I_s,H], ws_down [H,I_s] bf16 (required iff S = 1), x [T,H] bf16 (read by the
- * shared expert; required iff S = 1).  Weights are read-only and may be shared by contexts. */
+ * shared expert and by the row gather; required iff S = 1 or row_gather = 1; it must be the x
+ * that moe_dispatch_layout was given).  Weights are read-only and may be shared by contexts. */
 moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_down, const void* x,
                            const void* ws_gate_up, const void* ws_down, int32_t T);
 

@@ -39,7 +39,7 @@ class moe_config(ctypes.Structure):
     _fields_ = [("hidden", ctypes.c_int32), ("n_experts", ctypes.c_int32), ("top_k", ctypes.c_int32),
                 ("inter", ctypes.c_int32), ("n_shared", ctypes.c_int32), ("shared_inter", ctypes.c_int32),
                 ("max_tokens", ctypes.c_int32), ("phase", ctypes.c_int32), ("sm_budget", ctypes.c_int32),
-                ("gemm_variant", ctypes.c_int32), ("routed_scale", ctypes.c_float)]
+                ("gemm_variant", ctypes.c_int32), ("row_gather", ctypes.c_int32), ("routed_scale", ctypes.c_float)]
 
 
 class moe_stage_times(ctypes.Structure):
@@ -126,9 +126,9 @@ def _dev(t: Optional[torch.Tensor], dtype, name):
 
 
 def make_config(hidden, n_experts, top_k, inter, shared_inter=0, max_tokens=1, phase=MOE_PHASE_PREFILL, sm_budget=0,
-                gemm_variant=MOE_GEMM_AUTO, routed_scale=1.0) -> moe_config:
+                gemm_variant=MOE_GEMM_AUTO, routed_scale=1.0, row_gather=0) -> moe_config:
     return moe_config(hidden, n_experts, top_k, inter, 1 if shared_inter else 0, shared_inter, max_tokens, phase,
-                      sm_budget, gemm_variant, routed_scale)
+                      sm_budget, gemm_variant, row_gather, routed_scale)
 
 
 def moe_ctx_workspace_bytes(cfg: moe_config) -> int:

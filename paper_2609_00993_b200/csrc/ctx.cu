@@ -88,6 +88,7 @@ const char* validate_config(const moe_config* c) {
   if (c->phase != MOE_PHASE_PREFILL && c->phase != MOE_PHASE_DECODE) return "phase must be MOE_PHASE_PREFILL or MOE_PHASE_DECODE";
   if (c->sm_budget < 0) return "sm_budget must be >= 0";
   if (c->gemm_variant < MOE_GEMM_AUTO || c->gemm_variant > MOE_GEMM_VALIDATION) return "unknown gemm_variant";
+  if (c->row_gather != 0 && c->row_gather != 1) return "row_gather must be 0 or 1";
   if (!(c->routed_scale == c->routed_scale)) return "routed_scale is NaN";
   return nullptr;
 }
@@ -208,6 +209,9 @@ int gemm_variant_of(const moe_ctx* ctx) {
   const int v = ctx->cfg.gemm_variant;
   return v != MOE_GEMM_AUTO ? v : (ctx->cfg.phase == MOE_PHASE_DECODE ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M);
 }
+
+// GEMM1 gathers its rows itself only on the large-M tensor-core variant.
+bool gathers_rows(const moe_ctx* ctx) { return ctx->cfg.row_gather == 1 && gemm_variant_of(ctx) == MOE_GEMM_LARGE_M; }
 
 // `dense` (the shared expert's pass, or nullptr) rides in the same launch on the tensor-core path.
 cudaError_t run_gemm(moe_ctx* ctx, const moe::GemmProblem& p, const moe::GemmDenseGroup* dense, int T, int* n) {
@@ -402,7 +406,7 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
     e = moe::launch_layout(topk_idx, (int64_t)T * ctx->cfg.top_k, ctx->cfg.n_experts, ctx->counts, ctx->offsets,
                            ctx->perm, ctx->inv_perm, b.scan, ctx->status, ctx->stream, &n);
   }
-  if (e == cudaSuccess && x != nullptr) {
+  if (e == cudaSuccess && x != nullptr && !gathers_rows(ctx)) {
     StageTimer tm(ctx, 2);
     e = moe::launch_permute(x, ctx->inv_perm, b.x_perm, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->status, ctx->stream,
                             &n);
@@ -424,6 +428,7 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
   const bool shared = ctx->cfg.n_shared != 0;
   if (shared && (!ws_gate_up || !ws_down || (!x && T > 0)))
     return fail(ctx, MOE_ERR_INVALID_ARG, "the shared expert needs ws_gate_up, ws_down and x");
+  if (gathers_rows(ctx) && !x && T > 0) return fail(ctx, MOE_ERR_INVALID_ARG, "the row gather needs x");
   if (misaligned(w_gate_up) || misaligned(w_down) || misaligned(x) || misaligned(ws_gate_up) || misaligned(ws_down))
     return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
   DeviceGuard guard(ctx->device);
@@ -447,6 +452,11 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
     };
     moe::GemmProblem g1{b.x_perm, w_gate_up, b.act, ctx->offsets, 0, Ncap, N, c.n_experts, c.inter, c.hidden, true};
     moe::GemmProblem g2{b.act, w_down, b.y_perm, ctx->offsets, 0, Ncap, N, c.n_experts, c.hidden, c.inter, false};
+    if (gathers_rows(ctx)) {
+      g1.gather_src = x;
+      g1.perm = ctx->perm;
+      g1.top_k = c.top_k;
+    }
     moe::GemmDenseGroup s1{x, ws_gate_up, b.act_shared, T, c.shared_inter, c.hidden};
     moe::GemmDenseGroup s2{b.act_shared, ws_down, b.y_shared, T, c.hidden, c.shared_inter};
     // Unsegmented: the shared expert's two passes ride in the routed launches (two launches in all).

@@ -35,6 +35,9 @@ constexpr int kThreads = 192;
 constexpr int kEpilogueWarps = 4;
 constexpr int kProducerWarp = 4;
 constexpr int kMmaWarp = 5;
+constexpr int kGatherWarp0 = 6;      // row-gather variant: warps 6..9 fill the X tile themselves
+constexpr int kGatherThreads = 128;
+constexpr int kThreadsGather = kThreads + kGatherThreads;
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -52,6 +55,12 @@ struct TcParams {
   int32_t n_stages;
   int32_t x_tile_bytes;    // row_tile * 128
   int* status;
+  // row-gather variant: row p of the grouped operand is gather_src[perm[p] / top_k, :] (gather_src2[p, :] for
+  // the dense group); no permuted copy of the rows exists
+  const __nv_bfloat16* gather_src;
+  const __nv_bfloat16* gather_src2;
+  const int32_t* perm;
+  int32_t top_k;
   // optional dense group (shared expert) computed by the same launch; rows2 == 0: none
   int32_t rows2;
   int32_t n_feat2;
@@ -158,6 +167,16 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// 16-byte asynchronous copy global -> shared (generic proxy), grouped per thread
+__device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+// The mbarrier receives one arrival (already counted in its initial count) once all cp.async copies this thread
+// has issued so far are complete.
+__device__ __forceinline__ void cp_async_arrive_on(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
 // Shared-memory matrix descriptor: K-major tile of 128-byte rows written by TMA with the 128-byte swizzle;
 // 8-row groups are 1024 bytes apart (stride byte offset), the leading byte offset is unused for this layout.
 __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr) {
@@ -212,8 +231,12 @@ __device__ __forceinline__ Tile decode_tile(int tile, int dense_tiles, int n_ft2
 }
 
 // ------------------------------------------------------------------------------------- the kernel
-template <bool SWAP, bool GATED>
-__global__ void __launch_bounds__(kThreads, 1)
+// GATHER (large-M, gated pass only): the token rows are not read from a permuted copy.  Four extra warps copy
+// each row's 128-byte slice for the current k-block from its source row (perm[p] / top_k) into the X tile with
+// 16-byte cp.async, in the same 128-byte-swizzled layout TMA would produce; the stage's barrier counts one
+// arrival per gather thread, delivered when that thread's copies have landed.  TMA then carries the weights only.
+template <bool SWAP, bool GATED, bool GATHER>
+__global__ void __launch_bounds__(GATHER ? kThreadsGather : kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_x2, const __grid_constant__ CUtensorMap map_w2,
                        const __grid_constant__ TcParams p) {
@@ -275,7 +298,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   }
   if (threadIdx.x == 32) {
     for (int s = 0; s < p.n_stages; ++s) {
-      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_full + 8u * s, GATHER ? 1 + kGatherThreads : 1);
       mbar_init(bar_empty + 8u * s, 1);
     }
     for (int a = 0; a < 2; ++a) {
@@ -311,10 +334,10 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t full = bar_full + 8u * s;
           const uint32_t st = base_addr + s * (uint32_t)stage_bytes;
-          mbar_expect_tx(full, (uint32_t)stage_bytes);
+          mbar_expect_tx(full, GATHER ? 2u * kWBoxBytes : (uint32_t)stage_bytes);
           tma_load_3d(st, mw, full, kb * kBlockK, w_row0, w_e);
           tma_load_3d(st + kWBoxBytes, mw, full, kb * kBlockK, w_row1, w_e);
-          tma_load_2d(st + 2 * kWBoxBytes, mx, full, kb * kBlockK, t.row0);
+          if (!GATHER) tma_load_2d(st + 2 * kWBoxBytes, mx, full, kb * kBlockK, t.row0);
         }
       }
       if (!ok) {
@@ -340,6 +363,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const uint32_t s = it % (uint32_t)p.n_stages, ph = (it / (uint32_t)p.n_stages) & 1u;
           if (!mbar_wait(bar_full + 8u * s, ph, abort_flag)) { ok = false; break; }
+          if (GATHER) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // X rows came by cp.async
           tc_fence_after();
           const uint32_t st = base_addr + s * (uint32_t)stage_bytes;
           const uint64_t dw0 = umma_smem_desc(st);
@@ -364,6 +388,54 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         *abort_flag = 1;
         atomicCAS(p.status, kStOk, kStTimeout);
       }
+    }
+  } else if (GATHER && warp >= kGatherWarp0) {
+    // ================================================================= row gather (warps 6-9)
+    // thread g owns the 16-byte piece (g & 7) of rows (g >> 3) + 16 i, i < 8, of every stage
+    const int g = (int)threadIdx.x - kGatherWarp0 * 32;
+    const int piece = g & 7, rbase = g >> 3;
+    const uint32_t dst_off = (uint32_t)(rbase * 128 + ((piece ^ (rbase & 7)) << 4));  // 128-byte swizzle
+    uint32_t it = 0;
+    bool ok = true;
+    // The source row of each of this thread's 8 rows (flat slot = perm[row]; source row = slot / top_k; the
+    // dense group's rows are their own source) is fetched one tile ahead, so that the dependent perm load is
+    // not on the path of a tile's first copies.  -1: the row lies past the tile's end.
+    int slot_next[8];
+    auto fetch_slots = [&](int tile, int (&slot)[8]) {
+      if (tile >= total_tiles) return;
+      const Tile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, seg, tile_rows);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int r = rbase + 16 * i;
+        slot[i] = -1;
+        if (r < t.rows) slot[i] = t.dense ? (t.row0 + r) * p.top_k : __ldg(p.perm + t.row0 + r);
+      }
+    };
+    fetch_slots(unit, slot_next);
+    for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
+      const Tile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, seg, tile_rows);
+      const __nv_bfloat16* src = t.dense ? p.gather_src2 : p.gather_src;
+      const int Kt = t.dense ? p.K2 : p.K;
+      const __nv_bfloat16* row_ptr[8];  // nullptr: the row is left as it is; its result is never stored
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        row_ptr[i] = slot_next[i] < 0 ? nullptr : src + (size_t)(slot_next[i] / p.top_k) * Kt + piece * 8;
+      fetch_slots(tile + n_units, slot_next);
+      const int num_kb = t.dense ? num_kb2 : num_kb1;
+      for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        const uint32_t s = it % (uint32_t)p.n_stages, ph = (it / (uint32_t)p.n_stages) & 1u;
+        if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t xs = base_addr + s * (uint32_t)stage_bytes + 2 * kWBoxBytes + dst_off;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (row_ptr[i] != nullptr) cp_async_16(xs + (uint32_t)(i * 16 * 128), row_ptr[i] + kb * kBlockK);
+        // one arrival on the stage's barrier, delivered by the hardware when this thread's copies have landed
+        cp_async_arrive_on(bar_full + 8u * s);
+      }
+    }
+    if (!ok) {
+      *abort_flag = 1;
+      atomicCAS(p.status, kStOk, kStTimeout);
     }
   } else {
     // ================================================================= epilogue (warps 0-3)
@@ -419,10 +491,9 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         for (int pc = 0; pc < kPairs; ++pc) {
           const int f0 = t.ft * kFeatPerTile + pc * 64;
           if (f0 >= n_feat) break;  // uniform across the CTA
-          uint32_t packed[32];
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
-            uint32_t ra[32];
+            uint32_t ra[32], packed[16];
             tmem_ld32(d0 + (uint32_t)(pc * 64 + h * 32), ra);
             if (GATED) {
               uint32_t rb[32];
@@ -430,23 +501,22 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
               tmem_ld_wait();
 #pragma unroll
               for (int i = 0; i < 16; ++i)
-                packed[h * 16 + i] = pack_bf16(silu_mul(__uint_as_float(ra[2 * i]), __uint_as_float(rb[2 * i])),
-                                               silu_mul(__uint_as_float(ra[2 * i + 1]), __uint_as_float(rb[2 * i + 1])));
+                packed[i] = pack_bf16(silu_mul(__uint_as_float(ra[2 * i]), __uint_as_float(rb[2 * i])),
+                                      silu_mul(__uint_as_float(ra[2 * i + 1]), __uint_as_float(rb[2 * i + 1])));
             } else {
               tmem_ld_wait();
 #pragma unroll
-              for (int i = 0; i < 16; ++i)
-                packed[h * 16 + i] = pack_bf16(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1]));
+              for (int i = 0; i < 16; ++i) packed[i] = pack_bf16(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1]));
             }
-          }
-          if (pc == kPairs - 1 || f0 + 64 >= n_feat) {
-            release_acc();  // the accumulator has been read completely: hand it back before the stores go out
-            released = true;
-          }
+            if (h == 1 && (pc == kPairs - 1 || f0 + 64 >= n_feat)) {
+              release_acc();  // the accumulator has been read completely: hand it back before the stores go out
+              released = true;
+            }
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            *reinterpret_cast<uint4*>(stage_tile + lane * 128 + ((j ^ (lane & 7)) << 4)) =
-                make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+            for (int j = 0; j < 4; ++j)
+              *reinterpret_cast<uint4*>(stage_tile + lane * 128 + (((h * 4 + j) ^ (lane & 7)) << 4)) =
+                  make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+          }
           __syncwarp();
 #pragma unroll
           for (int it = 0; it < 8; ++it) {
@@ -502,11 +572,12 @@ bool encode_map(CUtensorMap* map, const void* base, int rank, const uint64_t* di
 }
 
 template <typename Kernel>
-cudaError_t launch_variant(Kernel kern, const CUtensorMap& mx, const CUtensorMap& mw, const CUtensorMap& mx2,
-                           const CUtensorMap& mw2, const TcParams& prm, int grid, size_t smem, cudaStream_t stream) {
+cudaError_t launch_variant(Kernel kern, int threads, const CUtensorMap& mx, const CUtensorMap& mw,
+                           const CUtensorMap& mx2, const CUtensorMap& mw2, const TcParams& prm, int grid, size_t smem,
+                           cudaStream_t stream) {
   cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (err != cudaSuccess) return err;
-  kern<<<grid, kThreads, smem, stream>>>(mx, mw, mx2, mw2, prm);
+  kern<<<grid, threads, smem, stream>>>(mx, mw, mx2, mw2, prm);
   return cudaGetLastError();
 }
 
@@ -536,6 +607,10 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
   if (g_encode == nullptr && !gemm_tc_init(nullptr)) return cudaErrorNotSupported;
   if (p.K % 8 != 0 || p.n_feat % 8 != 0 || p.E < 1 || p.E > 1024) return cudaErrorNotSupported;
   if (!swap_ab) row_tile = 128;
+  const bool gather = p.gather_src != nullptr;
+  if (gather && (swap_ab || !p.gated || p.perm == nullptr || p.top_k < 1 || p.K % kBlockK != 0 ||
+                 (dense != nullptr && dense->K % kBlockK != 0)))
+    return cudaErrorNotSupported;
   if (row_tile < 16 || row_tile > 128 || (row_tile & (row_tile - 1)) != 0) return cudaErrorNotSupported;
   if (p.rows_bound > 0x7fffffffLL / 2) return cudaErrorNotSupported;
 
@@ -543,10 +618,12 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
   const uint64_t w_rows = (uint64_t)(p.gated ? 2 : 1) * (uint64_t)p.n_feat;
   CUtensorMap mx, mw;
   {
-    const uint64_t dims[2] = {(uint64_t)p.K, (uint64_t)p.rows_bound};
+    const uint64_t src_rows = gather ? (uint64_t)((p.rows_bound + p.top_k - 1) / p.top_k) : (uint64_t)p.rows_bound;
+    const uint64_t dims[2] = {(uint64_t)p.K, src_rows};
     const uint64_t str[1] = {(uint64_t)p.K * 2};
     const uint32_t box[2] = {(uint32_t)kBlockK, (uint32_t)row_tile};
-    if (!encode_map(&mx, p.A, 2, dims, str, box)) return cudaErrorInvalidValue;
+    // with the row gather no tensor map of the token rows is used; encode the source so that the map is valid
+    if (!encode_map(&mx, gather ? p.gather_src : p.A, 2, dims, str, box)) return cudaErrorInvalidValue;
   }
   {
     const uint64_t dims[3] = {(uint64_t)p.K, w_rows, (uint64_t)groups};
@@ -571,6 +648,10 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
     if (!encode_map(&mw2, dense->W, 3, dw, sw, bw)) return cudaErrorInvalidValue;
   }
   TcParams prm;
+  prm.gather_src = static_cast<const __nv_bfloat16*>(p.gather_src);
+  prm.gather_src2 = dense ? static_cast<const __nv_bfloat16*>(dense->A) : nullptr;
+  prm.perm = p.perm ? p.perm + 0 : nullptr;
+  prm.top_k = p.top_k;
   prm.rows2 = dense ? dense->rows : 0;
   prm.n_feat2 = dense ? dense->n_feat : 8;
   prm.K2 = dense ? dense->K : 8;
@@ -604,10 +685,14 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
   int grid = (int)(tiles < (int64_t)max_ctas ? tiles : (int64_t)max_ctas);
   if (grid < 1) grid = 1;
   cudaError_t err;
-  if (swap_ab) err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true>, mx, mw, mx2, mw2, prm, grid, smem, stream)
-                             : launch_variant(grouped_gemm_tc_kernel<true, false>, mx, mw, mx2, mw2, prm, grid, smem, stream);
-  else err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true>, mx, mw, mx2, mw2, prm, grid, smem, stream)
-                     : launch_variant(grouped_gemm_tc_kernel<false, false>, mx, mw, mx2, mw2, prm, grid, smem, stream);
+  if (gather)
+    err = launch_variant(grouped_gemm_tc_kernel<false, true, true>, kThreadsGather, mx, mw, mx2, mw2, prm, grid, smem, stream);
+  else if (swap_ab)
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
+                  : launch_variant(grouped_gemm_tc_kernel<true, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
+  else
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
+                  : launch_variant(grouped_gemm_tc_kernel<false, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }

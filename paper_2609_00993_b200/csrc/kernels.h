@@ -51,6 +51,11 @@ struct GemmProblem {
   bool gated;
   int32_t e_begin = 0;     // this launch covers experts [e_begin, e_end) only (a prefill segment);
   int32_t e_end = -1;      // e_end < 0 means E
+  // Row gather (tensor-core large-M gated pass only): when gather_src is set, A is not read; row p of the
+  // operand is gather_src[perm[p] / top_k, :] instead (gather_src is bf16 [T, K], perm is [rows_bound]).
+  const void* gather_src = nullptr;
+  const int32_t* perm = nullptr;
+  int32_t top_k = 1;
 };
 
 // A dense group (the shared expert) that rides in the same launch as a grouped problem: its tiles are added

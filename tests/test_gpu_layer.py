@@ -17,8 +17,9 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-def _ctx_for(shape, phase, max_tokens=None, sm_budget=0, stream=None):
-    cfg = B.make_config(shape.H, shape.E, shape.k, shape.I, shape.shared_I, max_tokens or shape.T, phase, sm_budget)
+def _ctx_for(shape, phase, max_tokens=None, sm_budget=0, stream=None, row_gather=0):
+    cfg = B.make_config(shape.H, shape.E, shape.k, shape.I, shape.shared_I, max_tokens or shape.T, phase, sm_budget,
+                        row_gather=row_gather)
     return B.MoeContext(cfg, stream=stream)
 
 
@@ -72,11 +73,12 @@ def test_c1_tiny_prefill_full_comparison():
     ctx.close()
 
 
-def test_c3_prefill_qwen3_shaped():
+@pytest.mark.parametrize("row_gather", [0, 1])
+def test_c3_prefill_qwen3_shaped(row_gather):
     shape = wl.C3
     w = wl.make_weights(shape, 3, DEV)
     a = wl.make_activations(shape, 3, DEV)
-    ctx = _ctx_for(shape, B.MOE_PHASE_PREFILL)
+    ctx = _ctx_for(shape, B.MOE_PHASE_PREFILL, row_gather=row_gather)
     out, bufs = _step(ctx, a, w)
     counts, offsets, perm = _check_integers(bufs, a["logits"], a["bias"], shape, shape.T)
     toks = sample_tokens(shape.T, counts, offsets, perm, shape.k, 48, seed=3)

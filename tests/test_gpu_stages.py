@@ -13,8 +13,8 @@ DEV = "cuda"
 
 
 def _ctx(H=256, E=8, k=2, I=512, shared_I=0, max_tokens=64, phase=B.MOE_PHASE_PREFILL, variant=B.MOE_GEMM_AUTO,
-         sm_budget=0):
-    cfg = B.make_config(H, E, k, I, shared_I, max_tokens, phase, sm_budget, variant)
+         sm_budget=0, row_gather=0):
+    cfg = B.make_config(H, E, k, I, shared_I, max_tokens, phase, sm_budget, variant, row_gather=row_gather)
     return B.MoeContext(cfg)
 
 
@@ -170,9 +170,10 @@ def _oracle_step(a, w, k, emulate=False):
                         None if w["ws_down"] is None else wl.bits(w["ws_down"]), emulate_bf16=emulate)
 
 
-VARIANTS = [(B.MOE_GEMM_VALIDATION, B.MOE_PHASE_PREFILL, "validation"),
-            (B.MOE_GEMM_LARGE_M, B.MOE_PHASE_PREFILL, "large-M"),
-            (B.MOE_GEMM_SMALL_M, B.MOE_PHASE_DECODE, "small-M")]
+VARIANTS = [(B.MOE_GEMM_VALIDATION, B.MOE_PHASE_PREFILL, "validation", 0),
+            (B.MOE_GEMM_LARGE_M, B.MOE_PHASE_PREFILL, "large-M", 0),
+            (B.MOE_GEMM_LARGE_M, B.MOE_PHASE_PREFILL, "large-M-gather", 1),  # GEMM1 gathers its rows; no x_perm
+            (B.MOE_GEMM_SMALL_M, B.MOE_PHASE_DECODE, "small-M", 0)]
 
 SHAPES = [
     # T,   H,    E,  k, I,   shared_I
@@ -183,9 +184,9 @@ SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("variant,phase,vname", VARIANTS)
+@pytest.mark.parametrize("variant,phase,vname,row_gather", VARIANTS)
 @pytest.mark.parametrize("T,H,E,k,I,shared_I", SHAPES)
-def test_ffn_and_combine_match_oracle(variant, phase, vname, T, H, E, k, I, shared_I):
+def test_ffn_and_combine_match_oracle(variant, phase, vname, row_gather, T, H, E, k, I, shared_I):
     shape = wl.LayerShape("t", T=T, H=H, E=E, k=k, I=I, shared_I=shared_I, select_bias=True)
     w = wl.make_weights(shape, 5, DEV)
     # scale the weights up so that the outputs are O(1) and a wrong tile or a dropped k-block is far outside tolerance
@@ -193,7 +194,7 @@ def test_ffn_and_combine_match_oracle(variant, phase, vname, T, H, E, k, I, shar
         if w[n] is not None:
             w[n] = (w[n].float() * (1.0 / (0.02 * (w[n].shape[-1] ** 0.5)))).to(torch.bfloat16)
     a = wl.make_activations(shape, 6, DEV)
-    ctx = _ctx(H=H, E=E, k=k, I=I, shared_I=shared_I, max_tokens=T, phase=phase, variant=variant)
+    ctx = _ctx(H=H, E=E, k=k, I=I, shared_I=shared_I, max_tokens=T, phase=phase, variant=variant, row_gather=row_gather)
     out, bufs = _run_step(ctx, a, w, T)
     ref = _oracle_step(a, w, k)
     emu = _oracle_step(a, w, k, emulate=True)
