@@ -241,6 +241,25 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm):
     alone = time_d(iters)
     res["alone_us"] = {"p50": percentile(alone, 50), "p99": percentile(alone, 99), "max": max(alone)}
 
+    # the same D step replayed from a CUDA graph (stable phase-owned addresses): launch overhead off the path
+    try:
+        graph = torch.cuda.CUDAGraph()
+        a0 = ads[0]
+        with torch.cuda.graph(graph, stream=sd):
+            ctx_d.layer(a0["x"], a0["logits"], a0["bias"], *wargs, out=od, bufs=bd)
+        evs = []
+        for _ in range(iters):
+            with torch.cuda.stream(sd):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(sd); graph.replay(); e1.record(sd)
+            evs.append((e0, e1))
+        torch.cuda.synchronize(dev)
+        rep = [1e3 * a.elapsed_time(b) for a, b in evs]
+        res["graph_replay_us"] = {"p50": percentile(rep, 50), "p99": percentile(rep, 99)}
+        del graph
+    except Exception as exc:
+        res["graph_replay_us"] = {"error": repr(exc)}
+
     ctx_p = mk(wl.C4_P, B.MOE_PHASE_PREFILL, sp)
     bp = B.alloc_step_buffers(wl.C4_P.T, 8, 256, dev)
     op = torch.empty(wl.C4_P.T, 7168, dtype=torch.bfloat16, device=dev)

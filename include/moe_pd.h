@@ -27,6 +27,13 @@
  *
  * Per step, in order:  moe_route (optional) -> moe_dispatch_layout -> moe_grouped_ffn
  * -> moe_combine.  Any other order returns MOE_ERR_STATE.
+ *
+ * CUDA graphs.  The four step calls only enqueue kernels, so a step may be recorded while the
+ * context's stream is being captured and replayed later (D keeps stable graph addresses: the
+ * graph holds the buffer set that was current at capture, whatever the double-buffer index
+ * does afterwards).  Run one step eagerly first (it configures the kernels), keep every
+ * array the step touches alive and in place, and do not capture moe_layer_host,
+ * moe_ctx_status or moe_ctx_read_profile (they synchronise).
  */
 #ifndef MOE_PD_H_
 #define MOE_PD_H_

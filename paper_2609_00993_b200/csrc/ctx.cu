@@ -5,7 +5,9 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <mutex>
+#include <utility>
 #include <new>
 #include <vector>
 
@@ -169,9 +171,21 @@ struct DeviceGuard {
   }
 };
 
+bool capturing(const moe_ctx* ctx) {
+  cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(ctx->stream, &st) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return false;
+  }
+  return st != cudaStreamCaptureStatusNone;
+}
+
+// After the last enqueue of a call: count the launches and mark the stream position.  While the stream is
+// being captured into a CUDA graph nothing executes, so there is no position to mark (and an event recorded
+// during capture could not be queried later).
 void mark(moe_ctx* ctx, int n) {
   ctx->launches += n;
-  cudaEventRecord(ctx->done, ctx->stream);
+  if (!capturing(ctx)) cudaEventRecord(ctx->done, ctx->stream);
 }
 
 // Brackets the launches of one stage with events when profiling is on.
@@ -179,7 +193,7 @@ struct StageTimer {
   moe_ctx* ctx;
   moe_ctx::Span* span = nullptr;
   StageTimer(moe_ctx* c, int stage) : ctx(c) {
-    if (!c->profiling) return;
+    if (!c->profiling || capturing(c)) return;  // event timing is meaningless inside a capture
     if (c->spans_used == c->spans.size()) {
       moe_ctx::Span s;
       if (cudaEventCreate(&s.beg) != cudaSuccess || cudaEventCreate(&s.end) != cudaSuccess) return;
@@ -231,6 +245,27 @@ cudaError_t run_gemm(moe_ctx* ctx, const moe::GemmProblem& p, const moe::GemmDen
 }
 
 }  // namespace
+
+namespace moe {
+
+cudaError_t ensure_dynamic_smem_impl(const void* kern, size_t bytes) {
+  static std::mutex mu;
+  static std::map<std::pair<const void*, int>, size_t> configured;  // (kernel, device) -> largest size set
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  std::lock_guard<std::mutex> lock(mu);
+  size_t& have = configured[{kern, dev}];
+  if (bytes <= have) return cudaSuccess;
+  if (bytes > 48 * 1024) {
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (err != cudaSuccess) return err;
+  }
+  have = bytes;
+  return cudaSuccess;
+}
+
+}  // namespace moe
 
 extern "C" {
 
@@ -445,7 +480,7 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
     int bound = 0;
     auto boundary = [&]() {
       if (ctx->seg_experts > 0 && ctx->boundary_fn) {
-        cudaEventRecord(ctx->done, ctx->stream);
+        if (!capturing(ctx)) cudaEventRecord(ctx->done, ctx->stream);
         ctx->boundary_fn(ctx->boundary_user, bound, n_bound);
       }
       ++bound;

@@ -575,7 +575,7 @@ template <typename Kernel>
 cudaError_t launch_variant(Kernel kern, int threads, const CUtensorMap& mx, const CUtensorMap& mw,
                            const CUtensorMap& mx2, const CUtensorMap& mw2, const TcParams& prm, int grid, size_t smem,
                            cudaStream_t stream) {
-  cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t err = ensure_dynamic_smem(kern, smem);
   if (err != cudaSuccess) return err;
   kern<<<grid, threads, smem, stream>>>(mx, mw, mx2, mw2, prm);
   return cudaGetLastError();

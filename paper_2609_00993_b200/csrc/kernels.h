@@ -6,6 +6,14 @@
 
 namespace moe {
 
+// Raises a kernel's dynamic shared-memory limit once per kernel, device and size, so that steady-state launches
+// make no driver calls besides the launch itself (which also keeps them legal while a stream is being captured).
+cudaError_t ensure_dynamic_smem_impl(const void* kern, size_t bytes);
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kern, size_t bytes) {
+  return ensure_dynamic_smem_impl(reinterpret_cast<const void*>(kern), bytes);
+}
+
 // Device status codes (same values as moe_status in the public header).
 constexpr int kStOk = 0;
 constexpr int kStTimeout = 6;

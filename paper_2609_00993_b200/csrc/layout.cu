@@ -269,10 +269,7 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
   if (n_slots <= (int64_t)kFusedWarps * kFusedMaxSlotsPerWarp && fused_smem <= 200 * 1024) {
     int spw = (int)((n_slots + kFusedWarps - 1) / kFusedWarps);
     spw = (spw + 31) / 32 * 32;
-    if (fused_smem > 48 * 1024) {
-      err = cudaFuncSetAttribute(layout_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fused_smem);
-      if (err != cudaSuccess) return err;
-    }
+    if ((err = ensure_dynamic_smem(layout_fused_kernel, fused_smem)) != cudaSuccess) return err;
     layout_fused_kernel<<<1, kFusedWarps * 32, fused_smem, stream>>>(topk_idx, (int)n_slots, E, spw, counts, offsets,
                                                                      perm, inv_perm, status);
     err = cudaGetLastError();

@@ -220,6 +220,7 @@ combine_kernel(const __nv_bfloat16* __restrict__ y_perm, const __nv_bfloat16* __
   }
 }
 
+// CTAs of `kern` that fit on the device at once (one resident wave for a persistent grid).
 int resident_ctas(const void* kern, int threads, size_t smem) {
   int dev = 0, sms = 148, per_sm = 1;
   cudaGetDevice(&dev);
@@ -237,7 +238,7 @@ cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm,
   const int col_blocks = (H + kPermuteChunkCols - 1) / kPermuteChunkCols;
   const int slot_bytes = (H < kPermuteChunkCols ? H : kPermuteChunkCols) * 2;
   const size_t smem = (size_t)kPermuteSlots * slot_bytes + 8 * kPermuteSlots;
-  cudaError_t err = cudaFuncSetAttribute(permute_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t err = ensure_dynamic_smem(permute_rows_kernel, smem);
   if (err != cudaSuccess) return err;
   const long long n_items = (long long)T * col_blocks;
   const long long cap = resident_ctas(reinterpret_cast<const void*>(permute_rows_kernel), 32, smem);
@@ -261,7 +262,7 @@ cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32
   if (stages > kCombineMaxStages) stages = kCombineMaxStages;
   if (stages < 2) stages = 2;
   const size_t smem = (size_t)stages * stage_bytes + 16 * stages;
-  cudaError_t err = cudaFuncSetAttribute(combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t err = ensure_dynamic_smem(combine_kernel, smem);
   if (err != cudaSuccess) return err;
   const long long n_items = (long long)T * col_blocks;
   const long long cap = resident_ctas(reinterpret_cast<const void*>(combine_kernel), kCombineThreads, smem);

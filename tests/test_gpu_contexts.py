@@ -202,3 +202,48 @@ def test_decode_step_admitted_at_a_prefill_boundary():
     assert p.moe_ctx_status() == B.MOE_OK and d.moe_ctx_status() == B.MOE_OK
     p.moe_ctx_set_segments(0)
     p.close(); d.close()
+
+
+def test_decode_step_replays_from_a_cuda_graph():
+    """D retains stable graph addresses: a captured D step replays with new inputs written into the same
+    tensors and gives the bits of the eager step, with a P context busy on another stream or idle."""
+    shape = wl.LayerShape("t", T=48, H=512, E=16, k=4, I=256, shared_I=128, select_bias=True)
+    w = wl.make_weights(shape, 1, DEV)
+    a1, a2 = wl.make_activations(shape, 2, DEV), wl.make_activations(shape, 3, DEV)
+    sd, sp = torch.cuda.Stream(), torch.cuda.Stream()
+    d = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 48, B.MOE_PHASE_DECODE), stream=sd)
+    wargs = (w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+    torch.cuda.synchronize()
+    eager1, _ = d.layer(a1["x"], a1["logits"], a1["bias"], *wargs)
+    eager2, _ = d.layer(a2["x"], a2["logits"], a2["bias"], *wargs)
+    torch.cuda.synchronize()
+    # static inputs/outputs of the graph
+    x, logits, bias = a1["x"].clone(), a1["logits"].clone(), a1["bias"].clone()
+    bufs = B.alloc_step_buffers(48, 4, 16, DEV)
+    out = torch.empty(48, 512, dtype=torch.bfloat16, device=DEV)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=sd):
+        d.layer(x, logits, bias, *wargs, out=out, bufs=bufs)
+    out.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager1)
+    # new inputs in place, and a P context hammering the GPU meanwhile
+    pshape = shape.with_tokens(1024)
+    ap = wl.make_activations(pshape, 4, DEV)
+    p = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 1024, B.MOE_PHASE_PREFILL), stream=sp)
+    x.copy_(a2["x"]); logits.copy_(a2["logits"]); bias.copy_(a2["bias"])
+    torch.cuda.synchronize()
+    for _ in range(3):
+        p.layer(ap["x"], ap["logits"], ap["bias"], *wargs)
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager2)
+    assert d.moe_ctx_status() == B.MOE_OK and p.moe_ctx_status() == B.MOE_OK
+    # eager steps still work after a capture
+    again, _ = d.layer(a1["x"], a1["logits"], a1["bias"], *wargs)
+    torch.cuda.synchronize()
+    assert torch.equal(again, eager1)
+    del g
+    p.close(); d.close()
