@@ -448,7 +448,7 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_dispatch_layout");
   ctx->T = T;
-  ctx->state = x ? ST_LAID_OUT : ST_LAYOUT_ONLY;
+  ctx->state = (x != nullptr || T == 0) ? ST_LAID_OUT : ST_LAYOUT_ONLY;  // an empty batch has no rows to move
   mark(ctx, n);
   return MOE_OK;
 }
