@@ -174,6 +174,36 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
 typedef void (*moe_boundary_fn)(void* user, int32_t boundary, int32_t n_boundaries);
 moe_status moe_ctx_set_segments(moe_ctx* ctx, int32_t experts_per_segment, moe_boundary_fn fn, void* user);
 
+/* Segment turnstile -- the host-side boundary controller (Sections "Rank-Aligned Segment Boundaries" and
+ * "Distributed Segment Turnstile").  Host-only: it orders host enqueue, never waits for GPU work and launches
+ * nothing.  One controller per rank keeps the current P epoch e, the largest reached boundary r (-1 at the start
+ * of an epoch), the permitted endpoint p, the positive span K and the task state.
+ *   P side   moe_turnstile_begin_epoch(e, d_already_enqueued): r = -1; p = K if a D iteration is already
+ *            enqueued, else 0 (so that a ready D is ordered before P enters CUDA).
+ *            moe_turnstile_publish(e, i): step P1/P2 -- publish boundary i (r = i), then wait while i >= p.
+ *            Call it with i = 0 before the first segment is enqueued and with i + 1 after segment i has been
+ *            (the boundary hook of moe_ctx_set_segments is the place).  moe_turnstile_task_done(e) after the
+ *            final segment.
+ *   D side   moe_turnstile_d_enter: step D1 -- if p > 0 wait until r >= p or the epoch is done; *p_active says
+ *            whether a P epoch is running.  The caller then runs its PreDRendezvous over all ranks (any CPU
+ *            barrier), enqueues the D calls (D2), runs its PostDRendezvous (D3) and calls
+ *            moe_turnstile_d_release: step D4 -- p <- p + K for an active epoch, without waiting for P's GPU work.
+ * Rejected with MOE_ERR_STATE: a stale or duplicate epoch, a publication or completion for an epoch that was
+ * never begun (missing producer), a boundary that is not larger than the last one, a boundary beyond the
+ * current permit, beginning an epoch while one is active, destroying a controller with an active epoch.
+ * Every wait takes timeout_ms (negative = unbounded) and returns MOE_ERR_TIMEOUT when it runs out. */
+typedef struct moe_turnstile moe_turnstile;
+moe_status moe_turnstile_create(int32_t span, moe_turnstile** out);
+moe_status moe_turnstile_destroy(moe_turnstile* ts);
+moe_status moe_turnstile_set_span(moe_turnstile* ts, int32_t span);
+moe_status moe_turnstile_begin_epoch(moe_turnstile* ts, int64_t epoch, int32_t d_already_enqueued);
+moe_status moe_turnstile_publish(moe_turnstile* ts, int64_t epoch, int32_t boundary, int32_t timeout_ms);
+moe_status moe_turnstile_task_done(moe_turnstile* ts, int64_t epoch);
+moe_status moe_turnstile_d_enter(moe_turnstile* ts, int32_t timeout_ms, int32_t* p_active);
+moe_status moe_turnstile_d_release(moe_turnstile* ts);
+moe_status moe_turnstile_state(moe_turnstile* ts, int64_t* epoch, int32_t* reached, int32_t* permit, int32_t* span,
+                               int32_t* active);
+
 /* Stage a9 -- weighted combine back to token order:
  *   out[t,:] = sum_j topk_w[t,j] * y_perm[inv_perm[t*k+j],:]  (+ y_shared[t,:]),  fp32 sum, bf16 store.
  * topk_w [T,k] fp32; inv_perm [N] int32 or NULL to use the layout of this step kept by the

@@ -28,7 +28,9 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_CAPACITY", 3:
 EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_destroy", "moe_ctx_status",
            "moe_last_error", "moe_route", "moe_dispatch_layout", "moe_grouped_ffn", "moe_combine", "moe_layer_host",
            "moe_ctx_debug_ptrs", "moe_ctx_launch_count", "moe_ctx_set_profiling", "moe_ctx_read_profile",
-           "moe_dispatch_layout_static", "moe_ctx_set_segments")
+           "moe_dispatch_layout_static", "moe_ctx_set_segments", "moe_turnstile_create", "moe_turnstile_destroy",
+           "moe_turnstile_set_span", "moe_turnstile_begin_epoch", "moe_turnstile_publish", "moe_turnstile_task_done",
+           "moe_turnstile_d_enter", "moe_turnstile_d_release", "moe_turnstile_state")
 
 BOUNDARY_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32)
 
@@ -96,6 +98,13 @@ def load_library() -> ctypes.CDLL:
     lib.moe_ctx_set_profiling.argtypes = [vp, i32]
     lib.moe_ctx_read_profile.restype = i32
     lib.moe_ctx_read_profile.argtypes = [vp, ctypes.POINTER(moe_stage_times)]
+    for name, args in (("moe_turnstile_create", [i32, ctypes.POINTER(vp)]), ("moe_turnstile_destroy", [vp]),
+                       ("moe_turnstile_set_span", [vp, i32]), ("moe_turnstile_begin_epoch", [vp, i64, i32]),
+                       ("moe_turnstile_publish", [vp, i64, i32, i32]), ("moe_turnstile_task_done", [vp, i64]),
+                       ("moe_turnstile_d_enter", [vp, i32, ctypes.POINTER(i32)]), ("moe_turnstile_d_release", [vp]),
+                       ("moe_turnstile_state", [vp, ctypes.POINTER(i64)] + [ctypes.POINTER(i32)] * 4)):
+        getattr(lib, name).restype = i32
+        getattr(lib, name).argtypes = args
     lib.moe_ctx_set_segments.restype = i32
     lib.moe_ctx_set_segments.argtypes = [vp, i32, BOUNDARY_FN, vp]
     lib.moe_dispatch_layout_static.restype = i32
@@ -304,3 +313,49 @@ def moe_dispatch_layout_static(topk_idx, n_experts, counts, offsets, perm, inv_p
     with torch.cuda.device(topk_idx.device):
         return int(lib.moe_dispatch_layout_static(_ptr(topk_idx), T, top_k, n_experts, _ptr(counts), _ptr(offsets),
                                                   _ptr(perm), _ptr(inv_perm), ctypes.c_void_p(s.cuda_stream)))
+
+
+class Turnstile:
+    """One rank's segment-turnstile controller (`moe_turnstile`): host-only, no GPU needed.  Methods return the
+    moe_status code (MOE_OK, MOE_ERR_STATE for a protocol violation, MOE_ERR_TIMEOUT) instead of raising."""
+
+    def __init__(self, span: int = 1):
+        self.lib = load_library()
+        h = ctypes.c_void_p()
+        st = self.lib.moe_turnstile_create(span, ctypes.byref(h))
+        if st != MOE_OK:
+            raise MoeError(st, "moe_turnstile_create")
+        self.handle = h
+
+    def begin_epoch(self, epoch: int, d_already_enqueued: bool = False) -> int:
+        return int(self.lib.moe_turnstile_begin_epoch(self.handle, epoch, int(d_already_enqueued)))
+
+    def publish(self, epoch: int, boundary: int, timeout_ms: int = -1) -> int:
+        return int(self.lib.moe_turnstile_publish(self.handle, epoch, boundary, timeout_ms))
+
+    def task_done(self, epoch: int) -> int:
+        return int(self.lib.moe_turnstile_task_done(self.handle, epoch))
+
+    def d_enter(self, timeout_ms: int = -1):
+        active = ctypes.c_int32(0)
+        st = int(self.lib.moe_turnstile_d_enter(self.handle, timeout_ms, ctypes.byref(active)))
+        return st, bool(active.value)
+
+    def d_release(self) -> int:
+        return int(self.lib.moe_turnstile_d_release(self.handle))
+
+    def set_span(self, span: int) -> int:
+        return int(self.lib.moe_turnstile_set_span(self.handle, span))
+
+    def state(self) -> dict:
+        e = ctypes.c_int64(0)
+        r, p, k, a = (ctypes.c_int32(0) for _ in range(4))
+        self.lib.moe_turnstile_state(self.handle, ctypes.byref(e), ctypes.byref(r), ctypes.byref(p), ctypes.byref(k),
+                                     ctypes.byref(a))
+        return {"epoch": e.value, "reached": r.value, "permit": p.value, "span": k.value, "active": bool(a.value)}
+
+    def destroy(self) -> int:
+        st = int(self.lib.moe_turnstile_destroy(self.handle)) if self.handle else MOE_OK
+        if st == MOE_OK:
+            self.handle = None
+        return st

@@ -247,3 +247,77 @@ def test_decode_step_replays_from_a_cuda_graph():
     assert torch.equal(again, eager1)
     del g
     p.close(); d.close()
+
+
+def test_turnstile_controller_drives_two_contexts_from_two_host_threads():
+    """The paper's protocol end to end on one GPU: a P host thread publishes boundaries from the segment hook and
+    stops at its permitted endpoint (P1/P2); a D host thread waits for P to stand there (D1), enqueues a D step
+    (D2), orders P's next segment after it on the device and moves the endpoint (D4)."""
+    import threading
+    shape = wl.LayerShape("t", T=48, H=512, E=16, k=4, I=256, shared_I=128)
+    pshape = shape.with_tokens(2048)
+    w = wl.make_weights(shape, 1, DEV)
+    ad, ap = wl.make_activations(shape, 2, DEV), wl.make_activations(pshape, 3, DEV)
+    sp, sd = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    d = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 48, B.MOE_PHASE_DECODE), stream=sd)
+    p = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 2048, B.MOE_PHASE_PREFILL), stream=sp)
+    wargs = (w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+    torch.cuda.synchronize()
+    d_alone, _ = d.layer(ad["x"], ad["logits"], None, *wargs)
+    p_alone, _ = p.layer(ap["x"], ap["logits"], None, *wargs)
+    torch.cuda.synchronize()
+
+    ts = B.Turnstile(span=2)
+    n_epochs, errors, d_outs, p_outs = 3, [], [], []
+    p_done = threading.Event()
+
+    def p_thread():
+        try:
+            for e in range(n_epochs):
+                assert ts.begin_epoch(e) == B.MOE_OK
+                assert ts.publish(e, 0, 20000) == B.MOE_OK          # p = 0: a ready D goes first
+
+                def hook(i, n, e=e):
+                    if i + 1 < n:
+                        st = ts.publish(e, i + 1, 20000)
+                        if st != B.MOE_OK:
+                            errors.append(("publish", e, i + 1, st))
+
+                p.moe_ctx_set_segments(4, hook)
+                out, _ = p.layer(ap["x"], ap["logits"], None, *wargs)
+                p_outs.append(out)
+                assert ts.task_done(e) == B.MOE_OK
+        except Exception as exc:  # noqa: BLE001
+            errors.append(repr(exc))
+        finally:
+            p_done.set()
+
+    def d_thread():
+        try:
+            while True:
+                stop = p_done.is_set()
+                st, active = ts.d_enter(20000)
+                assert st == B.MOE_OK
+                out, _ = d.layer(ad["x"], ad["logits"], None, *wargs)   # D2 (PreD/PostD rendezvous: one rank)
+                ev = torch.cuda.Event()
+                ev.record(sd)
+                sp.wait_event(ev)       # the P segment admitted next runs after this D step on the device
+                d_outs.append(out)
+                ts.d_release()          # D4
+                if stop:
+                    return
+        except Exception as exc:  # noqa: BLE001
+            errors.append(repr(exc))
+
+    tp, td = threading.Thread(target=p_thread), threading.Thread(target=d_thread)
+    tp.start(); td.start()
+    tp.join(120); td.join(120)
+    torch.cuda.synchronize()
+    assert not tp.is_alive() and not td.is_alive() and not errors, errors
+    assert len(p_outs) == n_epochs and len(d_outs) >= n_epochs * 5   # 10 boundaries per epoch, span 2
+    assert all(torch.equal(o, p_alone) for o in p_outs)
+    assert all(torch.equal(o, d_alone) for o in d_outs)
+    assert p.moe_ctx_status() == B.MOE_OK and d.moe_ctx_status() == B.MOE_OK
+    p.moe_ctx_set_segments(0)
+    assert ts.destroy() == B.MOE_OK
+    p.close(); d.close()

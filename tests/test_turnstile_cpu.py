@@ -1,0 +1,174 @@
+"""The segment turnstile's host-side controller, without a GPU: validation rules, the P1/P2 - D1..D4 protocol
+under injected skew (P thread and D thread), and two gloo ranks whose D iterations see matching epoch and
+boundary identifiers."""
+import os
+import random
+import socket
+import sys
+import threading
+import time
+
+import pytest
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+from paper_2609_00993_b200 import binding as B  # noqa: E402
+
+OK, STATE, TIMEOUT = B.MOE_OK, B.MOE_ERR_STATE, B.MOE_ERR_TIMEOUT
+
+
+def test_controller_rejects_protocol_violations():
+    ts = B.Turnstile(span=2)
+    assert ts.publish(0, 0, 10) == STATE               # missing producer: no epoch was begun
+    assert ts.task_done(0) == STATE
+    assert ts.begin_epoch(5) == OK
+    assert ts.state() == {"epoch": 5, "reached": -1, "permit": 0, "span": 2, "active": True}
+    assert ts.begin_epoch(6) == STATE                  # the running epoch has not reported TaskDone
+    assert ts.publish(4, 0, 10) == STATE               # stale epoch
+    assert ts.publish(5, 1, 10) == STATE               # endpoint beyond the current permit (p = 0)
+    assert ts.publish(5, 0, 10) == TIMEOUT             # P stops at i = p until a D iteration moves the endpoint
+    assert ts.state()["reached"] == 0
+    assert ts.publish(5, 0, 10) == STATE               # non-monotone publication
+    st, active = ts.d_enter(10)                        # target 0 needs no publication
+    assert st == OK and active
+    assert ts.d_release() == OK and ts.state()["permit"] == 2
+    assert ts.publish(5, 1, 10) == OK                  # 1 < p: P runs on
+    assert ts.publish(5, 2, 10) == TIMEOUT             # stops at the new endpoint
+    assert ts.publish(5, 3, 10) == STATE               # beyond the permit
+    assert ts.destroy() == STATE                       # an epoch is still active
+    assert ts.task_done(5) == OK and ts.task_done(5) == STATE
+    assert ts.begin_epoch(5) == STATE and ts.begin_epoch(3) == STATE  # duplicate and stale epochs
+    assert ts.begin_epoch(6, d_already_enqueued=True) == OK and ts.state()["permit"] == 2
+    assert ts.task_done(6) == OK
+    st, active = ts.d_enter(10)                        # no P epoch running: D proceeds on the no-work path
+    assert st == OK and not active
+    assert ts.d_release() == OK
+    assert ts.destroy() == OK
+
+
+def test_d_waits_until_p_stands_at_the_endpoint():
+    ts = B.Turnstile(span=1)
+    assert ts.begin_epoch(0, d_already_enqueued=True) == OK  # p = 1
+    st, _ = ts.d_enter(20)
+    assert st == TIMEOUT                                # r = -1 < p
+    t = threading.Thread(target=lambda: (ts.publish(0, 0, 2000), ts.publish(0, 1, 2000)))
+    t.start()
+    st, active = ts.d_enter(2000)
+    assert st == OK and active and ts.state()["reached"] == 1
+    ts.d_release()
+    t.join()
+    assert ts.task_done(0) == OK and ts.destroy() == OK
+
+
+def _run_protocol(seed, n_epochs, n_segments, span, max_skew_ms, log, rendezvous=None):
+    """One rank: a P thread walks n_epochs epochs of n_segments segments; a D thread runs turnstile steps until
+    every epoch is done.  `log` receives ('P', epoch, segment) and ('D', epoch, reached, permit, active)."""
+    rng = random.Random(seed)
+    ts = B.Turnstile(span)
+    errors = []
+    p_finished = threading.Event()
+
+    def p_thread():
+        r = random.Random(seed * 7 + 1)
+        for e in range(n_epochs):
+            if ts.begin_epoch(e) != OK:
+                errors.append(("begin", e)); return
+            if ts.publish(e, 0, 20000) != OK:            # P1: wait before entering CUDA when p = 0
+                errors.append(("publish", e, 0)); return
+            for i in range(n_segments):
+                time.sleep(r.random() * max_skew_ms * 1e-3)
+                log.append(("P", e, i, ts.state()["permit"]))  # "enqueue" segment i under the permit seen now
+                if i + 1 < n_segments and ts.publish(e, i + 1, 20000) != OK:
+                    errors.append(("publish", e, i + 1)); return
+            if ts.task_done(e) != OK:
+                errors.append(("done", e)); return
+        p_finished.set()
+
+    def d_thread():
+        while True:
+            time.sleep(rng.random() * max_skew_ms * 1e-3)
+            st, active = ts.d_enter(20000)
+            if st != OK:
+                errors.append(("d_enter", st)); return
+            if rendezvous:
+                stop = rendezvous(p_finished.is_set())     # PreDRendezvous (also agrees on when to stop)
+            else:
+                stop = p_finished.is_set()
+            s = ts.state()
+            log.append(("D", s["epoch"], s["reached"], s["permit"], s["active"]))
+            if rendezvous:
+                rendezvous(False)                          # PostDRendezvous
+            log.append(("R",))                             # logged BEFORE the release: what it admits comes after
+            ts.d_release()
+            if stop:
+                return
+
+    tp, td = threading.Thread(target=p_thread), threading.Thread(target=d_thread)
+    tp.start(); td.start()
+    tp.join(60); td.join(60)
+    assert not tp.is_alive() and not td.is_alive(), "protocol did not make progress"
+    assert not errors, errors
+    assert ts.destroy() == OK
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3, 4])
+@pytest.mark.parametrize("span", [1, 3])
+def test_turnstile_under_skew(seed, span):
+    """Model-free stress: P never passes its permit, D enters only with P at the endpoint, and at most `span`
+    P segments go out between two D iterations."""
+    log = []
+    n_epochs, n_segments = 8, 16
+    _run_protocol(seed, n_epochs, n_segments, span, max_skew_ms=1.0, log=log)
+    assert sum(1 for x in log if x[0] == "P") == n_epochs * n_segments
+    since_release = 0
+    for ev in log:
+        if ev[0] == "D":
+            _, e, reached, permit, active = ev
+            if active:
+                assert permit == 0 or reached >= permit, ev      # D1: P stands at the endpoint (or has not entered CUDA)
+        elif ev[0] == "R":
+            since_release = 0
+        else:
+            _, e, i, permit_seen = ev
+            assert i < permit_seen, ev                            # P2: segment i needs a permit p > i
+            since_release += 1
+            assert since_release <= span, ev                      # R- < G < R+: at most one span between D iterations
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _rank_main(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import torch
+
+    def rendezvous(local_done):
+        # a CPU all-rank rendezvous; it also carries "every rank's P has finished" so that all ranks stop together
+        t = torch.tensor([1 if local_done else 0])
+        dist.all_reduce(t, op=dist.ReduceOp.MIN)
+        return bool(t.item())
+
+    log = []
+    _run_protocol(seed=100 + rank, n_epochs=1, n_segments=24, span=2, max_skew_ms=2.0, log=log, rendezvous=rendezvous)
+    out[rank] = [ev[1:4] for ev in log if ev[0] == "D" and ev[4]]  # D iterations that overlapped the active P epoch
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_see_matching_epoch_and_boundary_identifiers():
+    world, port = 2, _free_port()
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_rank_main, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    n = min(len(res[0]), len(res[1]))
+    assert n >= 10
+    # every D iteration that ran against the active epoch saw P at the same endpoint on both ranks
+    assert res[0][:n] == res[1][:n], "ranks disagree on the (epoch, reached, permit) of their D iterations"
+    assert all(reached == permit or permit == 0 for _, reached, permit in res[0][:n])
