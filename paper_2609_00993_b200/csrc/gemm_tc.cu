@@ -22,6 +22,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "kernels.h"
 
 namespace moe {
@@ -40,7 +42,7 @@ constexpr int kGatherThreads = 128;
 constexpr int kThreadsGather = kThreads + kGatherThreads;
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 227 * 1024;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait
 constexpr int kEpiStagingBytes = kEpilogueWarps * 32 * 128;  // per-warp 32 x 128-byte staging tiles
 
 struct TcParams {
@@ -55,6 +57,7 @@ struct TcParams {
   int32_t n_stages;
   int32_t x_tile_bytes;    // row_tile * 128
   int* status;
+  int32_t inject_producer_stall;  // failure-detection test hook: the TMA producer issues nothing
   // row-gather variant: row p of the grouped operand is gather_src[perm[p] / top_k, :] (gather_src2[p, :] for
   // the dense group); no permuted copy of the rows exists
   const __nv_bfloat16* gather_src;
@@ -91,16 +94,27 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
-// Bounded wait.  Returns false if the limit ran out or another role of this CTA already gave up.
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after kWaitLimitNs of wall time (read from the global timer every 256 polls) or as soon
+// as another role of this CTA has given up.  Returns false in both cases.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+  unsigned long long t0 = 0;
+  for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (i >= 256u) {
-      if ((i & 255u) == 0u && *abort_flag) return false;
+      if ((i & 255u) == 0u) {
+        if (*abort_flag) return false;
+        const unsigned long long now = global_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > kWaitLimitNs) return false;
+      }
       __nanosleep(64);
     }
   }
-  return false;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
@@ -318,7 +332,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 
   if (warp == kProducerWarp) {
     // ================================================================= TMA producer (one lane)
-    if (lane == 0) {
+    if (lane == 0 && !p.inject_producer_stall) {
       uint32_t it = 0;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
@@ -555,6 +569,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
+// Failure-detection test hook, read once at library load: with MOE_PD_INJECT_PRODUCER_STALL=1 in the environment the
+// producer warp of the grouped GEMM issues no copies, so every consumer wait runs into its time limit; the kernel
+// must then report MOE_ERR_TIMEOUT through the status word and return with its TMEM freed.
+const bool g_inject_producer_stall = [] {
+  const char* v = getenv("MOE_PD_INJECT_PRODUCER_STALL");
+  return v != nullptr && v[0] == '1';
+}();
 const char* g_init_error = nullptr;
 
 bool encode_map(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
@@ -666,6 +687,7 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
   prm.row_tile = row_tile;
   prm.x_tile_bytes = row_tile * kBlockK * 2;
   prm.status = status;
+  prm.inject_producer_stall = g_inject_producer_stall ? 1 : 0;
   const int stage_bytes = 2 * kWBoxBytes + prm.x_tile_bytes;
   const size_t tail = (swap_ab ? 0 : kEpiStagingBytes) + (2 * kMaxStages + 4) * sizeof(uint64_t) +
                       2 * sizeof(uint32_t) + 2 * (size_t)(prm.E + 1) * sizeof(int);
