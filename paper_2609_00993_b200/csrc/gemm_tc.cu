@@ -143,14 +143,18 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 
-// D[tmem] (+)= A[smem] * B[smem]^T, both operands K-major bf16, fp32 accumulate.
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                          uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem]^T, both operands K-major bf16, fp32 accumulate.  The two shared-memory
+// descriptors are given as a 32-bit low word each (the part that changes from MMA to MMA) and one common high
+// word, so that the issuing thread's scalar work per MMA stays at a handful of instructions.
+__device__ __forceinline__ void umma_bf16_lo(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                             uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // The mbarrier gets one arrival when every MMA issued so far by this thread has completed.
@@ -208,6 +212,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&h);
 }
+
+// Position in the ring of pipeline stages, advanced without division: the role loops run on a single thread (or
+// a few), where every dependent scalar instruction's latency is exposed, so `it % stages` and `it / stages` per
+// k-block would cost more than the tensor core needs for the k-block's MMAs.
+struct RingCursor {
+  uint32_t stage = 0, phase = 0;
+  __device__ __forceinline__ void advance(uint32_t n_stages) {
+    if (++stage == n_stages) {
+      stage = 0;
+      phase ^= 1u;
+    }
+  }
+};
 
 struct Tile {
   int e, row0, rows, ft;
@@ -333,7 +350,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   if (warp == kProducerWarp) {
     // ================================================================= TMA producer (one lane)
     if (lane == 0 && !p.inject_producer_stall) {
-      uint32_t it = 0;
+      RingCursor ring;
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
         const Tile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, seg, tile_rows);
@@ -343,15 +360,15 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         const CUtensorMap* mx = t.dense ? &map_x2 : &map_x;
         const int w_e = t.dense ? 0 : p.e_base + t.e;
         const int num_kb = t.dense ? num_kb2 : num_kb1;
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
-          const uint32_t s = it % (uint32_t)p.n_stages, ph = (it / (uint32_t)p.n_stages) & 1u;
-          if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t full = bar_full + 8u * s;
-          const uint32_t st = base_addr + s * (uint32_t)stage_bytes;
+        for (int kb = 0, k0 = 0; kb < num_kb; ++kb, k0 += kBlockK) {
+          if (!mbar_wait(bar_empty + 8u * ring.stage, ring.phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t full = bar_full + 8u * ring.stage;
+          const uint32_t st = base_addr + ring.stage * (uint32_t)stage_bytes;
           mbar_expect_tx(full, GATHER ? 2u * kWBoxBytes : (uint32_t)stage_bytes);
-          tma_load_3d(st, mw, full, kb * kBlockK, w_row0, w_e);
-          tma_load_3d(st + kWBoxBytes, mw, full, kb * kBlockK, w_row1, w_e);
-          if (!GATHER) tma_load_2d(st + 2 * kWBoxBytes, mx, full, kb * kBlockK, t.row0);
+          tma_load_3d(st, mw, full, k0, w_row0, w_e);
+          tma_load_3d(st + kWBoxBytes, mw, full, k0, w_row1, w_e);
+          if (!GATHER) tma_load_2d(st + 2 * kWBoxBytes, mx, full, k0, t.row0);
+          ring.advance((uint32_t)p.n_stages);
         }
       }
       if (!ok) {
@@ -362,8 +379,13 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   } else if (warp == kMmaWarp) {
     // ================================================================= MMA issuer (one lane)
     if (lane == 0) {
-      uint32_t it = 0, tile_iter = 0;
+      uint32_t tile_iter = 0;
+      RingCursor ring;
       bool ok = true;
+      // descriptor words: only the 14-bit start-address field of the low word changes between MMAs
+      const uint32_t desc_hi = (uint32_t)(umma_smem_desc(0) >> 32);
+      const uint32_t lo_base = (uint32_t)umma_smem_desc(base_addr);  // stage 0, weight box 0
+      const uint32_t lo_stage = (uint32_t)stage_bytes >> 4, lo_box = (uint32_t)kWBoxBytes >> 4;
       for (int tile = unit; tile < total_tiles && ok; tile += n_units, ++tile_iter) {
         const Tile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, seg, tile_rows);
         const uint32_t as = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
@@ -374,27 +396,25 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         const uint32_t n_swap = (uint32_t)min(p.row_tile, (t.rows + 15) & ~15);
         const uint32_t idesc = SWAP ? umma_idesc(128, n_swap) : umma_idesc(128, 256);
         const int num_kb = t.dense ? num_kb2 : num_kb1;
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
-          const uint32_t s = it % (uint32_t)p.n_stages, ph = (it / (uint32_t)p.n_stages) & 1u;
-          if (!mbar_wait(bar_full + 8u * s, ph, abort_flag)) { ok = false; break; }
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(bar_full + 8u * ring.stage, ring.phase, abort_flag)) { ok = false; break; }
           if (GATHER) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // X rows came by cp.async
           tc_fence_after();
-          const uint32_t st = base_addr + s * (uint32_t)stage_bytes;
-          const uint64_t dw0 = umma_smem_desc(st);
-          const uint64_t dw1 = umma_smem_desc(st + kWBoxBytes);
-          const uint64_t dx = umma_smem_desc(st + 2 * kWBoxBytes);
+          const uint32_t lo_w0 = lo_base + ring.stage * lo_stage;  // weight box 0; box 1 and the X tile follow
 #pragma unroll
           for (int kk = 0; kk < kBlockK / kUmmaK; ++kk) {
-            const uint64_t adv = (uint64_t)((kk * kUmmaK * 2) >> 4);  // +32 bytes per K step, in 16-byte units
+            const uint32_t adv = (uint32_t)((kk * kUmmaK * 2) >> 4);  // +32 bytes per K step, in 16-byte units
             const uint32_t acc = (kb | kk) != 0 ? 1u : 0u;
             if (SWAP) {
-              umma_bf16(d0, dw0 + adv, dx + adv, idesc, acc);
-              umma_bf16(d0 + (uint32_t)p.row_tile, dw1 + adv, dx + adv, idesc, acc);
+              umma_bf16_lo(d0, lo_w0 + adv, lo_w0 + 2 * lo_box + adv, desc_hi, idesc, acc);
+              umma_bf16_lo(d0 + (uint32_t)p.row_tile, lo_w0 + lo_box + adv, lo_w0 + 2 * lo_box + adv, desc_hi, idesc, acc);
             } else {
-              umma_bf16(d0, dx + adv, dw0 + adv, idesc, acc);  // the two weight boxes are contiguous: N = 256
+              // the two weight boxes are contiguous: one N = 256 operand
+              umma_bf16_lo(d0, lo_w0 + 2 * lo_box + adv, lo_w0 + adv, desc_hi, idesc, acc);
             }
           }
-          umma_commit(bar_empty + 8u * s);  // the stage is free once these MMAs have read it
+          umma_commit(bar_empty + 8u * ring.stage);  // the stage is free once these MMAs have read it
+          ring.advance((uint32_t)p.n_stages);
         }
         if (ok) umma_commit(bar_tfull + 8u * as);  // accumulator complete
       }
@@ -409,7 +429,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     const int g = (int)threadIdx.x - kGatherWarp0 * 32;
     const int piece = g & 7, rbase = g >> 3;
     const uint32_t dst_off = (uint32_t)(rbase * 128 + ((piece ^ (rbase & 7)) << 4));  // 128-byte swizzle
-    uint32_t it = 0;
+    RingCursor ring;
     bool ok = true;
     // The source row of each of this thread's 8 rows (flat slot = perm[row]; source row = slot / top_k; the
     // dense group's rows are their own source) is fetched one tile ahead, so that the dependent perm load is
@@ -436,15 +456,15 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         row_ptr[i] = slot_next[i] < 0 ? nullptr : src + (size_t)(slot_next[i] / p.top_k) * Kt + piece * 8;
       fetch_slots(tile + n_units, slot_next);
       const int num_kb = t.dense ? num_kb2 : num_kb1;
-      for (int kb = 0; kb < num_kb; ++kb, ++it) {
-        const uint32_t s = it % (uint32_t)p.n_stages, ph = (it / (uint32_t)p.n_stages) & 1u;
-        if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_flag)) { ok = false; break; }
-        const uint32_t xs = base_addr + s * (uint32_t)stage_bytes + 2 * kWBoxBytes + dst_off;
+      for (int kb = 0, k0 = 0; kb < num_kb; ++kb, k0 += kBlockK) {
+        if (!mbar_wait(bar_empty + 8u * ring.stage, ring.phase ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t xs = base_addr + ring.stage * (uint32_t)stage_bytes + 2 * kWBoxBytes + dst_off;
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-          if (row_ptr[i] != nullptr) cp_async_16(xs + (uint32_t)(i * 16 * 128), row_ptr[i] + kb * kBlockK);
+          if (row_ptr[i] != nullptr) cp_async_16(xs + (uint32_t)(i * 16 * 128), row_ptr[i] + k0);
         // one arrival on the stage's barrier, delivered by the hardware when this thread's copies have landed
-        cp_async_arrive_on(bar_full + 8u * s);
+        cp_async_arrive_on(bar_full + 8u * ring.stage);
+        ring.advance((uint32_t)p.n_stages);
       }
     }
     if (!ok) {
