@@ -132,19 +132,21 @@ constexpr int kCombineConsumers = 128;   // one 16-byte vector (8 columns) per c
 constexpr int kCombineThreads = kCombineConsumers + 32;
 constexpr int kCombineMaxStages = 4;
 
+// acc += w * v for eight bf16 values; a bf16 widens to fp32 by a 16-bit shift (low half) or a mask (high half)
 __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4& v, float w) {
-  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+  const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    const float2 f = __bfloat1622float2(h[q]);
-    acc[2 * q] = fmaf(w, f.x, acc[2 * q]);
-    acc[2 * q + 1] = fmaf(w, f.y, acc[2 * q + 1]);
+    acc[2 * q] = fmaf(w, __uint_as_float(u[q] << 16), acc[2 * q]);
+    acc[2 * q + 1] = fmaf(w, __uint_as_float(u[q] & 0xffff0000u), acc[2 * q + 1]);
   }
 }
 
 // out[t, c0:c1] = sum_j w[t,j] * y_perm[inv_perm[t*k+j], c0:c1] (+ y_shared[t, c0:c1]); ascending j, then shared.
 // dynamic shared memory, per stage: (k+1) row chunks of chunk_bytes | k weights | valid mask; then barriers.
-// Producer lane j gathers row j; lane 0 also fetches the shared row.
+// Producer lane j gathers row j; lane 0 also fetches the shared row.  KT > 0 fixes k at compile time (the sum
+// over experts is then fully unrolled); KT = 0 takes k at run time.
+template <int KT>
 __global__ void __launch_bounds__(kCombineThreads)
 combine_kernel(const __nv_bfloat16* __restrict__ y_perm, const __nv_bfloat16* __restrict__ y_shared,
                const int32_t* __restrict__ inv_perm, const float* __restrict__ topk_w, __nv_bfloat16* __restrict__ out,
@@ -212,10 +214,17 @@ combine_kernel(const __nv_bfloat16* __restrict__ y_perm, const __nv_bfloat16* __
       const unsigned valid = *reinterpret_cast<const unsigned*>(st + meta_off + 4 * k);
       if (v * 8 < cols) {
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int j = 0; j < k; ++j)
-          if ((valid >> j) & 1u)
-            fma_bf16x8(acc, *reinterpret_cast<const uint4*>(st + (size_t)j * chunk_bytes + v * 16), wts[j]);
-        if (shared) fma_bf16x8(acc, *reinterpret_cast<const uint4*>(st + (size_t)k * chunk_bytes + v * 16), 1.0f);
+        const uint8_t* mine = st + v * 16;
+        if (KT > 0 && valid == (1u << KT) - 1u) {  // the usual case: every slot routed, k known at compile time
+#pragma unroll
+          for (int j = 0; j < KT; ++j)
+            fma_bf16x8(acc, *reinterpret_cast<const uint4*>(mine + (size_t)j * chunk_bytes), wts[j]);
+        } else {
+          for (int j = 0; j < k; ++j)
+            if ((valid >> j) & 1u)
+              fma_bf16x8(acc, *reinterpret_cast<const uint4*>(mine + (size_t)j * chunk_bytes), wts[j]);
+        }
+        if (shared) fma_bf16x8(acc, *reinterpret_cast<const uint4*>(mine + (size_t)k * chunk_bytes), 1.0f);
         uint4 o;
         __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
@@ -271,14 +280,20 @@ cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32
   if (stages > kCombineMaxStages) stages = kCombineMaxStages;
   if (stages < 2) stages = 2;
   const size_t smem = (size_t)stages * stage_bytes + 16 * stages;
-  cudaError_t err = ensure_dynamic_smem(combine_kernel, smem);
+  auto launch = [&](auto kern) -> cudaError_t {
+    cudaError_t e = ensure_dynamic_smem(kern, smem);
+    if (e != cudaSuccess) return e;
+    const long long n_items = (long long)T * col_blocks;
+    const long long cap = resident_ctas(reinterpret_cast<const void*>(kern), kCombineThreads, smem);
+    const int grid = (int)(n_items < cap ? n_items : cap);
+    kern<<<grid, kCombineThreads, smem, stream>>>(
+        static_cast<const __nv_bfloat16*>(y_perm), static_cast<const __nv_bfloat16*>(y_shared), inv_perm, topk_w,
+        static_cast<__nv_bfloat16*>(out), T, k, H, col_blocks, chunk_bytes, stage_bytes, stages, status);
+    return cudaSuccess;
+  };
+  cudaError_t err = k == 8 ? launch(combine_kernel<8>) : k == 4 ? launch(combine_kernel<4>)
+                  : k == 2 ? launch(combine_kernel<2>) : launch(combine_kernel<0>);
   if (err != cudaSuccess) return err;
-  const long long n_items = (long long)T * col_blocks;
-  const long long cap = resident_ctas(reinterpret_cast<const void*>(combine_kernel), kCombineThreads, smem);
-  const int grid = (int)(n_items < cap ? n_items : cap);
-  combine_kernel<<<grid, kCombineThreads, smem, stream>>>(
-      static_cast<const __nv_bfloat16*>(y_perm), static_cast<const __nv_bfloat16*>(y_shared), inv_perm, topk_w,
-      static_cast<__nv_bfloat16*>(out), T, k, H, col_blocks, chunk_bytes, stage_bytes, stages, status);
   err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
