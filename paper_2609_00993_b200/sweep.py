@@ -101,18 +101,22 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--tokens", type=int, nargs="*", default=list(wl.C5_TOKENS))
     ap.add_argument("--iters-min-ms", type=float, default=300.0, help="time each T for at least this long")
+    ap.add_argument("--experts", type=int, default=wl.C5.E,
+                    help="number of routed experts (fewer than 256 keeps the weights small enough for a profiler capture)")
     args = ap.parse_args()
     B.load_library()
     hbm, tfl, src = load_peaks()
-    weights = wl.make_weights(wl.C5, 2, "cuda")
+    import dataclasses
+    base = dataclasses.replace(wl.C5, E=args.experts)
+    weights = wl.make_weights(base, 2, "cuda")
     for T in args.tokens:
-        shape = wl.C5.with_tokens(T)
+        shape = base.with_tokens(T)
         step_us, n, stages, counts = run_one(shape, weights, args.iters_min_ms)
         floor_us, fl_us, by_us = layer_floor_us(shape, counts, hbm, tfl)
         cf = counts.double()
         nz = int((counts > 0).sum())
         print(json.dumps({
-            "workload": f"C5 zipf(1.2) T={T}", "phase": "decode" if T <= 256 else "prefill", "iters": n,
+            "workload": f"C5 zipf(1.2) E={shape.E} T={T}", "phase": "decode" if T <= 256 else "prefill", "iters": n,
             "step_us": round(step_us, 1), "tokens_per_s": round(T / (step_us * 1e-6), 1),
             "roofline_floor_us": round(floor_us, 1), "frac_of_roofline": round(floor_us / step_us, 3),
             "floor_tensor_only_us": round(fl_us, 1), "floor_bytes_only_us": round(by_us, 1),
