@@ -2,8 +2,9 @@
 //
 //   operands   bf16, K-major, staged in shared memory by TMA (128-byte swizzle), 64 K-elements per stage
 //   math       tcgen05.mma (kind::f16, M=128) issued by one thread, fp32 accumulators in TMEM
-//   epilogue   tcgen05.ld -> registers -> (SwiGLU) -> bf16 -> global, overlapped with the next tile's MMAs
-//              through two TMEM accumulator stages
+//   epilogue   tcgen05.ld -> registers -> (SwiGLU) -> bf16 -> a per-warp swizzled staging tile in shared
+//              memory -> full-line global stores; the accumulator stage is handed back as soon as it has
+//              been read, so the next tile's MMAs overlap the stores (two TMEM accumulator stages)
 //   schedule   persistent CTAs walk the tile list (expert, row tile, feature tile); the list is derived
 //              on the device from the expert offsets, so no host synchronisation is needed
 //
@@ -17,7 +18,9 @@
 // segments are NOT padded; rows that belong to the next expert are computed and simply not stored.
 //
 // Warp roles (192 threads): warps 0-3 epilogue (TMEM lanes 32w..32w+31), warp 4 TMA producer, warp 5 MMA
-// issuer and TMEM owner.  Every mbarrier wait is bounded: on expiry the kernel records a timeout in the
+// issuer and TMEM owner.  The optional row-gather instantiation adds warps 6-9, which fetch the routed
+// experts' token rows straight from the unpermuted activations with 16-byte asynchronous copies (the
+// permutation is applied on the fly, so the separate row-permute pass is skipped).  Every mbarrier wait is bounded: on expiry the kernel records a timeout in the
 // status word, raises a CTA-wide abort flag, lets copies in flight land, frees its TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>

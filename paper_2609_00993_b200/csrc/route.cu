@@ -1,8 +1,9 @@
 // Stage a1: top-k routing over given router logits.  One warp per token; each lane keeps
 // ceil(E/32) selection keys in registers (128-bit loads when E is a multiple of 128), and k rounds of
-// a shuffle arg-max on (key descending, expert index ascending) pick the experts.  The routed weights
-// are a max-subtracted softmax over the k selected unbiased logits.  The arg-max uses the integer warp
-// reductions (redux.sync) on an order-preserving integer image of the key.
+// a warp arg-max on (key descending, expert index ascending) pick the experts.  The arg-max is two integer
+// warp reductions (redux.sync): a max over an order-preserving integer image of the key, then a min over
+// the expert indices that hold it.  The routed weights are a max-subtracted softmax over the k selected
+// unbiased logits, summed in selection order.
 #include "kernels.h"
 
 namespace moe {

@@ -43,6 +43,7 @@ def _check(out, ref, label):
     (40, 128, 4, 4, 64, 64),     # k = E: every expert takes every token
     (300, 128, 1, 1, 192, 0),    # a single expert: the layer is a dense MLP
     (129, 192, 3, 2, 320, 64),   # one row past a tile boundary; H, I not powers of two
+    (200, 2560, 512, 8, 256, 0), # the paper's model shape: hidden 2,560, 512 routed experts, top-8 (I is not stated there)
 ])
 def test_small_and_degenerate_shapes(phase, pname, T, H, E, k, I, shared_I):
     shape = wl.LayerShape("t", T=T, H=H, E=E, k=k, I=I, shared_I=shared_I, select_bias=True)
