@@ -111,6 +111,14 @@ moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspa
  * host object.  Device memory is the caller's and is not freed. */
 moe_status moe_ctx_destroy(moe_ctx* ctx);
 
+/* Abandons the step in progress (after a failed call, or because the caller changed its plan) and returns the
+ * context to the state between steps; a no-op when no step is in progress.  Kernels already enqueued for the
+ * step still run.  Following the paper's lifetime rule that an abandoned operation retires its buffer until a
+ * quiescent point (Section "Network and Lifetime Isolation"), a DECODE context moves on to its other buffer
+ * set, so the abandoned step's buffers are written again only after one more whole step has been enqueued
+ * behind them on the stream.  Enqueues nothing and does not synchronise. */
+moe_status moe_ctx_abandon_step(moe_ctx* ctx);
+
 /* Synchronises the context's stream and returns the device status word (a moe_status:
  * MOE_OK, MOE_ERR_TIMEOUT or MOE_ERR_BAD_INDEX) in *device_status, then clears it. */
 moe_status moe_ctx_status(moe_ctx* ctx, int32_t* device_status);

@@ -28,7 +28,7 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_CAPACITY", 3:
 EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_destroy", "moe_ctx_status",
            "moe_last_error", "moe_route", "moe_dispatch_layout", "moe_grouped_ffn", "moe_combine", "moe_layer_host",
            "moe_ctx_debug_ptrs", "moe_ctx_launch_count", "moe_ctx_set_profiling", "moe_ctx_read_profile",
-           "moe_dispatch_layout_static", "moe_ctx_set_segments", "moe_turnstile_create", "moe_turnstile_destroy",
+           "moe_dispatch_layout_static", "moe_ctx_set_segments", "moe_ctx_abandon_step", "moe_turnstile_create", "moe_turnstile_destroy",
            "moe_turnstile_set_span", "moe_turnstile_begin_epoch", "moe_turnstile_publish", "moe_turnstile_task_done",
            "moe_turnstile_d_enter", "moe_turnstile_d_release", "moe_turnstile_state")
 
@@ -92,6 +92,8 @@ def load_library() -> ctypes.CDLL:
     lib.moe_layer_host.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp]
     lib.moe_ctx_debug_ptrs.restype = i32
     lib.moe_ctx_debug_ptrs.argtypes = [vp] + [ctypes.POINTER(vp)] * 6
+    lib.moe_ctx_abandon_step.restype = i32
+    lib.moe_ctx_abandon_step.argtypes = [vp]
     lib.moe_ctx_launch_count.restype = i64
     lib.moe_ctx_launch_count.argtypes = [vp]
     lib.moe_ctx_set_profiling.restype = i32
@@ -196,6 +198,9 @@ class MoeContext:
         v = ctypes.c_int32(0)
         self._check(self.lib.moe_ctx_status(self.handle, ctypes.byref(v)))
         return int(v.value)
+
+    def moe_ctx_abandon_step(self):
+        self._check(self.lib.moe_ctx_abandon_step(self.handle))
 
     def moe_ctx_launch_count(self) -> int:
         return int(self.lib.moe_ctx_launch_count(self.handle))

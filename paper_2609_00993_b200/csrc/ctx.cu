@@ -196,7 +196,11 @@ struct StageTimer {
     if (!c->profiling || capturing(c)) return;  // event timing is meaningless inside a capture
     if (c->spans_used == c->spans.size()) {
       moe_ctx::Span s;
-      if (cudaEventCreate(&s.beg) != cudaSuccess || cudaEventCreate(&s.end) != cudaSuccess) return;
+      if (cudaEventCreate(&s.beg) != cudaSuccess) return;
+      if (cudaEventCreate(&s.end) != cudaSuccess) {
+        cudaEventDestroy(s.beg);
+        return;
+      }
       c->spans.push_back(s);
     }
     span = &c->spans[c->spans_used++];
@@ -344,7 +348,10 @@ moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspa
   if (e != cudaSuccess) {
     std::lock_guard<std::mutex> lock(g_registry_mutex);
     for (size_t i = 0; i < g_registry.size(); ++i)
-      if (g_registry[i] == ctx) g_registry.erase(g_registry.begin() + i);
+      if (g_registry[i] == ctx) {
+        g_registry.erase(g_registry.begin() + i);
+        break;
+      }
     moe_status st = cuda_fail(nullptr, e, "context set-up");
     delete ctx;
     return st;
@@ -374,6 +381,15 @@ moe_status moe_ctx_destroy(moe_ctx* ctx) {
     cudaEventDestroy(sp.end);
   }
   delete ctx;
+  return MOE_OK;
+}
+
+moe_status moe_ctx_abandon_step(moe_ctx* ctx) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->state == ST_IDLE) return MOE_OK;
+  ctx->state = ST_IDLE;
+  ctx->T = 0;
+  if (ctx->n_sets == 2) ctx->cur ^= 1;  // D: the abandoned step's buffer set rests for one whole step
   return MOE_OK;
 }
 

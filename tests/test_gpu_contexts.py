@@ -5,6 +5,8 @@ import os
 import pytest
 import torch
 
+import oracle
+from helpers import check_layer, np_f32
 from paper_2609_00993_b200 import binding as B
 from paper_2609_00993_b200 import workloads as wl
 
@@ -87,6 +89,34 @@ def test_call_order_and_argument_errors():
     assert ctx.moe_ctx_status() == B.MOE_OK
     assert ctx.moe_ctx_launch_count() >= 5
     ctx.close()
+
+
+def test_an_abandoned_step_leaves_the_context_usable_and_rests_its_buffer_set():
+    """Lifetime rule of Section "Network and Lifetime Isolation": an abandoned operation retires its buffer."""
+    shape = wl.LayerShape("t", T=32, H=256, E=8, k=2, I=128)
+    w = wl.make_weights(shape, 1, DEV)
+    a, a2 = wl.make_activations(shape, 2, DEV), wl.make_activations(shape, 3, DEV)
+    torch.cuda.synchronize()
+    for phase in (B.MOE_PHASE_PREFILL, B.MOE_PHASE_DECODE):
+        ctx = B.MoeContext(_cfg(phase))
+        bufs = B.alloc_step_buffers(32, 2, 8, DEV)
+        ctx.moe_ctx_abandon_step()  # nothing in progress: a no-op
+        ctx.moe_route(a["logits"], None, bufs["topk_idx"], bufs["topk_w"])
+        ctx.moe_dispatch_layout(bufs["topk_idx"], a["x"])
+        abandoned = ctx.moe_ctx_debug_ptrs()["x_perm"].data_ptr()
+        with pytest.raises(B.MoeError):  # mid-step: a new step may not begin ...
+            ctx.moe_route(a2["logits"], None, bufs["topk_idx"], bufs["topk_w"])
+        ctx.moe_ctx_abandon_step()       # ... until the step is given up
+        out, _ = ctx.layer(a2["x"], a2["logits"], None, w["w_gate_up"], w["w_down"])
+        used = ctx.moe_ctx_debug_ptrs()["x_perm"].data_ptr()
+        torch.cuda.synchronize()
+        assert ctx.moe_ctx_status() == B.MOE_OK
+        if phase == B.MOE_PHASE_DECODE:
+            assert used != abandoned  # the next step worked in the other buffer set
+        ref = oracle.layer(wl.bits(a2["x"]), np_f32(a2["logits"]), None, 2, wl.bits(w["w_gate_up"]),
+                           wl.bits(w["w_down"]))
+        check_layer(out, ref["out"], label="after an abandoned step")
+        ctx.close()
 
 
 def test_create_rejects_bad_configurations():
