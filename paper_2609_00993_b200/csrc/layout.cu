@@ -4,7 +4,8 @@
 // atomic.  The flat slots are cut into warp-owned chunks; a warp walks its chunk 32 slots at a time
 // and ranks equal experts inside a step with __match_any_sync, which keeps ascending slot order.
 //   small N (decode, low latency): ONE CTA does count -> scan -> place in shared memory, one launch.
-//   large N (prefill):             count per chunk -> scan over chunks and experts -> place per chunk.
+//   large N (prefill):             count per chunk -> per-expert scan over chunks (one CTA per 32
+//                                  experts) -> scan over experts and place per chunk.
 #include <mutex>
 
 #include "kernels.h"
@@ -178,26 +179,26 @@ layout_count_kernel(const int32_t* __restrict__ topk_idx, int64_t n_slots, int E
   for (int e = lane; e < E; e += 32) chunk_counts[(size_t)chunk * E + e] = hist[e];
 }
 
-// (2) one CTA: per expert an exclusive prefix over chunks (in place), totals -> counts, then the
-//     exclusive scan over experts -> offsets.  The 1024 threads form `parts` x Epad: a thread owns one
-//     expert and one contiguous run of chunks, so the walk over chunks is `parts` times shorter, and its
-//     loads go out in batches of kBatch before the dependent stores.
-//     shared memory: partial[parts][Epad] | counts_sh[E] | offsets_sh[E+1] | warp_sums[33]
+// (2) per expert an exclusive prefix over chunks (in place) and the total -> counts.  One CTA per 32 experts;
+//     warp w owns the w-th of 32 contiguous runs of chunks, lane l the CTA's l-th expert, so a warp's loads are
+//     one 128-byte line per chunk and go out in batches of kBatch before anything depends on them.  A run of
+//     at most kBatch chunks (up to 65536 slots) is read once and kept in registers for the second walk.
 __global__ void __launch_bounds__(1024)
-layout_scan_kernel(int32_t* __restrict__ chunk_counts, int n_chunks, int E, int Epad, int parts,
-                   int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
-  extern __shared__ int sh[];
-  int* partial = sh;
-  int* counts_sh = partial + parts * Epad;
-  int* offsets_sh = counts_sh + E;
-  int* warp_sums = offsets_sh + (E + 1);
-  const int part = threadIdx.x / Epad, e = threadIdx.x % Epad;
-  const bool active = part < parts && e < E;
-  const int per = (n_chunks + parts - 1) / parts;
+layout_scan_kernel(int32_t* __restrict__ chunk_counts, int n_chunks, int E, int32_t* __restrict__ counts) {
+  __shared__ int partial[32][33];
+  const int lane = threadIdx.x & 31, part = threadIdx.x >> 5;
+  const int e = blockIdx.x * 32 + lane;
+  const bool active = e < E;
+  const int per = (n_chunks + 31) / 32;
   const int c0 = min(part * per, n_chunks), c1 = min(c0 + per, n_chunks);
+  int first[kBatch];  // the run's first batch
+#pragma unroll
+  for (int u = 0; u < kBatch; ++u) first[u] = (active && c0 + u < c1) ? chunk_counts[(size_t)(c0 + u) * E + e] : 0;
   int sum = 0;
+#pragma unroll
+  for (int u = 0; u < kBatch; ++u) sum += first[u];
   if (active) {
-    for (int cb = c0; cb < c1; cb += kBatch) {
+    for (int cb = c0 + kBatch; cb < c1; cb += kBatch) {
       int v[kBatch];
 #pragma unroll
       for (int u = 0; u < kBatch; ++u) v[u] = (cb + u < c1) ? chunk_counts[(size_t)(cb + u) * E + e] : 0;
@@ -205,41 +206,48 @@ layout_scan_kernel(int32_t* __restrict__ chunk_counts, int n_chunks, int E, int 
       for (int u = 0; u < kBatch; ++u) sum += v[u];
     }
   }
-  if (part < parts) partial[part * Epad + e] = sum;
+  partial[part][lane] = sum;
   __syncthreads();
-  if (active) {
-    int run = 0;
-    for (int q = 0; q < part; ++q) run += partial[q * Epad + e];
-    if (part == parts - 1) {
-      counts_sh[e] = run + sum;
-      counts[e] = run + sum;
-    }
-    for (int cb = c0; cb < c1; cb += kBatch) {
-      int v[kBatch];
+  if (!active) return;
+  int run = 0;
+  for (int q = 0; q < part; ++q) run += partial[q][lane];
+  if (part == 31) counts[e] = run + sum;
 #pragma unroll
-      for (int u = 0; u < kBatch; ++u) v[u] = (cb + u < c1) ? chunk_counts[(size_t)(cb + u) * E + e] : 0;
+  for (int u = 0; u < kBatch; ++u) {
+    if (c0 + u < c1) chunk_counts[(size_t)(c0 + u) * E + e] = run;
+    run += first[u];
+  }
+  for (int cb = c0 + kBatch; cb < c1; cb += kBatch) {
+    int v[kBatch];
 #pragma unroll
-      for (int u = 0; u < kBatch; ++u) {
-        if (cb + u < c1) chunk_counts[(size_t)(cb + u) * E + e] = run;
-        run += v[u];
-      }
+    for (int u = 0; u < kBatch; ++u) v[u] = (cb + u < c1) ? chunk_counts[(size_t)(cb + u) * E + e] : 0;
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      if (cb + u < c1) chunk_counts[(size_t)(cb + u) * E + e] = run;
+      run += v[u];
     }
   }
-  __syncthreads();
-  block_exclusive_scan(counts_sh, E, offsets, offsets_sh, warp_sums);
 }
 
-// (3) place each chunk at offsets[e] + (prefix of earlier chunks)[e]
+// (3) every CTA scans the counts over experts itself (CTA 0 also stores the result -> offsets) and places its
+//     chunks at offsets[e] + (prefix of earlier chunks)[e]
+//     shared memory: run[warps][E] | counts_sh[E] | offsets_sh[E+1] | warp_sums[33]
 __global__ void __launch_bounds__(kChunkWarpsPerBlock * 32)
 layout_place_kernel(const int32_t* __restrict__ topk_idx, int64_t n_slots, int E, int n_chunks,
-                    const int32_t* __restrict__ chunk_prefix, const int32_t* __restrict__ offsets,
-                    int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
+                    const int32_t* __restrict__ chunk_prefix, const int32_t* __restrict__ counts,
+                    int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
   extern __shared__ int sh[];
+  int* counts_sh = sh + kChunkWarpsPerBlock * E;
+  int* offsets_sh = counts_sh + E;
+  int* warp_sums = offsets_sh + (E + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int e = threadIdx.x; e < E; e += blockDim.x) counts_sh[e] = counts[e];
+  __syncthreads();
+  block_exclusive_scan(counts_sh, E, blockIdx.x == 0 ? offsets : nullptr, offsets_sh, warp_sums);
   const int chunk = blockIdx.x * kChunkWarpsPerBlock + warp;
   if (chunk >= n_chunks) return;
   int* run = sh + warp * E;
-  for (int e = lane; e < E; e += 32) run[e] = offsets[e] + chunk_prefix[(size_t)chunk * E + e];
+  for (int e = lane; e < E; e += 32) run[e] = offsets_sh[e] + chunk_prefix[(size_t)chunk * E + e];
   __syncwarp();
   const int64_t f0 = (int64_t)chunk * kLayoutChunk;
   const int64_t f1 = min(f0 + kLayoutChunk, n_slots);
@@ -282,15 +290,12 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
   layout_count_kernel<<<blocks, kChunkWarpsPerBlock * 32, chunk_smem, stream>>>(topk_idx, n_slots, E, n_chunks,
                                                                                 scratch, status);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
-  const int Epad = (E + 31) / 32 * 32;
-  int parts = 1024 / Epad;
-  if (parts > n_chunks) parts = n_chunks;
-  if (parts < 1) parts = 1;
-  const size_t scan_smem = ((size_t)parts * Epad + E + (E + 1) + 33) * sizeof(int);
-  layout_scan_kernel<<<1, 1024, scan_smem, stream>>>(scratch, n_chunks, E, Epad, parts, counts, offsets);
+  layout_scan_kernel<<<(E + 31) / 32, 1024, 0, stream>>>(scratch, n_chunks, E, counts);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
-  layout_place_kernel<<<blocks, kChunkWarpsPerBlock * 32, chunk_smem, stream>>>(topk_idx, n_slots, E, n_chunks,
-                                                                                scratch, offsets, perm, inv_perm);
+  const size_t place_smem = chunk_smem + ((size_t)E + (E + 1) + 33) * sizeof(int);
+  layout_place_kernel<<<blocks, kChunkWarpsPerBlock * 32, place_smem, stream>>>(topk_idx, n_slots, E, n_chunks,
+                                                                                scratch, counts, offsets, perm,
+                                                                                inv_perm);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;
   if (n_launches) *n_launches += 3;
   return cudaSuccess;
