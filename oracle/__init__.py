@@ -216,3 +216,91 @@ def layer(x_bits, logits, bias, k, w_gate_up_bits, w_down_bits, ws_gate_up_bits=
     out = combine(y, inv, w, y_sh)
     return dict(topk_idx=idx, topk_w=w, counts=counts, offsets=offsets, perm=perm, inv_perm=inv, x_perm=x_perm,
                 act=act, y=y, y_shared=y_sh, out=out)
+
+
+# ----------------------------------------------------------------------------- FP8 precision variant
+def e4m3_decode(codes):
+    """E4M3 codes (uint8) -> fp32 values."""
+    codes = _c(codes, np.uint8)
+    out = np.empty(codes.shape, np.float32)
+    _load().oracle_e4m3_decode(_p(codes), ctypes.c_int64(codes.size), _p(out))
+    return out
+
+
+def e4m3_encode(vals):
+    """fp32 values -> E4M3 codes (round to nearest even, saturating at +-448)."""
+    vals = _c(vals, np.float32)
+    out = np.empty(vals.shape, np.uint8)
+    _load().oracle_e4m3_encode(_p(vals), ctypes.c_int64(vals.size), _p(out))
+    return out
+
+
+def quantize_rows(x_bits):
+    """Per-row dynamic quantisation of bf16 rows [M,n]: (codes [M,n] uint8, scale [M] fp32)."""
+    x_bits = _c(x_bits, np.uint16)
+    M, n = x_bits.shape
+    q = np.empty((M, n), np.uint8)
+    s = np.empty(M, np.float32)
+    _chk(_load().oracle_quantize_rows(_p(x_bits), ctypes.c_int64(M), ctypes.c_int32(n), _p(q), _p(s)))
+    return q, s
+
+
+def gemm1_fp8(xq, sx, wq_gate_up, sw_gate_up):
+    """GEMM1 + SwiGLU of the FP8 variant for one expert: act [M,I] bf16 bits."""
+    xq, sx = _c(xq, np.uint8), _c(sx, np.float32)
+    wq_gate_up, sw_gate_up = _c(wq_gate_up, np.uint8), _c(sw_gate_up, np.float32)
+    M, H = xq.shape
+    I = wq_gate_up.shape[0] // 2
+    assert wq_gate_up.shape == (2 * I, H) and sw_gate_up.shape == (2 * I,) and sx.shape == (M,)
+    act = np.empty((M, I), np.uint16)
+    _chk(_load().oracle_gemm1_fp8(_p(xq), _p(sx), ctypes.c_int64(M), _p(wq_gate_up), _p(sw_gate_up),
+                                  ctypes.c_int32(H), ctypes.c_int32(I), _p(act)))
+    return act
+
+
+def gemm2_fp8(aq, sa, wq_down, sw_down):
+    """GEMM2 of the FP8 variant for one expert: y [M,H] fp32."""
+    aq, sa = _c(aq, np.uint8), _c(sa, np.float32)
+    wq_down, sw_down = _c(wq_down, np.uint8), _c(sw_down, np.float32)
+    M, I = aq.shape
+    H = wq_down.shape[0]
+    assert wq_down.shape == (H, I) and sw_down.shape == (H,) and sa.shape == (M,)
+    y = np.empty((M, H), np.float32)
+    _chk(_load().oracle_gemm2_fp8(_p(aq), _p(sa), ctypes.c_int64(M), _p(wq_down), _p(sw_down), ctypes.c_int32(H),
+                                  ctypes.c_int32(I), _p(y)))
+    return y
+
+
+def ffn_fp8(x_rows_bits, wq_gate_up, sw_gate_up, wq_down, sw_down, want_stages=False):
+    """One expert of the FP8 variant on bf16 rows: quantise -> GEMM1 + SwiGLU -> quantise -> GEMM2.
+    Returns y [M,H] fp32 (and a dict of the intermediate stages)."""
+    xq, sx = quantize_rows(x_rows_bits)
+    act = gemm1_fp8(xq, sx, wq_gate_up, sw_gate_up)
+    aq, sa = quantize_rows(act)
+    y = gemm2_fp8(aq, sa, wq_down, sw_down)
+    return (y, dict(xq=xq, sx=sx, act=act, aq=aq, sa=sa)) if want_stages else y
+
+
+def layer_fp8(x_bits, logits, bias, k, wq_gate_up, sw_gate_up, wq_down, sw_down, wsq_gate_up=None, sws_gate_up=None,
+              wsq_down=None, sws_down=None, routed_scale=1.0):
+    """Whole layer of the FP8 variant through the explicit stages; routing, layout, row movement and combine are
+    the bf16 layer's.  Returns a dict of every stage's result."""
+    E = wq_down.shape[0]
+    H = x_bits.shape[1]
+    idx, w = route(logits, bias, k, routed_scale)
+    counts, offsets, perm, inv = layout(idx, E)
+    x_perm = permute(x_bits, perm, k)
+    y = np.zeros((x_perm.shape[0], H), np.float32)
+    act = np.zeros((x_perm.shape[0], wq_down.shape[2]), np.uint16)
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        if r1 > r0:
+            y[r0:r1], st = ffn_fp8(x_perm[r0:r1], wq_gate_up[e], sw_gate_up[e], wq_down[e], sw_down[e],
+                                   want_stages=True)
+            act[r0:r1] = st["act"]
+    y_sh = None
+    if wsq_gate_up is not None:
+        y_sh = ffn_fp8(x_bits, wsq_gate_up, sws_gate_up, wsq_down, sws_down)
+    out = combine(y, inv, w, y_sh)
+    return dict(topk_idx=idx, topk_w=w, counts=counts, offsets=offsets, perm=perm, inv_perm=inv, x_perm=x_perm,
+                act=act, y=y, y_shared=y_sh, out=out)

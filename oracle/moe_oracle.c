@@ -340,3 +340,123 @@ int oracle_layer_tokens(const uint16_t* x, const int32_t* topk_idx, const float*
   free(mag);
   return rc;
 }
+
+/* ===================================================================== FP8
+ * Precision variant: 8-bit weights and activations (the paper evaluates its
+ * models in BF16 and in FP8, Section "Evaluation", "Methodology", but prints no
+ * recipe).  The reading taken here, step by step:
+ *
+ *   format     OCP E4M3 ("e4m3fn"): 1 sign, 4 exponent (bias 7), 3 mantissa
+ *              bits; no infinities; largest finite value 448; subnormals are
+ *              multiples of 2^-9.
+ *   weights    given as E4M3 codes with one fp32 scale per output channel
+ *              (per weight row): W[r,:] = scale_w[r] * decode(code[r,:]).
+ *   activation a bf16 row v[0..n) entering a GEMM is quantised per row:
+ *                amax  = max_i |v_i|                         (fp32)
+ *                scale = amax / 448   (one fp32 division; 1 if amax == 0)
+ *                code_i = e4m3( v_i / scale )  (fp32 division, then round to
+ *                         nearest even, saturating at +-448)
+ *   GEMM1      g_i = (sum_h dq_x[h] * dq_wg[i,h]) * scale_x * scale_w[i],
+ *              u_i likewise with the up row, a_i = silu(g_i) * u_i,
+ *              a stored as bf16 (round to nearest even)
+ *   GEMM2      the bf16 row a is quantised as above, then
+ *              y_c = (sum_i dq_a[i] * dq_wd[c,i]) * scale_a * scale_w[c]
+ *
+ * The quantisation decides integers (codes), so it is written in fp32 with
+ * exactly the operations listed; the sums accumulate in fp64.
+ */
+static inline float e4m3_to_f32(uint8_t c) {
+  int sign = c >> 7, ex = (c >> 3) & 15, man = c & 7;
+  float v;
+  if (ex == 15 && man == 7) return NAN;
+  if (ex == 0) v = ldexpf((float)man, -9);
+  else v = ldexpf(1.0f + (float)man / 8.0f, ex - 7);
+  return sign ? -v : v;
+}
+
+static inline uint8_t f32_to_e4m3(float f) {
+  if (f != f) return 0x7f;
+  uint8_t sign = (uint8_t)(signbit(f) ? 0x80 : 0);
+  float a = fabsf(f);
+  if (a >= 448.0f) return (uint8_t)(sign | 0x7e); /* saturate (also everything that would round past 448) */
+  if (a < ldexpf(1.0f, -6)) {                     /* subnormal range: multiples of 2^-9; 8 is the first normal */
+    int q = (int)rintf(ldexpf(a, 9));
+    return (uint8_t)(sign | q);
+  }
+  int e;
+  (void)frexpf(a, &e);
+  e -= 1; /* a = m * 2^e, m in [1,2) */
+  int man = (int)rintf(ldexpf(a, 3 - e)) - 8; /* round m*8 to nearest even; exact scaling */
+  if (man == 8) {
+    man = 0;
+    e += 1;
+  }
+  if (e > 8 || (e == 8 && man > 6)) return (uint8_t)(sign | 0x7e);
+  return (uint8_t)(sign | ((e + 7) << 3) | man);
+}
+
+void oracle_e4m3_decode(const uint8_t* in, int64_t n, float* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = e4m3_to_f32(in[i]);
+}
+void oracle_e4m3_encode(const float* in, int64_t n, uint8_t* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = f32_to_e4m3(in[i]);
+}
+
+/* Per-row dynamic quantisation of bf16 rows: x [M,n] bf16 -> q [M,n] codes, scale [M] fp32. */
+int oracle_quantize_rows(const uint16_t* x, int64_t M, int32_t n, uint8_t* q, float* scale) {
+  if (M < 0 || n <= 0) return ORACLE_ERR_ARG;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < M; ++r) {
+    float amax = 0.0f;
+    for (int32_t i = 0; i < n; ++i) {
+      float a = fabsf(bf16_to_f32(x[r * n + i]));
+      if (a > amax) amax = a;
+    }
+    float s = amax > 0.0f ? amax / 448.0f : 1.0f;
+    scale[r] = s;
+    for (int32_t i = 0; i < n; ++i) q[r * n + i] = f32_to_e4m3(bf16_to_f32(x[r * n + i]) / s);
+  }
+  return ORACLE_OK;
+}
+
+/* GEMM1 + SwiGLU of the FP8 variant for one expert: xq [M,H] codes, sx [M]; wq [2I,H] codes (rows 0..I-1 gate,
+ * I..2I-1 up), sw [2I]; act_out [M,I] bf16 bits. */
+int oracle_gemm1_fp8(const uint8_t* xq, const float* sx, int64_t M, const uint8_t* wq, const float* sw,
+                     int32_t H, int32_t I, uint16_t* act_out) {
+  if (M < 0 || H <= 0 || I <= 0) return ORACLE_ERR_ARG;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int64_t r = 0; r < M; ++r) {
+    for (int32_t i = 0; i < I; ++i) {
+      const uint8_t* xr = xq + r * H;
+      const uint8_t* wg = wq + (int64_t)i * H;
+      const uint8_t* wu = wq + ((int64_t)I + i) * H;
+      double g = 0.0, u = 0.0;
+      for (int32_t h = 0; h < H; ++h) {
+        double xv = (double)e4m3_to_f32(xr[h]);
+        g += xv * (double)e4m3_to_f32(wg[h]);
+        u += xv * (double)e4m3_to_f32(wu[h]);
+      }
+      g *= (double)sx[r] * (double)sw[i];
+      u *= (double)sx[r] * (double)sw[I + i];
+      act_out[r * I + i] = f32_to_bf16((float)(g / (1.0 + exp(-g)) * u));
+    }
+  }
+  return ORACLE_OK;
+}
+
+/* GEMM2 of the FP8 variant for one expert: aq [M,I] codes, sa [M]; wq [H,I] codes, sw [H]; y_out [M,H] fp32. */
+int oracle_gemm2_fp8(const uint8_t* aq, const float* sa, int64_t M, const uint8_t* wq, const float* sw,
+                     int32_t H, int32_t I, float* y_out) {
+  if (M < 0 || H <= 0 || I <= 0) return ORACLE_ERR_ARG;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int64_t r = 0; r < M; ++r) {
+    for (int32_t c = 0; c < H; ++c) {
+      const uint8_t* ar = aq + r * I;
+      const uint8_t* wd = wq + (int64_t)c * I;
+      double y = 0.0;
+      for (int32_t i = 0; i < I; ++i) y += (double)e4m3_to_f32(ar[i]) * (double)e4m3_to_f32(wd[i]);
+      y_out[r * H + c] = (float)(y * (double)sa[r] * (double)sw[c]);
+    }
+  }
+  return ORACLE_OK;
+}
