@@ -71,6 +71,11 @@ typedef enum {
   MOE_GEMM_VALIDATION = 3 /* plain CUDA-core kernel, slow; exists to localise tensor-core bugs   */
 } moe_gemm_variant;
 
+/* Precision of the expert weights a context will be given.  BF16 is the path the whole library is measured
+ * on; FP8_E4M3 enables moe_grouped_ffn_fp8 (the paper evaluates its models in BF16 and in FP8, Section
+ * "Evaluation", "Methodology"). */
+typedef enum { MOE_WEIGHTS_BF16 = 0, MOE_WEIGHTS_FP8_E4M3 = 1 } moe_weight_format;
+
 typedef struct {
   int32_t hidden;       /* H, multiple of 64                                            */
   int32_t n_experts;    /* E, 1..1024                                                   */
@@ -89,6 +94,7 @@ typedef struct {
                               through perm while it runs; x_perm is not written, and x must
                               be passed to moe_grouped_ffn.  Ignored by the other variants. */
   float routed_scale;   /* multiplies the routed weights; 1.0f unless the model says so */
+  int32_t weight_format; /* moe_weight_format; FP8 adds the quantisation buffers to the workspace */
 } moe_config;
 
 /* Bytes of device workspace `moe_ctx_create` needs for this configuration (0 on a bad config).
@@ -169,6 +175,27 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
  * that moe_dispatch_layout was given).  Weights are read-only and may be shared by contexts. */
 moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_down, const void* x,
                            const void* ws_gate_up, const void* ws_down, int32_t T);
+
+/* Stages a6-a8 with FP8 weights and activations (context created with weight_format = MOE_WEIGHTS_FP8_E4M3;
+ * same place in the step as moe_grouped_ffn).  The paper names FP8 runs but prints no recipe; this one is
+ * W8A8 with OCP E4M3 codes (1-4-3 bits, bias 7, largest finite value 448, no infinities):
+ *   weights      wq_* hold E4M3 codes, sw_* one fp32 scale per output channel (weight row):
+ *                W[e,r,:] = sw[e,r] * decode(wq[e,r,:])
+ *   activations  every bf16 row v entering a GEMM is quantised on the fly, per row:
+ *                scale = max|v| / 448 (1 for an all-zero row), code_i = e4m3(v_i / scale), both divisions in
+ *                IEEE fp32, conversion round-to-nearest-even saturating at +-448
+ *   GEMM1        g, u = (sum_h x_code * w_code) * scale_x[p] * sw[e,row], act = silu(g) * u stored as bf16
+ *   GEMM2        act is quantised per row as above; y = (sum_i a_code * w_code) * scale_a[p] * sw[e,c], bf16
+ * The sums run on the tensor cores (tcgen05 kind::f8f6f4) with fp32 accumulation.  The shared expert (S = 1)
+ * is computed the same way from x with its own codes and scales.
+ * wq_gate_up [E,2I,H] uint8, sw_gate_up [E,2I] fp32, wq_down [E,H,I] uint8, sw_down [E,H] fp32;
+ * wsq_gate_up [2I_s,H], sws_gate_up [2I_s], wsq_down [H,I_s], sws_down [H] (required iff S = 1);
+ * x [T,H] bf16 (required iff S = 1).  H, I and I_s may not exceed 8192.  The row gather and prefill
+ * segmentation do not apply to this call.  Errors as for moe_grouped_ffn; MOE_ERR_STATE if the context was
+ * created for BF16 weights. */
+moe_status moe_grouped_ffn_fp8(moe_ctx* ctx, const void* wq_gate_up, const float* sw_gate_up, const void* wq_down,
+                               const float* sw_down, const void* x, const void* wsq_gate_up,
+                               const float* sws_gate_up, const void* wsq_down, const float* sws_down, int32_t T);
 
 /* Prefill segmentation.  A single P execution spans several D iterations, so the paper divides P into
  * segments delimited by backend-provided boundaries (Section "In-Place P/D Execution"; the span K of Section
@@ -254,14 +281,18 @@ moe_status moe_layer_host(moe_ctx* ctx, const float* logits_host, const float* s
 moe_status moe_ctx_debug_ptrs(moe_ctx* ctx, void** x_perm, void** act, void** y_perm, void** y_shared,
                               int32_t** counts, int32_t** offsets);
 
+/* Test/inspection only, FP8 variant: the quantised GEMM1 input rows and activation rows of the same buffer set
+ * (codes [N,H] / [N,I] uint8, scales [N] fp32).  Any out-pointer may be NULL. */
+moe_status moe_ctx_debug_ptrs_fp8(moe_ctx* ctx, void** xq, float** sx, void** aq, float** sa);
+
 /* Per-stage device timing (measurement aid; off by default).  While enabled, every stage's launches are
  * bracketed by CUDA events on the context's stream.  moe_ctx_read_profile synchronises the stream, returns
  * the summed device time and the number of bracketed launches per stage since the last read, and resets.
  * Stage order: 0 route, 1 layout (counts+scan+permutation), 2 permute rows, 3 routed GEMM1+SwiGLU,
  * 4 routed GEMM2, 5 shared GEMM1+SwiGLU, 6 shared GEMM2, 7 combine.  Without prefill segmentation the shared
  * expert's passes ride in the routed launches, so their time is part of stages 3 and 4 and stages 5 and 6
- * stay empty. */
-#define MOE_N_STAGES 8
+ * stay empty.  FP8 variant only: 8 quantise the GEMM1 input rows, 9 quantise the activation rows. */
+#define MOE_N_STAGES 10
 typedef struct {
   double ms[MOE_N_STAGES];
   int64_t calls[MOE_N_STAGES];

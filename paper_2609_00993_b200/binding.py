@@ -20,32 +20,36 @@ MOE_OK = 0
 MOE_ERR_INVALID_ARG, MOE_ERR_CAPACITY, MOE_ERR_STATE, MOE_ERR_UNSUPPORTED = 1, 2, 3, 4
 MOE_ERR_CUDA, MOE_ERR_TIMEOUT, MOE_ERR_BAD_INDEX = 5, 6, 7
 MOE_GEMM_AUTO, MOE_GEMM_LARGE_M, MOE_GEMM_SMALL_M, MOE_GEMM_VALIDATION = 0, 1, 2, 3
+MOE_WEIGHTS_BF16, MOE_WEIGHTS_FP8_E4M3 = 0, 1
 
 STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_CAPACITY", 3: "MOE_ERR_STATE",
                 4: "MOE_ERR_UNSUPPORTED", 5: "MOE_ERR_CUDA", 6: "MOE_ERR_TIMEOUT", 7: "MOE_ERR_BAD_INDEX"}
 
 # every symbol include/moe_pd.h declares
 EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_destroy", "moe_ctx_status",
-           "moe_last_error", "moe_route", "moe_dispatch_layout", "moe_grouped_ffn", "moe_combine", "moe_layer_host",
-           "moe_ctx_debug_ptrs", "moe_ctx_launch_count", "moe_ctx_set_profiling", "moe_ctx_read_profile",
+           "moe_last_error", "moe_route", "moe_dispatch_layout", "moe_grouped_ffn", "moe_grouped_ffn_fp8", "moe_combine",
+           "moe_layer_host",
+           "moe_ctx_debug_ptrs", "moe_ctx_debug_ptrs_fp8", "moe_ctx_launch_count", "moe_ctx_set_profiling", "moe_ctx_read_profile",
            "moe_dispatch_layout_static", "moe_ctx_set_segments", "moe_ctx_abandon_step", "moe_turnstile_create", "moe_turnstile_destroy",
            "moe_turnstile_set_span", "moe_turnstile_begin_epoch", "moe_turnstile_publish", "moe_turnstile_task_done",
            "moe_turnstile_d_enter", "moe_turnstile_d_release", "moe_turnstile_state")
 
 BOUNDARY_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32)
 
-STAGE_NAMES = ("route", "layout", "permute", "gemm1_swiglu", "gemm2", "shared_gemm1_swiglu", "shared_gemm2", "combine")
+STAGE_NAMES = ("route", "layout", "permute", "gemm1_swiglu", "gemm2", "shared_gemm1_swiglu", "shared_gemm2", "combine",
+               "quantize_x", "quantize_act")
 
 
 class moe_config(ctypes.Structure):
     _fields_ = [("hidden", ctypes.c_int32), ("n_experts", ctypes.c_int32), ("top_k", ctypes.c_int32),
                 ("inter", ctypes.c_int32), ("n_shared", ctypes.c_int32), ("shared_inter", ctypes.c_int32),
                 ("max_tokens", ctypes.c_int32), ("phase", ctypes.c_int32), ("sm_budget", ctypes.c_int32),
-                ("gemm_variant", ctypes.c_int32), ("row_gather", ctypes.c_int32), ("routed_scale", ctypes.c_float)]
+                ("gemm_variant", ctypes.c_int32), ("row_gather", ctypes.c_int32), ("routed_scale", ctypes.c_float),
+                ("weight_format", ctypes.c_int32)]
 
 
 class moe_stage_times(ctypes.Structure):
-    _fields_ = [("ms", ctypes.c_double * 8), ("calls", ctypes.c_int64 * 8)]
+    _fields_ = [("ms", ctypes.c_double * 10), ("calls", ctypes.c_int64 * 10)]
 
 
 class MoeError(RuntimeError):
@@ -86,6 +90,10 @@ def load_library() -> ctypes.CDLL:
     lib.moe_dispatch_layout.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
     lib.moe_grouped_ffn.restype = i32
     lib.moe_grouped_ffn.argtypes = [vp, vp, vp, vp, vp, vp, i32]
+    lib.moe_ctx_debug_ptrs_fp8.restype = i32
+    lib.moe_ctx_debug_ptrs_fp8.argtypes = [vp] + [ctypes.POINTER(vp)] * 4
+    lib.moe_grouped_ffn_fp8.restype = i32
+    lib.moe_grouped_ffn_fp8.argtypes = [vp] * 10 + [i32]
     lib.moe_combine.restype = i32
     lib.moe_combine.argtypes = [vp, vp, vp, i32, vp]
     lib.moe_layer_host.restype = i32
@@ -137,9 +145,9 @@ def _dev(t: Optional[torch.Tensor], dtype, name):
 
 
 def make_config(hidden, n_experts, top_k, inter, shared_inter=0, max_tokens=1, phase=MOE_PHASE_PREFILL, sm_budget=0,
-                gemm_variant=MOE_GEMM_AUTO, routed_scale=1.0, row_gather=0) -> moe_config:
+                gemm_variant=MOE_GEMM_AUTO, routed_scale=1.0, row_gather=0, weight_format=MOE_WEIGHTS_BF16) -> moe_config:
     return moe_config(hidden, n_experts, top_k, inter, 1 if shared_inter else 0, shared_inter, max_tokens, phase,
-                      sm_budget, gemm_variant, row_gather, routed_scale)
+                      sm_budget, gemm_variant, row_gather, routed_scale, weight_format)
 
 
 def moe_ctx_workspace_bytes(cfg: moe_config) -> int:
@@ -244,6 +252,21 @@ class MoeContext:
         self._check(self.lib.moe_grouped_ffn(self.handle, _ptr(w_gate_up), _ptr(w_down), _ptr(x), _ptr(ws_gate_up),
                                              _ptr(ws_down), T))
 
+    def moe_grouped_ffn_fp8(self, wq_gate_up, sw_gate_up, wq_down, sw_down, x, wsq_gate_up=None, sws_gate_up=None,
+                            wsq_down=None, sws_down=None, T=None):
+        """wq_* are uint8 tensors of E4M3 codes, sw_* fp32 per-output-channel scales."""
+        for n, t in (("wq_gate_up", wq_gate_up), ("wq_down", wq_down), ("wsq_gate_up", wsq_gate_up),
+                     ("wsq_down", wsq_down)):
+            _dev(t, torch.uint8, n)
+        for n, t in (("sw_gate_up", sw_gate_up), ("sw_down", sw_down), ("sws_gate_up", sws_gate_up),
+                     ("sws_down", sws_down)):
+            _dev(t, torch.float32, n)
+        _dev(x, torch.bfloat16, "x")
+        T = x.shape[0] if T is None else T
+        self._check(self.lib.moe_grouped_ffn_fp8(self.handle, _ptr(wq_gate_up), _ptr(sw_gate_up), _ptr(wq_down),
+                                                 _ptr(sw_down), _ptr(x), _ptr(wsq_gate_up), _ptr(sws_gate_up),
+                                                 _ptr(wsq_down), _ptr(sws_down), T))
+
     def moe_combine(self, topk_w, inv_perm, out, T=None):
         _dev(topk_w, torch.float32, "topk_w"); _dev(inv_perm, torch.int32, "inv_perm"); _dev(out, torch.bfloat16, "out")
         T = out.shape[0] if T is None else T
@@ -280,6 +303,18 @@ class MoeContext:
                 "y_shared": view(ptrs[3], c.max_tokens, c.hidden, torch.bfloat16) if c.n_shared else None,
                 "counts": view(ptrs[4], 1, c.n_experts, torch.int32), "offsets": view(ptrs[5], 1, c.n_experts + 1, torch.int32)}
 
+    def fp8_debug_view(self, name: str, shape, dtype):
+        """View of one FP8 buffer of the last step: name in xq, sx, aq, sa."""
+        ptrs = [ctypes.c_void_p() for _ in range(4)]
+        self._check(self.lib.moe_ctx_debug_ptrs_fp8(self.handle, *[ctypes.byref(p) for p in ptrs]))
+        p = ptrs[("xq", "sx", "aq", "sa").index(name)]
+        n = 1
+        for d in shape:
+            n *= d
+        esz = torch.empty(0, dtype=dtype).element_size()
+        off = p.value - self.workspace.data_ptr()
+        return self.workspace[off:off + n * esz].view(dtype).view(*shape)
+
     # -- convenience: one whole step on device tensors (calls the four entry points in order)
     def layer(self, x, logits, select_bias, w_gate_up, w_down, ws_gate_up=None, ws_down=None, out=None, bufs=None):
         T, k, E = x.shape[0], self.cfg.top_k, self.cfg.n_experts
@@ -291,6 +326,23 @@ class MoeContext:
         self.moe_dispatch_layout(bufs["topk_idx"], x, bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"],
                                  T=T)
         self.moe_grouped_ffn(w_gate_up, w_down, x, ws_gate_up, ws_down, T=T)
+        self.moe_combine(bufs["topk_w"], bufs["inv_perm"], out, T=T)
+        return out, bufs
+
+    def layer_fp8(self, x, logits, select_bias, w8: dict, out=None, bufs=None):
+        """One step with FP8 weights; `w8` holds wq_gate_up, sw_gate_up, wq_down, sw_down and, with a shared
+        expert, wsq_gate_up, sws_gate_up, wsq_down, sws_down (see workloads.make_weights_fp8)."""
+        T, k, E = x.shape[0], self.cfg.top_k, self.cfg.n_experts
+        if bufs is None:
+            bufs = alloc_step_buffers(T, k, E, x.device)
+        if out is None:
+            out = torch.empty(T, self.cfg.hidden, dtype=torch.bfloat16, device=x.device)
+        self.moe_route(logits, select_bias, bufs["topk_idx"], bufs["topk_w"], T=T)
+        self.moe_dispatch_layout(bufs["topk_idx"], x, bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"],
+                                 T=T)
+        self.moe_grouped_ffn_fp8(w8["wq_gate_up"], w8["sw_gate_up"], w8["wq_down"], w8["sw_down"], x,
+                                 w8.get("wsq_gate_up"), w8.get("sws_gate_up"), w8.get("wsq_down"), w8.get("sws_down"),
+                                 T=T)
         self.moe_combine(bufs["topk_w"], bufs["inv_perm"], out, T=T)
         return out, bufs
 

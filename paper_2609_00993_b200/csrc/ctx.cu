@@ -37,6 +37,15 @@ struct BufferSet {
   char* x_stage;     // bf16 [T,H]
   char* out_stage;   // bf16 [T,H]
   int32_t* scan;     // layout scratch
+  // FP8 variant only: quantised activations and their per-row scales
+  char* xq;          // e4m3 [N,H]
+  float* sx;         // [N]
+  char* aq;          // e4m3 [N,I]
+  float* sa;         // [N]
+  char* xq_shared;   // e4m3 [T,H]
+  float* sx_shared;  // [T]
+  char* aq_shared;   // e4m3 [T,Is]
+  float* sa_shared;  // [T]
 };
 
 struct Layout {
@@ -73,6 +82,15 @@ size_t carve_set(const moe_config& c, char* base, BufferSet* out) {
   b.x_stage = take(T * H * 2);
   b.out_stage = take(T * H * 2);
   b.scan = reinterpret_cast<int32_t*>(take(moe::layout_scratch_ints((int64_t)N, (int)E) * 4));
+  const size_t f8 = c.weight_format == MOE_WEIGHTS_FP8_E4M3 ? 1 : 0;
+  b.xq = take(f8 * N * H);
+  b.sx = reinterpret_cast<float*>(take(f8 * N * 4));
+  b.aq = take(f8 * N * I);
+  b.sa = reinterpret_cast<float*>(take(f8 * N * 4));
+  b.xq_shared = take(f8 * (c.n_shared ? T * H : 0));
+  b.sx_shared = reinterpret_cast<float*>(take(f8 * (c.n_shared ? T * 4 : 0)));
+  b.aq_shared = take(f8 * T * Is);
+  b.sa_shared = reinterpret_cast<float*>(take(f8 * (c.n_shared ? T * 4 : 0)));
   if (out) *out = b;
   return off;
 }
@@ -92,6 +110,13 @@ const char* validate_config(const moe_config* c) {
   if (c->gemm_variant < MOE_GEMM_AUTO || c->gemm_variant > MOE_GEMM_VALIDATION) return "unknown gemm_variant";
   if (c->row_gather != 0 && c->row_gather != 1) return "row_gather must be 0 or 1";
   if (!(c->routed_scale == c->routed_scale)) return "routed_scale is NaN";
+  if (c->weight_format != MOE_WEIGHTS_BF16 && c->weight_format != MOE_WEIGHTS_FP8_E4M3) return "unknown weight_format";
+  if (c->weight_format == MOE_WEIGHTS_FP8_E4M3) {
+    if (c->hidden > 8192 || c->inter > 8192 || (c->n_shared && c->shared_inter > 8192))
+      return "FP8 weights: hidden, inter and shared_inter may not exceed 8192";
+    if (c->gemm_variant == MOE_GEMM_VALIDATION) return "FP8 weights need a tensor-core gemm_variant";
+    if (c->row_gather) return "the row gather does not apply to FP8 weights";
+  }
   return nullptr;
 }
 
@@ -548,6 +573,70 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
   return MOE_OK;
 }
 
+moe_status moe_grouped_ffn_fp8(moe_ctx* ctx, const void* wq_gate_up, const float* sw_gate_up, const void* wq_down,
+                               const float* sw_down, const void* x, const void* wsq_gate_up,
+                               const float* sws_gate_up, const void* wsq_down, const float* sws_down, int32_t T) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->cfg.weight_format != MOE_WEIGHTS_FP8_E4M3)
+    return fail(ctx, MOE_ERR_STATE, "the context was not created with weight_format = MOE_WEIGHTS_FP8_E4M3");
+  if (ctx->state != ST_LAID_OUT)
+    return fail(ctx, MOE_ERR_STATE, "moe_grouped_ffn_fp8 needs a moe_dispatch_layout with x in the same step");
+  if (T != ctx->T) return fail(ctx, MOE_ERR_INVALID_ARG, "T = %d differs from the layout's T = %d", T, ctx->T);
+  if (!wq_gate_up || !sw_gate_up || !wq_down || !sw_down)
+    return fail(ctx, MOE_ERR_INVALID_ARG, "routed weights or scales are NULL");
+  const bool shared = ctx->cfg.n_shared != 0;
+  if (shared && (!wsq_gate_up || !sws_gate_up || !wsq_down || !sws_down || (!x && T > 0)))
+    return fail(ctx, MOE_ERR_INVALID_ARG, "the shared expert needs its weights, scales and x");
+  if (misaligned(wq_gate_up) || misaligned(sw_gate_up) || misaligned(wq_down) || misaligned(sw_down) ||
+      misaligned(x) || misaligned(wsq_gate_up) || misaligned(sws_gate_up) || misaligned(wsq_down) ||
+      misaligned(sws_down))
+    return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+  DeviceGuard guard(ctx->device);
+  BufferSet& b = ctx->sets[ctx->cur];
+  const moe_config& c = ctx->cfg;
+  const int64_t N = (int64_t)T * c.top_k, Ncap = (int64_t)c.max_tokens * c.top_k;
+  int n = 0;
+  cudaError_t e = cudaSuccess;
+  if (T > 0) {
+    // quantise -> GEMM1 + SwiGLU -> quantise -> GEMM2; the shared expert's passes ride in the routed launches
+    {
+      StageTimer tm(ctx, 8);
+      e = moe::launch_quantize_rows(b.x_perm, N, c.hidden, b.xq, b.sx, ctx->stream, &n);
+      if (e == cudaSuccess && shared)
+        e = moe::launch_quantize_rows(x, T, c.hidden, b.xq_shared, b.sx_shared, ctx->stream, &n);
+    }
+    moe::GemmProblem g1{b.xq, wq_gate_up, b.act, ctx->offsets, 0, Ncap, N, c.n_experts, c.inter, c.hidden, true};
+    g1.fp8 = true;
+    g1.row_scale = b.sx;
+    g1.w_scale = sw_gate_up;
+    moe::GemmDenseGroup s1{b.xq_shared, wsq_gate_up, b.act_shared, T, c.shared_inter, c.hidden, b.sx_shared,
+                           sws_gate_up};
+    if (e == cudaSuccess) {
+      StageTimer tm(ctx, 3);
+      e = run_gemm(ctx, g1, shared ? &s1 : nullptr, T, &n);
+    }
+    if (e == cudaSuccess) {
+      StageTimer tm(ctx, 9);
+      e = moe::launch_quantize_rows(b.act, N, c.inter, b.aq, b.sa, ctx->stream, &n);
+      if (e == cudaSuccess && shared)
+        e = moe::launch_quantize_rows(b.act_shared, T, c.shared_inter, b.aq_shared, b.sa_shared, ctx->stream, &n);
+    }
+    moe::GemmProblem g2{b.aq, wq_down, b.y_perm, ctx->offsets, 0, Ncap, N, c.n_experts, c.hidden, c.inter, false};
+    g2.fp8 = true;
+    g2.row_scale = b.sa;
+    g2.w_scale = sw_down;
+    moe::GemmDenseGroup s2{b.aq_shared, wsq_down, b.y_shared, T, c.hidden, c.shared_inter, b.sa_shared, sws_down};
+    if (e == cudaSuccess) {
+      StageTimer tm(ctx, 4);
+      e = run_gemm(ctx, g2, shared ? &s2 : nullptr, T, &n);
+    }
+  }
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_grouped_ffn_fp8");
+  ctx->state = ST_FFN_DONE;
+  mark(ctx, n);
+  return MOE_OK;
+}
+
 moe_status moe_combine(moe_ctx* ctx, const float* topk_w, const int32_t* inv_perm, int32_t T, void* out) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
   if (ctx->state != ST_FFN_DONE) return fail(ctx, MOE_ERR_STATE, "moe_combine needs moe_grouped_ffn in the same step");
@@ -651,6 +740,19 @@ moe_status moe_ctx_debug_ptrs(moe_ctx* ctx, void** x_perm, void** act, void** y_
   if (y_shared) *y_shared = b.y_shared;
   if (counts) *counts = b.counts;
   if (offsets) *offsets = b.offsets;
+  return MOE_OK;
+}
+
+moe_status moe_ctx_debug_ptrs_fp8(moe_ctx* ctx, void** xq, float** sx, void** aq, float** sa) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->cfg.weight_format != MOE_WEIGHTS_FP8_E4M3)
+    return fail(ctx, MOE_ERR_STATE, "the context was not created with weight_format = MOE_WEIGHTS_FP8_E4M3");
+  const int set = (ctx->n_sets == 2 && ctx->state == ST_IDLE) ? (ctx->cur ^ 1) : ctx->cur;
+  BufferSet& b = ctx->sets[set];
+  if (xq) *xq = b.xq;
+  if (sx) *sx = b.sx;
+  if (aq) *aq = b.aq;
+  if (sa) *sa = b.sa;
   return MOE_OK;
 }
 

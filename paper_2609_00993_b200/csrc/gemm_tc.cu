@@ -72,6 +72,12 @@ struct TcParams {
   int32_t n_feat2;
   int32_t K2;
   __nv_bfloat16* out2;
+  // FP8 variant: operands are E4M3 codes; the accumulator is scaled by row_scale[row] * w_scale[weight row]
+  // (w_scale: [experts, weight rows of one expert]; *2: the dense group's)
+  const float* row_scale;
+  const float* row_scale2;
+  const float* w_scale;
+  const float* w_scale2;
 };
 
 // ---------------------------------------------------------------------------------- PTX wrappers
@@ -160,6 +166,18 @@ __device__ __forceinline__ void umma_bf16_lo(uint32_t tmem_d, uint32_t a_lo, uin
       ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same for E4M3 operands (kind::f8f6f4, 32 K-elements per instruction).
+__device__ __forceinline__ void umma_e4m3_lo(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                             uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %4, p;\n\t}"
+      ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // The mbarrier gets one arrival when every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -207,6 +225,11 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr) {
 // Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, dense, M x N.
 __device__ __forceinline__ uint32_t umma_idesc(uint32_t M, uint32_t N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+// The same with E4M3 A and B (format code 0 in both fields).
+__device__ __forceinline__ uint32_t umma_idesc_e4m3(uint32_t M, uint32_t N) {
+  return (1u << 4) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
 __device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
@@ -269,11 +292,15 @@ __device__ __forceinline__ Tile decode_tile(int tile, int dense_tiles, int n_ft2
 // each row's 128-byte slice for the current k-block from its source row (perm[p] / top_k) into the X tile with
 // 16-byte cp.async, in the same 128-byte-swizzled layout TMA would produce; the stage's barrier counts one
 // arrival per gather thread, delivered when that thread's copies have landed.  TMA then carries the weights only.
-template <bool SWAP, bool GATED, bool GATHER>
+// FP8: both operands are E4M3 codes, a pipeline stage holds 128 K-elements (still 128 bytes per row), and the
+// epilogue multiplies the accumulator by the row's and the weight row's scale.
+template <bool SWAP, bool GATED, bool GATHER, bool FP8>
 __global__ void __launch_bounds__(GATHER ? kThreadsGather : kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_x2, const __grid_constant__ CUtensorMap map_w2,
                        const __grid_constant__ TcParams p) {
+  static_assert(!(GATHER && FP8), "the row gather exists for bf16 operands only");
+  constexpr int kbk = FP8 ? 2 * kBlockK : kBlockK;  // K elements per stage
   extern __shared__ uint8_t smem_raw[];
   // carve: [stages] | epilogue staging (large-M) | barriers | tmem slot | abort | prefix[E+1] | seg[E+1]
   //   stage: W box0 | W box1 | X tile
@@ -298,7 +325,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   const int tile_rows = p.row_tile;  // token rows per tile of the list
   constexpr int kFeatPerTile = GATED ? 128 : 256;
   const int n_ft = (p.n_feat + kFeatPerTile - 1) / kFeatPerTile;
-  const int num_kb1 = (p.K + kBlockK - 1) / kBlockK, num_kb2 = (p.K2 + kBlockK - 1) / kBlockK;
+  const int num_kb1 = (p.K + kbk - 1) / kbk, num_kb2 = (p.K2 + kbk - 1) / kbk;
   const int n_ft2 = (p.n_feat2 + kFeatPerTile - 1) / kFeatPerTile;
   const int dense_tiles = p.rows2 > 0 ? ((p.rows2 + p.row_tile - 1) / p.row_tile) * n_ft2 : 0;
   const uint32_t acc_cols = SWAP ? 2u * (uint32_t)p.row_tile : 256u;  // TMEM columns per accumulator stage
@@ -363,7 +390,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         const CUtensorMap* mx = t.dense ? &map_x2 : &map_x;
         const int w_e = t.dense ? 0 : p.e_base + t.e;
         const int num_kb = t.dense ? num_kb2 : num_kb1;
-        for (int kb = 0, k0 = 0; kb < num_kb; ++kb, k0 += kBlockK) {
+        for (int kb = 0, k0 = 0; kb < num_kb; ++kb, k0 += kbk) {
           if (!mbar_wait(bar_empty + 8u * ring.stage, ring.phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t full = bar_full + 8u * ring.stage;
           const uint32_t st = base_addr + ring.stage * (uint32_t)stage_bytes;
@@ -397,7 +424,8 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         const uint32_t d0 = tmem_base + as * acc_cols;
         // small-M: the MMA N covers only the rows this tile really has, rounded up to 16
         const uint32_t n_swap = (uint32_t)min(p.row_tile, (t.rows + 15) & ~15);
-        const uint32_t idesc = SWAP ? umma_idesc(128, n_swap) : umma_idesc(128, 256);
+        const uint32_t n_mma = SWAP ? n_swap : 256u;
+        const uint32_t idesc = FP8 ? umma_idesc_e4m3(128, n_mma) : umma_idesc(128, n_mma);
         const int num_kb = t.dense ? num_kb2 : num_kb1;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(bar_full + 8u * ring.stage, ring.phase, abort_flag)) { ok = false; break; }
@@ -406,14 +434,18 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           const uint32_t lo_w0 = lo_base + ring.stage * lo_stage;  // weight box 0; box 1 and the X tile follow
 #pragma unroll
           for (int kk = 0; kk < kBlockK / kUmmaK; ++kk) {
-            const uint32_t adv = (uint32_t)((kk * kUmmaK * 2) >> 4);  // +32 bytes per K step, in 16-byte units
+            const uint32_t adv = (uint32_t)((kk * kUmmaK * 2) >> 4);  // +32 bytes per MMA (16 bf16 or 32 E4M3), in 16-byte units
             const uint32_t acc = (kb | kk) != 0 ? 1u : 0u;
+            auto mma = [&](uint32_t d, uint32_t a_lo, uint32_t b_lo) {
+              if (FP8) umma_e4m3_lo(d, a_lo, b_lo, desc_hi, idesc, acc);
+              else umma_bf16_lo(d, a_lo, b_lo, desc_hi, idesc, acc);
+            };
             if (SWAP) {
-              umma_bf16_lo(d0, lo_w0 + adv, lo_w0 + 2 * lo_box + adv, desc_hi, idesc, acc);
-              umma_bf16_lo(d0 + (uint32_t)p.row_tile, lo_w0 + lo_box + adv, lo_w0 + 2 * lo_box + adv, desc_hi, idesc, acc);
+              mma(d0, lo_w0 + adv, lo_w0 + 2 * lo_box + adv);
+              mma(d0 + (uint32_t)p.row_tile, lo_w0 + lo_box + adv, lo_w0 + 2 * lo_box + adv);
             } else {
               // the two weight boxes are contiguous: one N = 256 operand
-              umma_bf16_lo(d0, lo_w0 + 2 * lo_box + adv, lo_w0 + adv, desc_hi, idesc, acc);
+              mma(d0, lo_w0 + 2 * lo_box + adv, lo_w0 + adv);
             }
           }
           umma_commit(bar_empty + 8u * ring.stage);  // the stage is free once these MMAs have read it
@@ -492,12 +524,21 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       const uint32_t d0 = tmem_base + as * acc_cols + lane_base;
       __nv_bfloat16* const out = t.dense ? p.out2 : p.out;
       const int n_feat = t.dense ? p.n_feat2 : p.n_feat;
+      // FP8: scales of this tile's rows and of its expert's weight rows (gate rows first, then up rows)
+      const float* const rsp = FP8 ? (t.dense ? p.row_scale2 : p.row_scale) + t.row0 : nullptr;
+      const float* const wsp =
+          FP8 ? (t.dense ? p.w_scale2 : p.w_scale + (size_t)(p.e_base + t.e) * (GATED ? 2 : 1) * n_feat) : nullptr;
       bool released = false;  // has this warp already handed the accumulator stage back?
       if (SWAP) {
         // lane = weight row (output feature), column = token
         const int fl = warp * 32 + lane;
         const int f_a = t.ft * kFeatPerTile + fl;                 // box 0 feature
         const int f_b = f_a + kWBoxRows;                          // box 1 feature (down pass only)
+        float ws_a = 1.f, ws_b = 1.f;  // FP8: scales of this lane's two weight rows
+        if (FP8) {
+          if (f_a < n_feat) ws_a = wsp[f_a];
+          if (GATED ? f_a < n_feat : f_b < n_feat) ws_b = wsp[GATED ? n_feat + f_a : f_b];
+        }
         for (int c = 0; c < t.rows; c += 16) {
           uint32_t ra[16], rb[16];
           tmem_ld16(d0 + (uint32_t)c, ra);
@@ -507,7 +548,12 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           for (int i = 0; i < 16; ++i) {
             if (c + i < t.rows) {
               __nv_bfloat16* orow = out + (size_t)(t.row0 + c + i) * n_feat;
-              const float a = __uint_as_float(ra[i]), b = __uint_as_float(rb[i]);
+              float a = __uint_as_float(ra[i]), b = __uint_as_float(rb[i]);
+              if (FP8) {
+                const float rs = __ldg(rsp + c + i);
+                a *= rs * ws_a;
+                b *= rs * ws_b;
+              }
               if (GATED) {
                 if (f_a < n_feat) orow[f_a] = __float2bfloat16_rn(silu_mul(a, b));
               } else {
@@ -525,6 +571,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         constexpr int kPairs = kFeatPerTile / 64;
         uint8_t* stage_tile = epi_smem + warp * 4096;  // 32 rows x 128 bytes
         const int rows_here = t.rows - warp * 32;       // rows of this warp's 32 that are valid (may be <= 0)
+        const float rs = (FP8 && lane < rows_here) ? rsp[warp * 32 + lane] : 0.f;  // FP8: this lane's row scale
         for (int pc = 0; pc < kPairs; ++pc) {
           const int f0 = t.ft * kFeatPerTile + pc * 64;
           if (f0 >= n_feat) break;  // uniform across the CTA
@@ -532,16 +579,47 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
           for (int h = 0; h < 2; ++h) {
             uint32_t ra[32], packed[16];
             tmem_ld32(d0 + (uint32_t)(pc * 64 + h * 32), ra);
+            // FP8: the 32 columns' weight-row scales (the same for every lane: broadcast loads); a chunk that
+            // reaches past n_feat reads no scales and is not stored either
+            const bool scaled = FP8 && f0 + h * 32 + 32 <= n_feat;
             if (GATED) {
               uint32_t rb[32];
               tmem_ld32(d0 + (uint32_t)(128 + pc * 64 + h * 32), rb);
               tmem_ld_wait();
+              if (FP8) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                  const float4 sg = scaled ? __ldg(reinterpret_cast<const float4*>(wsp + f0 + h * 32) + q)
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+                  const float4 su = scaled ? __ldg(reinterpret_cast<const float4*>(wsp + n_feat + f0 + h * 32) + q)
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+                  ra[4 * q + 0] = __float_as_uint(__uint_as_float(ra[4 * q + 0]) * (rs * sg.x));
+                  ra[4 * q + 1] = __float_as_uint(__uint_as_float(ra[4 * q + 1]) * (rs * sg.y));
+                  ra[4 * q + 2] = __float_as_uint(__uint_as_float(ra[4 * q + 2]) * (rs * sg.z));
+                  ra[4 * q + 3] = __float_as_uint(__uint_as_float(ra[4 * q + 3]) * (rs * sg.w));
+                  rb[4 * q + 0] = __float_as_uint(__uint_as_float(rb[4 * q + 0]) * (rs * su.x));
+                  rb[4 * q + 1] = __float_as_uint(__uint_as_float(rb[4 * q + 1]) * (rs * su.y));
+                  rb[4 * q + 2] = __float_as_uint(__uint_as_float(rb[4 * q + 2]) * (rs * su.z));
+                  rb[4 * q + 3] = __float_as_uint(__uint_as_float(rb[4 * q + 3]) * (rs * su.w));
+                }
+              }
 #pragma unroll
               for (int i = 0; i < 16; ++i)
                 packed[i] = pack_bf16(silu_mul(__uint_as_float(ra[2 * i]), __uint_as_float(rb[2 * i])),
                                       silu_mul(__uint_as_float(ra[2 * i + 1]), __uint_as_float(rb[2 * i + 1])));
             } else {
               tmem_ld_wait();
+              if (FP8) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                  const float4 sw = scaled ? __ldg(reinterpret_cast<const float4*>(wsp + f0 + h * 32) + q)
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+                  ra[4 * q + 0] = __float_as_uint(__uint_as_float(ra[4 * q + 0]) * (rs * sw.x));
+                  ra[4 * q + 1] = __float_as_uint(__uint_as_float(ra[4 * q + 1]) * (rs * sw.y));
+                  ra[4 * q + 2] = __float_as_uint(__uint_as_float(ra[4 * q + 2]) * (rs * sw.z));
+                  ra[4 * q + 3] = __float_as_uint(__uint_as_float(ra[4 * q + 3]) * (rs * sw.w));
+                }
+              }
 #pragma unroll
               for (int i = 0; i < 16; ++i) packed[i] = pack_bf16(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1]));
             }
@@ -602,14 +680,14 @@ const bool g_inject_producer_stall = [] {
 const char* g_init_error = nullptr;
 
 bool encode_map(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                const uint32_t* box) {
+                const uint32_t* box, bool bytes = false) {
   cuuint64_t gdim[3];
   cuuint64_t gstr[2];
   cuuint32_t bdim[3];
   cuuint32_t estr[3] = {1, 1, 1};
   for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bdim[i] = box[i]; }
   for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
-  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr,
+  CUresult r = g_encode(map, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr,
                         bdim, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -658,22 +736,29 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
   if (row_tile < 16 || row_tile > 128 || (row_tile & (row_tile - 1)) != 0) return cudaErrorNotSupported;
   if (p.rows_bound > 0x7fffffffLL / 2) return cudaErrorNotSupported;
 
+  const bool fp8 = p.fp8;
+  if (fp8 && (gather || p.row_scale == nullptr || p.w_scale == nullptr || p.K % 16 != 0 || p.n_feat % 64 != 0 ||
+              (dense != nullptr && (dense->row_scale == nullptr || dense->w_scale == nullptr || dense->K % 16 != 0 ||
+                                    dense->n_feat % 64 != 0))))
+    return cudaErrorNotSupported;
+  const uint64_t esz = fp8 ? 1 : 2;                                    // bytes per operand element
+  const uint32_t box_k = (uint32_t)(fp8 ? 2 * kBlockK : kBlockK);      // 128 bytes of K per stage row
   const int groups = p.offsets ? p.E : 1;
   const uint64_t w_rows = (uint64_t)(p.gated ? 2 : 1) * (uint64_t)p.n_feat;
   CUtensorMap mx, mw;
   {
     const uint64_t src_rows = gather ? (uint64_t)((p.rows_bound + p.top_k - 1) / p.top_k) : (uint64_t)p.rows_bound;
     const uint64_t dims[2] = {(uint64_t)p.K, src_rows};
-    const uint64_t str[1] = {(uint64_t)p.K * 2};
-    const uint32_t box[2] = {(uint32_t)kBlockK, (uint32_t)row_tile};
+    const uint64_t str[1] = {(uint64_t)p.K * esz};
+    const uint32_t box[2] = {box_k, (uint32_t)row_tile};
     // with the row gather no tensor map of the token rows is used; encode the source so that the map is valid
-    if (!encode_map(&mx, gather ? p.gather_src : p.A, 2, dims, str, box)) return cudaErrorInvalidValue;
+    if (!encode_map(&mx, gather ? p.gather_src : p.A, 2, dims, str, box, fp8)) return cudaErrorInvalidValue;
   }
   {
     const uint64_t dims[3] = {(uint64_t)p.K, w_rows, (uint64_t)groups};
-    const uint64_t str[2] = {(uint64_t)p.K * 2, w_rows * (uint64_t)p.K * 2};
-    const uint32_t box[3] = {(uint32_t)kBlockK, (uint32_t)kWBoxRows, 1u};
-    if (!encode_map(&mw, p.W, 3, dims, str, box)) return cudaErrorInvalidValue;
+    const uint64_t str[2] = {(uint64_t)p.K * esz, w_rows * (uint64_t)p.K * esz};
+    const uint32_t box[3] = {box_k, (uint32_t)kWBoxRows, 1u};
+    if (!encode_map(&mw, p.W, 3, dims, str, box, fp8)) return cudaErrorInvalidValue;
   }
 
   const int e_begin = p.offsets ? p.e_begin : 0;
@@ -683,13 +768,13 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
   if (dense != nullptr) {
     const uint64_t w2_rows = (uint64_t)(p.gated ? 2 : 1) * (uint64_t)dense->n_feat;
     const uint64_t dx[2] = {(uint64_t)dense->K, (uint64_t)dense->rows};
-    const uint64_t sx[1] = {(uint64_t)dense->K * 2};
-    const uint32_t bx[2] = {(uint32_t)kBlockK, (uint32_t)row_tile};
-    if (!encode_map(&mx2, dense->A, 2, dx, sx, bx)) return cudaErrorInvalidValue;
+    const uint64_t sx[1] = {(uint64_t)dense->K * esz};
+    const uint32_t bx[2] = {box_k, (uint32_t)row_tile};
+    if (!encode_map(&mx2, dense->A, 2, dx, sx, bx, fp8)) return cudaErrorInvalidValue;
     const uint64_t dw[3] = {(uint64_t)dense->K, w2_rows, 1};
-    const uint64_t sw[2] = {(uint64_t)dense->K * 2, w2_rows * (uint64_t)dense->K * 2};
-    const uint32_t bw[3] = {(uint32_t)kBlockK, (uint32_t)kWBoxRows, 1u};
-    if (!encode_map(&mw2, dense->W, 3, dw, sw, bw)) return cudaErrorInvalidValue;
+    const uint64_t sw[2] = {(uint64_t)dense->K * esz, w2_rows * (uint64_t)dense->K * esz};
+    const uint32_t bw[3] = {box_k, (uint32_t)kWBoxRows, 1u};
+    if (!encode_map(&mw2, dense->W, 3, dw, sw, bw, fp8)) return cudaErrorInvalidValue;
   }
   TcParams prm;
   prm.gather_src = static_cast<const __nv_bfloat16*>(p.gather_src);
@@ -700,6 +785,10 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
   prm.n_feat2 = dense ? dense->n_feat : 8;
   prm.K2 = dense ? dense->K : 8;
   prm.out2 = dense ? static_cast<__nv_bfloat16*>(dense->out) : nullptr;
+  prm.row_scale = p.row_scale;
+  prm.w_scale = p.w_scale;
+  prm.row_scale2 = dense ? dense->row_scale : nullptr;
+  prm.w_scale2 = dense ? dense->w_scale : nullptr;
   prm.offsets = p.offsets ? p.offsets + e_begin : nullptr;
   prm.fixed_rows = p.fixed_rows;
   prm.E = e_end - e_begin;
@@ -731,13 +820,19 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
   if (grid < 1) grid = 1;
   cudaError_t err;
   if (gather)
-    err = launch_variant(grouped_gemm_tc_kernel<false, true, true>, kThreadsGather, mx, mw, mx2, mw2, prm, grid, smem, stream);
+    err = launch_variant(grouped_gemm_tc_kernel<false, true, true, false>, kThreadsGather, mx, mw, mx2, mw2, prm, grid, smem, stream);
+  else if (fp8 && swap_ab)
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true, false, true>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
+                  : launch_variant(grouped_gemm_tc_kernel<true, false, false, true>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
+  else if (fp8)
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true, false, true>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
+                  : launch_variant(grouped_gemm_tc_kernel<false, false, false, true>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
   else if (swap_ab)
-    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
-                  : launch_variant(grouped_gemm_tc_kernel<true, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
+                  : launch_variant(grouped_gemm_tc_kernel<true, false, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
   else
-    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
-                  : launch_variant(grouped_gemm_tc_kernel<false, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
+                  : launch_variant(grouped_gemm_tc_kernel<false, false, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }

@@ -64,6 +64,11 @@ struct GemmProblem {
   const void* gather_src = nullptr;
   const int32_t* perm = nullptr;
   int32_t top_k = 1;
+  // FP8 variant (tensor-core path only): A and W hold E4M3 codes; the result is scaled by
+  // row_scale[row] * w_scale[expert, weight row] (w_scale: [E, (gated?2:1)*n_feat]) before the epilogue's maths.
+  bool fp8 = false;
+  const float* row_scale = nullptr;
+  const float* w_scale = nullptr;
 };
 
 // A dense group (the shared expert) that rides in the same launch as a grouped problem: its tiles are added
@@ -75,7 +80,14 @@ struct GemmDenseGroup {
   int32_t rows;
   int32_t n_feat;
   int32_t K;
+  const float* row_scale = nullptr;  // FP8 variant: [rows]
+  const float* w_scale = nullptr;    // FP8 variant: [(gated?2:1)*n_feat]
 };
+
+// FP8 variant: per-row dynamic quantisation of bf16 rows [rows, n] -> E4M3 codes [rows, n] + scale [rows]
+// (n a multiple of 8, at most 8192).
+cudaError_t launch_quantize_rows(const void* x, int64_t rows, int n, void* q, float* scale, cudaStream_t stream,
+                                 int* n_launches);
 
 cudaError_t launch_gemm_validation(const GemmProblem& p, cudaStream_t stream, int* n_launches);
 

@@ -1,0 +1,79 @@
+// FP8 precision variant: per-row dynamic quantisation of bf16 activation rows to E4M3.
+//
+//   amax  = max_i |v_i|                    scale = amax / 448   (1 when the row is all zero)
+//   code_i = e4m3(v_i / scale)             round to nearest even, saturating at +-448
+//
+// The codes are integers decided by floating point, so every operation that decides them is spelled out in
+// IEEE fp32 (__fdiv_rn, cvt.rn.satfinite) and no fast-math substitute (reciprocal, fused scaling) is used.
+// One CTA of 128 threads per row; the row stays in registers between the two passes (rows of up to 8192
+// elements), so it is read once: 2 n bytes in, n + 4 bytes out per row.
+#include <cuda_bf16.h>
+#include <cuda_fp8.h>
+
+#include "kernels.h"
+
+namespace moe {
+namespace {
+
+constexpr int kQuantThreads = 128;
+constexpr int kQuantMaxVecs = 8;  // 16-byte vectors (8 bf16) per thread
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+
+__device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
+  return (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);  // lo in bits 0-7
+}
+
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_rows_kernel(const uint4* __restrict__ x, int n_vec, uint2* __restrict__ q, float* __restrict__ scale) {
+  __shared__ uint32_t warp_max[kQuantThreads / 32];
+  const int64_t row = blockIdx.x;
+  const uint4* xr = x + row * n_vec;
+  uint4 v[kQuantMaxVecs];
+  uint32_t m = 0;  // largest |bf16| as a bit pattern: for finite values the integer order is the value order
+#pragma unroll
+  for (int j = 0; j < kQuantMaxVecs; ++j) {
+    const int i = threadIdx.x + j * kQuantThreads;
+    v[j] = i < n_vec ? xr[i] : make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      m = max(m, w[c] & 0x7fffu);
+      m = max(m, (w[c] >> 16) & 0x7fffu);
+    }
+  }
+  m = __reduce_max_sync(0xffffffffu, m);
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  m = max(max(warp_max[0], warp_max[1]), max(warp_max[2], warp_max[3]));
+  const float amax = bf16_bits_to_f32(m);
+  const float s = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+  if (threadIdx.x == 0) scale[row] = s;
+  uint2* qr = q + row * n_vec;
+#pragma unroll
+  for (int j = 0; j < kQuantMaxVecs; ++j) {
+    const int i = threadIdx.x + j * kQuantThreads;
+    if (i >= n_vec) continue;
+    const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+    uint32_t pair[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      pair[c] = e4m3x2(__fdiv_rn(bf16_bits_to_f32(w[c] & 0xffffu), s), __fdiv_rn(bf16_bits_to_f32(w[c] >> 16), s));
+    qr[i] = make_uint2(pair[0] | (pair[1] << 16), pair[2] | (pair[3] << 16));
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_quantize_rows(const void* x, int64_t rows, int n, void* q, float* scale, cudaStream_t stream,
+                                 int* n_launches) {
+  if (rows <= 0) return cudaSuccess;
+  if (n <= 0 || n % 8 != 0 || n > 8 * kQuantThreads * kQuantMaxVecs || rows > 0x7fffffffLL) return cudaErrorNotSupported;
+  quantize_rows_kernel<<<(unsigned)rows, kQuantThreads, 0, stream>>>(static_cast<const uint4*>(x), n / 8,
+                                                                     static_cast<uint2*>(q), scale);
+  cudaError_t err = cudaGetLastError();
+  if (err == cudaSuccess && n_launches) *n_launches += 1;
+  return err;
+}
+
+}  // namespace moe

@@ -81,6 +81,40 @@ def make_weights(shape: LayerShape, seed: int, device="cpu") -> dict:
     return out
 
 
+def make_weights_fp8(shape: LayerShape, seed: int, device="cpu", std: float = 0.02) -> dict:
+    """Random-init layer weights in the FP8 checkpoint format: E4M3 codes (uint8) plus one fp32 scale per output
+    channel.  A channel's codes are N(0, 112) clamped to the E4M3 range and converted by torch's own float8 type
+    (4 sigma reaches the largest code, as a per-channel absmax quantiser would produce); its scale is
+    std / 112 times a factor drawn from [0.8, 1.2], so that scale * code ~ N(0, std) like the bf16 weights.
+
+    wq_gate_up [E, 2I, H], sw_gate_up [E, 2I], wq_down [E, H, I], sw_down [E, H]; with a shared expert also
+    wsq_gate_up [2Is, H], sws_gate_up [2Is], wsq_down [H, Is], sws_down [H].
+    """
+    g = _gen(seed, device)
+
+    def codes(rows, cols):
+        v = (torch.randn(rows, cols, generator=g, device=device) * 112.0).clamp_(-448.0, 448.0)
+        return v.to(torch.float8_e4m3fn).view(torch.uint8)
+
+    def scales(*dims):
+        return ((0.8 + 0.4 * torch.rand(*dims, generator=g, device=device)) * (std / 112.0)).float()
+
+    wq_gate_up = torch.empty(shape.E, 2 * shape.I, shape.H, dtype=torch.uint8, device=device)
+    wq_down = torch.empty(shape.E, shape.H, shape.I, dtype=torch.uint8, device=device)
+    for e in range(shape.E):
+        wq_gate_up[e].copy_(codes(2 * shape.I, shape.H))
+        wq_down[e].copy_(codes(shape.H, shape.I))
+    out = {"wq_gate_up": wq_gate_up, "sw_gate_up": scales(shape.E, 2 * shape.I), "wq_down": wq_down,
+           "sw_down": scales(shape.E, shape.H), "wsq_gate_up": None, "sws_gate_up": None, "wsq_down": None,
+           "sws_down": None}
+    if shape.shared_I:
+        out["wsq_gate_up"] = codes(2 * shape.shared_I, shape.H)
+        out["sws_gate_up"] = scales(2 * shape.shared_I)
+        out["wsq_down"] = codes(shape.H, shape.shared_I)
+        out["sws_down"] = scales(shape.H)
+    return out
+
+
 def zipf_log_weight(E: int, s: float, seed: int, device="cpu") -> torch.Tensor:
     """log of Zipf(s) popularity per expert id: rank r in 1..E gets r^-s, ranks
     assigned to expert ids by a seeded permutation (hot experts are not adjacent)."""
