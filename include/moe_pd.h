@@ -177,8 +177,9 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
                            const void* ws_gate_up, const void* ws_down, int32_t T);
 
 /* Stages a6-a8 with FP8 weights and activations (context created with weight_format = MOE_WEIGHTS_FP8_E4M3;
- * same place in the step as moe_grouped_ffn).  The paper names FP8 runs but prints no recipe; this one is
- * W8A8 with OCP E4M3 codes (1-4-3 bits, bias 7, largest finite value 448, no infinities):
+ * same place in the step as moe_grouped_ffn, which such a context refuses).  The paper names FP8 runs but
+ * prints no recipe; this one is W8A8 with OCP E4M3 codes (1-4-3 bits, bias 7, largest finite value 448, no
+ * infinities):
  *   weights      wq_* hold E4M3 codes, sw_* one fp32 scale per output channel (weight row):
  *                W[e,r,:] = sw[e,r] * decode(wq[e,r,:])
  *   activations  every bf16 row v entering a GEMM is quantised on the fly, per row:
@@ -186,16 +187,17 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
  *                IEEE fp32, conversion round-to-nearest-even saturating at +-448
  *   GEMM1        g, u = (sum_h x_code * w_code) * scale_x[p] * sw[e,row], act = silu(g) * u stored as bf16
  *   GEMM2        act is quantised per row as above; y = (sum_i a_code * w_code) * scale_a[p] * sw[e,c], bf16
- * The sums run on the tensor cores (tcgen05 kind::f8f6f4) with fp32 accumulation.  The shared expert (S = 1)
- * is computed the same way from x with its own codes and scales.
+ * The sums run on the tensor cores (tcgen05 kind::f8f6f4) with fp32 accumulation.  On such a context
+ * moe_dispatch_layout quantises each row of x once (stage 8 of the profile) and moves the codes and the row
+ * scales instead of the bf16 rows, so the workspace holds no bf16 x_perm.  The shared expert (S = 1) is computed
+ * the same way from the quantised x with its own codes and scales.
  * wq_gate_up [E,2I,H] uint8, sw_gate_up [E,2I] fp32, wq_down [E,H,I] uint8, sw_down [E,H] fp32;
- * wsq_gate_up [2I_s,H], sws_gate_up [2I_s], wsq_down [H,I_s], sws_down [H] (required iff S = 1);
- * x [T,H] bf16 (required iff S = 1).  H, I and I_s may not exceed 8192.  The row gather and prefill
- * segmentation do not apply to this call.  Errors as for moe_grouped_ffn; MOE_ERR_STATE if the context was
- * created for BF16 weights. */
+ * wsq_gate_up [2I_s,H], sws_gate_up [2I_s], wsq_down [H,I_s], sws_down [H] (required iff S = 1).
+ * H, I and I_s may not exceed 8192.  The row gather, prefill segmentation and moe_layer_host do not apply to
+ * an FP8 context.  Errors as for moe_grouped_ffn; MOE_ERR_STATE if the context was created for BF16 weights. */
 moe_status moe_grouped_ffn_fp8(moe_ctx* ctx, const void* wq_gate_up, const float* sw_gate_up, const void* wq_down,
-                               const float* sw_down, const void* x, const void* wsq_gate_up,
-                               const float* sws_gate_up, const void* wsq_down, const float* sws_down, int32_t T);
+                               const float* sw_down, const void* wsq_gate_up, const float* sws_gate_up,
+                               const void* wsq_down, const float* sws_down, int32_t T);
 
 /* Prefill segmentation.  A single P execution spans several D iterations, so the paper divides P into
  * segments delimited by backend-provided boundaries (Section "In-Place P/D Execution"; the span K of Section

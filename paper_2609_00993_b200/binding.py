@@ -93,7 +93,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_ctx_debug_ptrs_fp8.restype = i32
     lib.moe_ctx_debug_ptrs_fp8.argtypes = [vp] + [ctypes.POINTER(vp)] * 4
     lib.moe_grouped_ffn_fp8.restype = i32
-    lib.moe_grouped_ffn_fp8.argtypes = [vp] * 10 + [i32]
+    lib.moe_grouped_ffn_fp8.argtypes = [vp] * 9 + [i32]
     lib.moe_combine.restype = i32
     lib.moe_combine.argtypes = [vp, vp, vp, i32, vp]
     lib.moe_layer_host.restype = i32
@@ -252,7 +252,7 @@ class MoeContext:
         self._check(self.lib.moe_grouped_ffn(self.handle, _ptr(w_gate_up), _ptr(w_down), _ptr(x), _ptr(ws_gate_up),
                                              _ptr(ws_down), T))
 
-    def moe_grouped_ffn_fp8(self, wq_gate_up, sw_gate_up, wq_down, sw_down, x, wsq_gate_up=None, sws_gate_up=None,
+    def moe_grouped_ffn_fp8(self, wq_gate_up, sw_gate_up, wq_down, sw_down, wsq_gate_up=None, sws_gate_up=None,
                             wsq_down=None, sws_down=None, T=None):
         """wq_* are uint8 tensors of E4M3 codes, sw_* fp32 per-output-channel scales."""
         for n, t in (("wq_gate_up", wq_gate_up), ("wq_down", wq_down), ("wsq_gate_up", wsq_gate_up),
@@ -261,11 +261,11 @@ class MoeContext:
         for n, t in (("sw_gate_up", sw_gate_up), ("sw_down", sw_down), ("sws_gate_up", sws_gate_up),
                      ("sws_down", sws_down)):
             _dev(t, torch.float32, n)
-        _dev(x, torch.bfloat16, "x")
-        T = x.shape[0] if T is None else T
+        if T is None:
+            raise ValueError("T is required")
         self._check(self.lib.moe_grouped_ffn_fp8(self.handle, _ptr(wq_gate_up), _ptr(sw_gate_up), _ptr(wq_down),
-                                                 _ptr(sw_down), _ptr(x), _ptr(wsq_gate_up), _ptr(sws_gate_up),
-                                                 _ptr(wsq_down), _ptr(sws_down), T))
+                                                 _ptr(sw_down), _ptr(wsq_gate_up), _ptr(sws_gate_up), _ptr(wsq_down),
+                                                 _ptr(sws_down), T))
 
     def moe_combine(self, topk_w, inv_perm, out, T=None):
         _dev(topk_w, torch.float32, "topk_w"); _dev(inv_perm, torch.int32, "inv_perm"); _dev(out, torch.bfloat16, "out")
@@ -340,7 +340,7 @@ class MoeContext:
         self.moe_route(logits, select_bias, bufs["topk_idx"], bufs["topk_w"], T=T)
         self.moe_dispatch_layout(bufs["topk_idx"], x, bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"],
                                  T=T)
-        self.moe_grouped_ffn_fp8(w8["wq_gate_up"], w8["sw_gate_up"], w8["wq_down"], w8["sw_down"], x,
+        self.moe_grouped_ffn_fp8(w8["wq_gate_up"], w8["sw_gate_up"], w8["wq_down"], w8["sw_down"],
                                  w8.get("wsq_gate_up"), w8.get("sws_gate_up"), w8.get("wsq_down"), w8.get("sws_down"),
                                  T=T)
         self.moe_combine(bufs["topk_w"], bufs["inv_perm"], out, T=T)

@@ -42,8 +42,8 @@ struct BufferSet {
   float* sx;         // [N]
   char* aq;          // e4m3 [N,I]
   float* sa;         // [N]
-  char* xq_shared;   // e4m3 [T,H]
-  float* sx_shared;  // [T]
+  char* xq_tok;      // e4m3 [T,H]: x quantised in token order (the shared expert's GEMM1 input)
+  float* sx_tok;     // [T]
   char* aq_shared;   // e4m3 [T,Is]
   float* sa_shared;  // [T]
 };
@@ -87,8 +87,8 @@ size_t carve_set(const moe_config& c, char* base, BufferSet* out) {
   b.sx = reinterpret_cast<float*>(take(f8 * N * 4));
   b.aq = take(f8 * N * I);
   b.sa = reinterpret_cast<float*>(take(f8 * N * 4));
-  b.xq_shared = take(f8 * (c.n_shared ? T * H : 0));
-  b.sx_shared = reinterpret_cast<float*>(take(f8 * (c.n_shared ? T * 4 : 0)));
+  b.xq_tok = take(f8 * T * H);
+  b.sx_tok = reinterpret_cast<float*>(take(f8 * T * 4));
   b.aq_shared = take(f8 * T * Is);
   b.sa_shared = reinterpret_cast<float*>(take(f8 * (c.n_shared ? T * 4 : 0)));
   if (out) *out = b;
@@ -482,7 +482,17 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
     e = moe::launch_layout(topk_idx, (int64_t)T * ctx->cfg.top_k, ctx->cfg.n_experts, ctx->counts, ctx->offsets,
                            ctx->perm, ctx->inv_perm, b.scan, ctx->status, ctx->stream, &n);
   }
-  if (e == cudaSuccess && x != nullptr && !gathers_rows(ctx)) {
+  const bool fp8 = ctx->cfg.weight_format == MOE_WEIGHTS_FP8_E4M3;
+  if (e == cudaSuccess && x != nullptr && fp8) {
+    // FP8 variant: quantise each token row once, then move the codes (half the bytes) and the row scales
+    StageTimer tm(ctx, 8);
+    e = moe::launch_quantize_rows(x, T, ctx->cfg.hidden, b.xq_tok, b.sx_tok, ctx->stream, &n);
+  }
+  if (e == cudaSuccess && x != nullptr && fp8) {
+    StageTimer tm(ctx, 2);
+    e = moe::launch_permute(b.xq_tok, ctx->inv_perm, b.xq, T, ctx->cfg.top_k, ctx->cfg.hidden / 2, ctx->status,
+                            ctx->stream, &n, b.sx_tok, b.sx);
+  } else if (e == cudaSuccess && x != nullptr && !gathers_rows(ctx)) {
     StageTimer tm(ctx, 2);
     e = moe::launch_permute(x, ctx->inv_perm, b.x_perm, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->status, ctx->stream,
                             &n);
@@ -497,6 +507,8 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
 moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_down, const void* x,
                            const void* ws_gate_up, const void* ws_down, int32_t T) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->cfg.weight_format != MOE_WEIGHTS_BF16)
+    return fail(ctx, MOE_ERR_STATE, "the context was created for FP8 weights: call moe_grouped_ffn_fp8");
   if (ctx->state != ST_LAID_OUT)
     return fail(ctx, MOE_ERR_STATE, "moe_grouped_ffn needs a moe_dispatch_layout with x in the same step");
   if (T != ctx->T) return fail(ctx, MOE_ERR_INVALID_ARG, "T = %d differs from the layout's T = %d", T, ctx->T);
@@ -574,8 +586,8 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
 }
 
 moe_status moe_grouped_ffn_fp8(moe_ctx* ctx, const void* wq_gate_up, const float* sw_gate_up, const void* wq_down,
-                               const float* sw_down, const void* x, const void* wsq_gate_up,
-                               const float* sws_gate_up, const void* wsq_down, const float* sws_down, int32_t T) {
+                               const float* sw_down, const void* wsq_gate_up, const float* sws_gate_up,
+                               const void* wsq_down, const float* sws_down, int32_t T) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
   if (ctx->cfg.weight_format != MOE_WEIGHTS_FP8_E4M3)
     return fail(ctx, MOE_ERR_STATE, "the context was not created with weight_format = MOE_WEIGHTS_FP8_E4M3");
@@ -585,11 +597,10 @@ moe_status moe_grouped_ffn_fp8(moe_ctx* ctx, const void* wq_gate_up, const float
   if (!wq_gate_up || !sw_gate_up || !wq_down || !sw_down)
     return fail(ctx, MOE_ERR_INVALID_ARG, "routed weights or scales are NULL");
   const bool shared = ctx->cfg.n_shared != 0;
-  if (shared && (!wsq_gate_up || !sws_gate_up || !wsq_down || !sws_down || (!x && T > 0)))
-    return fail(ctx, MOE_ERR_INVALID_ARG, "the shared expert needs its weights, scales and x");
+  if (shared && (!wsq_gate_up || !sws_gate_up || !wsq_down || !sws_down))
+    return fail(ctx, MOE_ERR_INVALID_ARG, "the shared expert needs its weights and scales");
   if (misaligned(wq_gate_up) || misaligned(sw_gate_up) || misaligned(wq_down) || misaligned(sw_down) ||
-      misaligned(x) || misaligned(wsq_gate_up) || misaligned(sws_gate_up) || misaligned(wsq_down) ||
-      misaligned(sws_down))
+      misaligned(wsq_gate_up) || misaligned(sws_gate_up) || misaligned(wsq_down) || misaligned(sws_down))
     return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
   DeviceGuard guard(ctx->device);
   BufferSet& b = ctx->sets[ctx->cur];
@@ -598,20 +609,14 @@ moe_status moe_grouped_ffn_fp8(moe_ctx* ctx, const void* wq_gate_up, const float
   int n = 0;
   cudaError_t e = cudaSuccess;
   if (T > 0) {
-    // quantise -> GEMM1 + SwiGLU -> quantise -> GEMM2; the shared expert's passes ride in the routed launches
-    {
-      StageTimer tm(ctx, 8);
-      e = moe::launch_quantize_rows(b.x_perm, N, c.hidden, b.xq, b.sx, ctx->stream, &n);
-      if (e == cudaSuccess && shared)
-        e = moe::launch_quantize_rows(x, T, c.hidden, b.xq_shared, b.sx_shared, ctx->stream, &n);
-    }
+    // GEMM1 + SwiGLU on the rows moe_dispatch_layout quantised -> quantise the activation -> GEMM2; the shared
+    // expert's passes ride in the routed launches
     moe::GemmProblem g1{b.xq, wq_gate_up, b.act, ctx->offsets, 0, Ncap, N, c.n_experts, c.inter, c.hidden, true};
     g1.fp8 = true;
     g1.row_scale = b.sx;
     g1.w_scale = sw_gate_up;
-    moe::GemmDenseGroup s1{b.xq_shared, wsq_gate_up, b.act_shared, T, c.shared_inter, c.hidden, b.sx_shared,
-                           sws_gate_up};
-    if (e == cudaSuccess) {
+    moe::GemmDenseGroup s1{b.xq_tok, wsq_gate_up, b.act_shared, T, c.shared_inter, c.hidden, b.sx_tok, sws_gate_up};
+    {
       StageTimer tm(ctx, 3);
       e = run_gemm(ctx, g1, shared ? &s1 : nullptr, T, &n);
     }

@@ -35,8 +35,11 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
                           int* n_launches);
 
 // ---- a5 permute, a9 combine ----------------------------------------------------------------
+// H counts 2-byte columns (a row of H E4M3 codes is H/2 of them).  row_val / row_val_perm (optional): one fp32
+// value per source row is copied to each of its destination rows.
 cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm, int T, int k, int H, int* status,
-                           cudaStream_t stream, int* n_launches);
+                           cudaStream_t stream, int* n_launches, const float* row_val = nullptr,
+                           float* row_val_perm = nullptr);
 cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32_t* inv_perm, const float* topk_w,
                            void* out, int T, int k, int H, int* status, cudaStream_t stream, int* n_launches);
 

@@ -5,8 +5,8 @@
 //
 // The codes are integers decided by floating point, so every operation that decides them is spelled out in
 // IEEE fp32 (__fdiv_rn, cvt.rn.satfinite) and no fast-math substitute (reciprocal, fused scaling) is used.
-// One CTA of 128 threads per row; the row stays in registers between the two passes (rows of up to 8192
-// elements), so it is read once: 2 n bytes in, n + 4 bytes out per row.
+// One warp (rows of up to 2048 elements) or one CTA of 128 threads (up to 8192) per row; the row stays in
+// registers between the two passes, so it is read once: 2 n bytes in, n + 4 bytes out per row.
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
 
@@ -24,16 +24,24 @@ __device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
   return (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);  // lo in bits 0-7
 }
 
+// ROW_WARPS = 4: one CTA per row (rows of up to 8192 elements).  ROW_WARPS = 1: one warp per row, four rows per
+// CTA and no CTA-wide barrier (rows of up to 2048 elements).
+template <int ROW_WARPS>
 __global__ void __launch_bounds__(kQuantThreads)
-quantize_rows_kernel(const uint4* __restrict__ x, int n_vec, uint2* __restrict__ q, float* __restrict__ scale) {
+quantize_rows_kernel(const uint4* __restrict__ x, long long rows, int n_vec, uint2* __restrict__ q,
+                     float* __restrict__ scale) {
   __shared__ uint32_t warp_max[kQuantThreads / 32];
-  const int64_t row = blockIdx.x;
+  constexpr int kRowThreads = 32 * ROW_WARPS;
+  const int tid = ROW_WARPS == 1 ? (int)(threadIdx.x & 31) : (int)threadIdx.x;
+  const long long row = ROW_WARPS == 1 ? (long long)blockIdx.x * (kQuantThreads / 32) + (threadIdx.x >> 5)
+                                       : (long long)blockIdx.x;
+  if (ROW_WARPS == 1 && row >= rows) return;  // whole warps leave; there is no barrier on this path
   const uint4* xr = x + row * n_vec;
   uint4 v[kQuantMaxVecs];
   uint32_t m = 0;  // largest |bf16| as a bit pattern: for finite values the integer order is the value order
 #pragma unroll
   for (int j = 0; j < kQuantMaxVecs; ++j) {
-    const int i = threadIdx.x + j * kQuantThreads;
+    const int i = tid + j * kRowThreads;
     v[j] = i < n_vec ? xr[i] : make_uint4(0u, 0u, 0u, 0u);
     const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
 #pragma unroll
@@ -43,16 +51,18 @@ quantize_rows_kernel(const uint4* __restrict__ x, int n_vec, uint2* __restrict__
     }
   }
   m = __reduce_max_sync(0xffffffffu, m);
-  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
-  __syncthreads();
-  m = max(max(warp_max[0], warp_max[1]), max(warp_max[2], warp_max[3]));
+  if (ROW_WARPS > 1) {
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    m = max(max(warp_max[0], warp_max[1]), max(warp_max[2], warp_max[3]));
+  }
   const float amax = bf16_bits_to_f32(m);
   const float s = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
-  if (threadIdx.x == 0) scale[row] = s;
+  if (tid == 0) scale[row] = s;
   uint2* qr = q + row * n_vec;
 #pragma unroll
   for (int j = 0; j < kQuantMaxVecs; ++j) {
-    const int i = threadIdx.x + j * kQuantThreads;
+    const int i = tid + j * kRowThreads;
     if (i >= n_vec) continue;
     const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
     uint32_t pair[4];
@@ -69,8 +79,15 @@ cudaError_t launch_quantize_rows(const void* x, int64_t rows, int n, void* q, fl
                                  int* n_launches) {
   if (rows <= 0) return cudaSuccess;
   if (n <= 0 || n % 8 != 0 || n > 8 * kQuantThreads * kQuantMaxVecs || rows > 0x7fffffffLL) return cudaErrorNotSupported;
-  quantize_rows_kernel<<<(unsigned)rows, kQuantThreads, 0, stream>>>(static_cast<const uint4*>(x), n / 8,
-                                                                     static_cast<uint2*>(q), scale);
+  const int n_vec = n / 8;
+  if (n_vec <= 32 * kQuantMaxVecs) {
+    const long long blocks = (rows + kQuantThreads / 32 - 1) / (kQuantThreads / 32);
+    quantize_rows_kernel<1><<<(unsigned)blocks, kQuantThreads, 0, stream>>>(static_cast<const uint4*>(x), rows, n_vec,
+                                                                            static_cast<uint2*>(q), scale);
+  } else {
+    quantize_rows_kernel<4><<<(unsigned)rows, kQuantThreads, 0, stream>>>(static_cast<const uint4*>(x), rows, n_vec,
+                                                                          static_cast<uint2*>(q), scale);
+  }
   cudaError_t err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;

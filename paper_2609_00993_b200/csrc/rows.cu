@@ -75,11 +75,12 @@ constexpr int kPermuteSlots = 4;
 constexpr int kPermuteChunkCols = 4096;  // bf16 columns per item: at most 8 KB per slot
 
 // x_perm[inv_perm[t*k+j], c0:c1] = x[t, c0:c1] for j < k.  One warp per CTA; lane j stores destination j.
+// Optionally one fp32 value per row travels with it: row_val_perm[inv_perm[t*k+j]] = row_val[t].
 // dynamic shared memory: kPermuteSlots slots of slot_bytes | full[kPermuteSlots]
 __global__ void __launch_bounds__(32)
 permute_rows_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ inv_perm,
                     __nv_bfloat16* __restrict__ x_perm, int T, int k, int H, int col_blocks, int slot_bytes,
-                    int* status) {
+                    const float* __restrict__ row_val, float* __restrict__ row_val_perm, int* status) {
   extern __shared__ __align__(128) uint8_t smem[];
   const uint32_t slots = smem_u32(smem);
   const uint32_t bar_full = slots + (uint32_t)(kPermuteSlots * slot_bytes);
@@ -117,6 +118,7 @@ permute_rows_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restri
     if (!ok) break;
     if (dst_row >= 0) bulk_store(x_perm + (size_t)dst_row * H + c0, slots + s * (uint32_t)slot_bytes, bytes);
     bulk_commit();
+    if (row_val != nullptr && c0 == 0 && dst_row >= 0) row_val_perm[dst_row] = __ldg(row_val + t);
     // the slot used one item ago may be refilled once every lane's stores from it have read shared memory
     bulk_wait_read<1>();
     __syncwarp();
@@ -250,7 +252,7 @@ int resident_ctas(const void* kern, int threads, size_t smem) {
 }  // namespace
 
 cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm, int T, int k, int H, int* status,
-                           cudaStream_t stream, int* n_launches) {
+                           cudaStream_t stream, int* n_launches, const float* row_val, float* row_val_perm) {
   if (T <= 0) return cudaSuccess;
   if (k > 32) return cudaErrorNotSupported;  // one storing lane per destination
   const int col_blocks = (H + kPermuteChunkCols - 1) / kPermuteChunkCols;
@@ -263,7 +265,7 @@ cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm,
   const int grid = (int)(n_items < cap ? n_items : cap);
   permute_rows_kernel<<<grid, 32, smem, stream>>>(static_cast<const __nv_bfloat16*>(x), inv_perm,
                                                   static_cast<__nv_bfloat16*>(x_perm), T, k, H, col_blocks, slot_bytes,
-                                                  status);
+                                                  row_val, row_val_perm, status);
   err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;

@@ -1,7 +1,8 @@
 """FP8 (E4M3) precision variant against the oracle's statement of the same recipe.
 
 Stage by stage, so that every comparison is as tight as its arithmetic allows:
-  * the quantisation of the GEMM1 input rows is integer work decided in fp32: codes and scales bit-exact;
+  * the quantisation of the GEMM1 input rows (done per token, then moved) is integer work decided in fp32: codes
+    and scales of the permuted rows bit-exact;
   * GEMM1 + SwiGLU from identical codes: the bf16 activation within bf16 rounding of the oracle's;
   * the activation's quantisation, applied by the oracle to the GPU's own activation: bit-exact again;
   * GEMM2 from the GPU's own codes: within bf16 rounding of the oracle's fp64 sums;
@@ -29,11 +30,6 @@ def _w8_host(w8):
     return {k: (None if v is None else (_np_u8(v) if v.dtype == torch.uint8 else np_f32(v))) for k, v in w8.items()}
 
 
-def _ws_view(ctx, ptr_name, shape, dtype):
-    """A view of one of the context's FP8 buffers (test inspection only)."""
-    return ctx.fp8_debug_view(ptr_name, shape, dtype)
-
-
 CASES = [
     # T, H, E, k, I, shared_I, phase, variant
     (64, 256, 8, 2, 512, 0, B.MOE_PHASE_PREFILL, B.MOE_GEMM_AUTO),      # the smallest config's shape
@@ -47,14 +43,10 @@ CASES = [
 def test_fp8_stages_against_the_oracle(T, H, E, k, I, shared_I, phase, variant):
     shape = wl.LayerShape("f8", T=T, H=H, E=E, k=k, I=I, shared_I=shared_I, select_bias=True)
     # weights ~ N(0, 1/sqrt(fan_in)): unit-variance pre-activations, so that an error anywhere is visible
-    w8_1 = wl.make_weights_fp8(shape, 11, DEV, std=1.0)
-    for name in ("sw_gate_up", "sws_gate_up"):
-        if w8_1[name] is not None:
-            w8_1[name] = (w8_1[name] / H ** 0.5).contiguous()
-    for name, fan in (("sw_down", I), ("sws_down", shared_I)):
-        if w8_1[name] is not None:
-            w8_1[name] = (w8_1[name] / fan ** 0.5).contiguous()
-    w8 = w8_1
+    w8 = wl.make_weights_fp8(shape, 11, DEV, std=1.0)
+    for name, fan in (("sw_gate_up", H), ("sws_gate_up", H), ("sw_down", I), ("sws_down", shared_I)):
+        if w8[name] is not None:
+            w8[name] = (w8[name] / fan ** 0.5).contiguous()
     a = wl.make_activations(shape, 12, DEV)
     ctx = B.MoeContext(B.make_config(H, E, k, I, shared_I, T, phase, 0, variant, weight_format=B.MOE_WEIGHTS_FP8_E4M3))
     torch.cuda.synchronize()
@@ -63,7 +55,7 @@ def test_fp8_stages_against_the_oracle(T, H, E, k, I, shared_I, phase, variant):
     assert ctx.moe_ctx_status() == B.MOE_OK
     N = T * k
     dbg = ctx.moe_ctx_debug_ptrs()
-    x_perm = wl.bits(dbg["x_perm"][:N])
+    x_perm = oracle.permute(wl.bits(a["x"]), np_i32(bufs["perm"]).reshape(-1), k)  # an FP8 context keeps no bf16 copy
     act_gpu = wl.bits(dbg["act"][:N])
     y_gpu = np_f32(dbg["y_perm"][:N])
     xq_gpu, sx_gpu = _np_u8(ctx.fp8_debug_view("xq", (N, H), torch.uint8)), np_f32(ctx.fp8_debug_view("sx", (N,), torch.float32))
