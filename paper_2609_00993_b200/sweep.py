@@ -2,7 +2,7 @@
 T in {1, 16, 128, 1024, 8192, 32768}.  For every T: layer time and tokens/s, per-stage device times, expert
 load imbalance, and the fraction of the layer's roofline floor that was reached.
 
-    python -m paper_2609_00993_b200.sweep [--tokens 1 16 128 ...] [--iters-min-ms 300]
+    python -m paper_2609_00993_b200.sweep [--tokens 1 16 128 ...] [--iters-min-ms 300] [--fp8]
 
 One JSON object per T on stdout.  The floor of a step is the sum over its stages of
 max(flops / tensor peak, algorithmic bytes / HBM peak); for the grouped GEMMs it is summed per expert
@@ -32,39 +32,49 @@ def load_peaks():
     return 6650.0, 1400.0, "fallback"
 
 
-def layer_floor_us(shape, counts, hbm_gbs, tflops):
-    """Roofline floor of one step in microseconds, and its tensor-only / bytes-only parts."""
+def layer_floor_us(shape, counts, hbm_gbs, tflops, fp8=False):
+    """Roofline floor of one step in microseconds, and its tensor-only / bytes-only parts.  FP8: one byte per
+    weight and per GEMM input element, and twice the bf16 tensor peak (the nominal fp8 : bf16 ratio)."""
     H, I, k, T = shape.H, shape.I, shape.k, shape.T
-    bw, peak = hbm_gbs * 1e9, tflops * 1e12
+    bw, peak = hbm_gbs * 1e9, tflops * 1e12 * (2.0 if fp8 else 1.0)
+    eb = 1.0 if fp8 else 2.0  # bytes per operand element
     gemm = fl_only = by_only = 0.0
     groups = [(int(c), I) for c in counts.tolist() if c > 0]
     if shape.shared_I:
         groups.append((T, shape.shared_I))
     for rows, inter in groups:
         flops = 6.0 * rows * H * inter
-        bytes_ = 6.0 * H * inter + 2.0 * rows * H + 4.0 * rows * inter + 2.0 * rows * H  # weights, in, act w+r, out
+        # weights, rows in, act written (bf16) and read (FP8: re-quantised: bf16 read + codes written + codes read), out
+        act = (2.0 + 2.0 + 1.0 + 1.0) * rows * inter if fp8 else 4.0 * rows * inter
+        bytes_ = 3.0 * eb * H * inter + eb * rows * H + act + 2.0 * rows * H
         gemm += max(flops / peak, bytes_ / bw)
         fl_only += flops / peak
         by_only += bytes_ / bw
     N = T * k
-    rows_bytes = (2.0 * T * H + 2.0 * N * H + 4.0 * N) + (2.0 * N * H + 2.0 * bool(shape.shared_I) * T * H + 8.0 * N + 2.0 * T * H)
+    rows_in = (2.0 * T * H + 1.0 * T * H) + (1.0 * T * H + 1.0 * N * H + 8.0 * N) if fp8 else 2.0 * T * H + 2.0 * N * H + 4.0 * N
+    rows_bytes = rows_in + (2.0 * N * H + 2.0 * bool(shape.shared_I) * T * H + 8.0 * N + 2.0 * T * H)
     route_bytes = 4.0 * T * shape.E + 8.0 * N + 12.0 * N
     other = (rows_bytes + route_bytes) / bw
     return 1e6 * (gemm + other), 1e6 * fl_only, 1e6 * by_only
 
 
-def run_one(shape, weights, min_ms, dev="cuda"):
+def run_one(shape, weights, min_ms, dev="cuda", fp8=False):
     phase = B.MOE_PHASE_DECODE if shape.T <= 256 else B.MOE_PHASE_PREFILL
     stream = torch.cuda.Stream()
-    ctx = B.MoeContext(B.make_config(shape.H, shape.E, shape.k, shape.I, shape.shared_I, shape.T, phase), stream=stream)
+    fmt = B.MOE_WEIGHTS_FP8_E4M3 if fp8 else B.MOE_WEIGHTS_BF16
+    ctx = B.MoeContext(B.make_config(shape.H, shape.E, shape.k, shape.I, shape.shared_I, shape.T, phase,
+                                     weight_format=fmt), stream=stream)
     acts = [wl.make_activations(shape, 600 + i, dev) for i in range(3)]
     bufs = B.alloc_step_buffers(shape.T, shape.k, shape.E, dev)
     out = torch.empty(shape.T, shape.H, dtype=torch.bfloat16, device=dev)
-    wargs = (weights["w_gate_up"], weights["w_down"], weights["ws_gate_up"], weights["ws_down"])
 
     def step(i):
         a = acts[i % 3]
-        ctx.layer(a["x"], a["logits"], a["bias"], *wargs, out=out, bufs=bufs)
+        if fp8:
+            ctx.layer_fp8(a["x"], a["logits"], a["bias"], weights, out=out, bufs=bufs)
+        else:
+            ctx.layer(a["x"], a["logits"], a["bias"], weights["w_gate_up"], weights["w_down"], weights["ws_gate_up"],
+                      weights["ws_down"], out=out, bufs=bufs)
 
     torch.cuda.synchronize()
     with torch.cuda.stream(stream):
@@ -103,20 +113,21 @@ def main():
     ap.add_argument("--iters-min-ms", type=float, default=300.0, help="time each T for at least this long")
     ap.add_argument("--experts", type=int, default=wl.C5.E,
                     help="number of routed experts (fewer than 256 keeps the weights small enough for a profiler capture)")
+    ap.add_argument("--fp8", action="store_true", help="the FP8 (E4M3) precision variant instead of bf16")
     args = ap.parse_args()
     B.load_library()
     hbm, tfl, src = load_peaks()
     import dataclasses
     base = dataclasses.replace(wl.C5, E=args.experts)
-    weights = wl.make_weights(base, 2, "cuda")
+    weights = (wl.make_weights_fp8 if args.fp8 else wl.make_weights)(base, 2, "cuda")
     for T in args.tokens:
         shape = base.with_tokens(T)
-        step_us, n, stages, counts = run_one(shape, weights, args.iters_min_ms)
-        floor_us, fl_us, by_us = layer_floor_us(shape, counts, hbm, tfl)
+        step_us, n, stages, counts = run_one(shape, weights, args.iters_min_ms, fp8=args.fp8)
+        floor_us, fl_us, by_us = layer_floor_us(shape, counts, hbm, tfl, fp8=args.fp8)
         cf = counts.double()
         nz = int((counts > 0).sum())
         print(json.dumps({
-            "workload": f"C5 zipf(1.2) E={shape.E} T={T}", "phase": "decode" if T <= 256 else "prefill", "iters": n,
+            "workload": f"C5 zipf(1.2) E={shape.E} T={T}" + (" fp8" if args.fp8 else ""), "phase": "decode" if T <= 256 else "prefill", "iters": n,
             "step_us": round(step_us, 1), "tokens_per_s": round(T / (step_us * 1e-6), 1),
             "roofline_floor_us": round(floor_us, 1), "frac_of_roofline": round(floor_us / step_us, 3),
             "floor_tensor_only_us": round(fl_us, 1), "floor_bytes_only_us": round(by_us, 1),
