@@ -14,6 +14,9 @@
 //   small-M (decode)   swap-AB: 128 weight rows fill M, the expert's tokens sit in N (16..128, chosen per
 //                      tile from the expert's row count), two MMAs per 16 K-elements (one per weight box).
 //                      Each weight byte is read once: the variant is HBM-bound by design.
+// Both variants also exist for E4M3 operands (the FP8 precision variant): the same pipeline with 128 K-elements
+// per stage row, tcgen05.mma.kind::f8f6f4 (32 K-elements per instruction) and an epilogue that multiplies the
+// accumulator by the row's and the weight row's scale before SwiGLU / the bf16 store.
 // An expert's row tile may run past the end of its segment: TMA needs no alignment on the row coordinate, so
 // segments are NOT padded; rows that belong to the next expert are computed and simply not stored.
 //
