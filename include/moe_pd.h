@@ -183,7 +183,7 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
  *   weights      wq_* hold E4M3 codes, sw_* one fp32 scale per output channel (weight row):
  *                W[e,r,:] = sw[e,r] * decode(wq[e,r,:])
  *   activations  every bf16 row v entering a GEMM is quantised on the fly, per row:
- *                scale = max|v| / 448 (1 for an all-zero row), code_i = e4m3(v_i / scale), both divisions in
+ *                amax = max(max|v|, 2^-100), scale = amax / 448, code_i = e4m3(v_i * (448 / amax)), all in
  *                IEEE fp32, conversion round-to-nearest-even saturating at +-448
  *   GEMM1        g, u = (sum_h x_code * w_code) * scale_x[p] * sw[e,row], act = silu(g) * u stored as bf16
  *   GEMM2        act is quantised per row as above; y = (sum_i a_code * w_code) * scale_a[p] * sw[e,c], bf16

@@ -352,10 +352,11 @@ int oracle_layer_tokens(const uint16_t* x, const int32_t* topk_idx, const float*
  *   weights    given as E4M3 codes with one fp32 scale per output channel
  *              (per weight row): W[r,:] = scale_w[r] * decode(code[r,:]).
  *   activation a bf16 row v[0..n) entering a GEMM is quantised per row:
- *                amax  = max_i |v_i|                         (fp32)
- *                scale = amax / 448   (one fp32 division; 1 if amax == 0)
- *                code_i = e4m3( v_i / scale )  (fp32 division, then round to
- *                         nearest even, saturating at +-448)
+ *                amax  = max( max_i |v_i|, 2^-100 )          (fp32; the floor
+ *                        keeps an all-zero row finite: its codes are 0)
+ *                scale = amax / 448,  inv = 448 / amax       (fp32 divisions)
+ *                code_i = e4m3( v_i * inv )  (one fp32 multiply, then round
+ *                         to nearest even, saturating at +-448)
  *   GEMM1      g_i = (sum_h dq_x[h] * dq_wg[i,h]) * scale_x * scale_w[i],
  *              u_i likewise with the up row, a_i = silu(g_i) * u_i,
  *              a stored as bf16 (round to nearest even)
@@ -412,9 +413,10 @@ int oracle_quantize_rows(const uint16_t* x, int64_t M, int32_t n, uint8_t* q, fl
       float a = fabsf(bf16_to_f32(x[r * n + i]));
       if (a > amax) amax = a;
     }
-    float s = amax > 0.0f ? amax / 448.0f : 1.0f;
-    scale[r] = s;
-    for (int32_t i = 0; i < n; ++i) q[r * n + i] = f32_to_e4m3(bf16_to_f32(x[r * n + i]) / s);
+    if (amax < 0x1p-100f) amax = 0x1p-100f;
+    float inv = 448.0f / amax;
+    scale[r] = amax / 448.0f;
+    for (int32_t i = 0; i < n; ++i) q[r * n + i] = f32_to_e4m3(bf16_to_f32(x[r * n + i]) * inv);
   }
   return ORACLE_OK;
 }

@@ -1,10 +1,11 @@
 // FP8 precision variant: per-row dynamic quantisation of bf16 activation rows to E4M3.
 //
-//   amax  = max_i |v_i|                    scale = amax / 448   (1 when the row is all zero)
-//   code_i = e4m3(v_i / scale)             round to nearest even, saturating at +-448
+//   amax  = max(max_i |v_i|, 2^-100)       scale = amax / 448,  inv = 448 / amax
+//   code_i = e4m3(v_i * inv)               round to nearest even, saturating at +-448
 //
 // The codes are integers decided by floating point, so every operation that decides them is spelled out in
-// IEEE fp32 (__fdiv_rn, cvt.rn.satfinite) and no fast-math substitute (reciprocal, fused scaling) is used.
+// IEEE fp32 (__fdiv_rn once per row, __fmul_rn per element, cvt.rn.satfinite) and nothing is contracted or
+// approximated.
 // One warp (rows of up to 2048 elements) or one CTA of 128 threads (up to 8192) per row; the row stays in
 // registers between the two passes, so it is read once: 2 n bytes in, n + 4 bytes out per row.
 #include <cuda_bf16.h>
@@ -56,9 +57,9 @@ quantize_rows_kernel(const uint4* __restrict__ x, long long rows, int n_vec, uin
     __syncthreads();
     m = max(max(warp_max[0], warp_max[1]), max(warp_max[2], warp_max[3]));
   }
-  const float amax = bf16_bits_to_f32(m);
-  const float s = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
-  if (tid == 0) scale[row] = s;
+  const float amax = fmaxf(bf16_bits_to_f32(m), 0x1p-100f);
+  const float inv = __fdiv_rn(448.f, amax);
+  if (tid == 0) scale[row] = __fdiv_rn(amax, 448.f);
   uint2* qr = q + row * n_vec;
 #pragma unroll
   for (int j = 0; j < kQuantMaxVecs; ++j) {
@@ -68,7 +69,7 @@ quantize_rows_kernel(const uint4* __restrict__ x, long long rows, int n_vec, uin
     uint32_t pair[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c)
-      pair[c] = e4m3x2(__fdiv_rn(bf16_bits_to_f32(w[c] & 0xffffu), s), __fdiv_rn(bf16_bits_to_f32(w[c] >> 16), s));
+      pair[c] = e4m3x2(__fmul_rn(bf16_bits_to_f32(w[c] & 0xffffu), inv), __fmul_rn(bf16_bits_to_f32(w[c] >> 16), inv));
     qr[i] = make_uint2(pair[0] | (pair[1] << 16), pair[2] | (pair[3] << 16));
   }
 }

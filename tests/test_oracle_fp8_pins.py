@@ -63,7 +63,7 @@ def test_quantize_rows_scale_codes_and_error_bound():
     xv = oracle.bf16_to_f32(bits)
     q, s = oracle.quantize_rows(bits)
     amax = np.abs(xv).max(axis=1)
-    assert s[5] == 1.0 and np.all(q[5] == 0)
+    assert s[5] == np.float32(2.0 ** -100) / np.float32(448.0) and np.all(q[5] == 0)  # the floor of amax
     nzr = amax > 0
     assert np.array_equal(s[nzr], (amax[nzr] / np.float32(448.0)).astype(np.float32))
     dq = oracle.e4m3_decode(q).astype(np.float64)
