@@ -3,8 +3,9 @@
 //   operands   bf16, K-major, staged in shared memory by TMA (128-byte swizzle), 64 K-elements per stage
 //   math       tcgen05.mma (kind::f16, M=128) issued by one thread, fp32 accumulators in TMEM
 //   epilogue   tcgen05.ld -> registers -> (SwiGLU) -> bf16 -> a per-warp swizzled staging tile in shared
-//              memory -> full-line global stores; the accumulator stage is handed back as soon as it has
-//              been read, so the next tile's MMAs overlap the stores (two TMEM accumulator stages)
+//              memory -> tiled bulk stores (TMA) of 32-row x 64-feature boxes; the accumulator stage is handed
+//              back as soon as it has been read, so the next tile's MMAs overlap the stores (two TMEM
+//              accumulator stages)
 //   schedule   persistent CTAs walk the tile list (expert, row tile, feature tile); the list is derived
 //              on the device from the expert offsets, so no host synchronisation is needed
 //
@@ -209,6 +210,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Output tensor maps (large-M epilogue): [rows, n_feat] bf16 with boxes of 64 features x 32 rows, 128-byte swizzle
+struct OutMaps {
+  CUtensorMap o, o2;
+};
+// Tiled bulk store shared -> global of one box, tracked in the issuing thread's bulk groups
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src_smem, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src_smem),
+               "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all of this thread's bulk stores have read their shared-memory source / have completed
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // 16-byte asynchronous copy global -> shared (generic proxy), grouped per thread
 __device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
@@ -301,7 +317,7 @@ template <bool SWAP, bool GATED, bool GATHER, bool FP8>
 __global__ void __launch_bounds__(GATHER ? kThreadsGather : kThreads, 1)
 grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
                        const __grid_constant__ CUtensorMap map_x2, const __grid_constant__ CUtensorMap map_w2,
-                       const __grid_constant__ TcParams p) {
+                       const __grid_constant__ OutMaps omaps, const __grid_constant__ TcParams p) {
   static_assert(!(GATHER && FP8), "the row gather exists for bf16 operands only");
   constexpr int kbk = FP8 ? 2 * kBlockK : kBlockK;  // K elements per stage
   extern __shared__ uint8_t smem_raw[];
@@ -568,9 +584,10 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         }
       } else {
         // lane = token row, column = output feature.  Two 32-column chunks (128 bytes of a row) at a time go
-        // through a per-warp staging tile in shared memory (16-byte pieces XOR-swizzled by row, conflict-free
-        // both ways), so that every global store instruction writes four whole 128-byte lines instead of
-        // touching 32 different rows.
+        // through a per-warp staging tile in shared memory whose 16-byte pieces are XOR-swizzled by row: that
+        // is conflict-free both ways and it is TMA's 128-byte swizzle, so a warp whose 32 rows are all valid
+        // sends the 4 KB box with one tiled bulk store.  A ragged warp (the expert's last rows) stores by hand,
+        // every store instruction writing four whole 128-byte lines.
         constexpr int kPairs = kFeatPerTile / 64;
         uint8_t* stage_tile = epi_smem + warp * 4096;  // 32 rows x 128 bytes
         const int rows_here = t.rows - warp * 32;       // rows of this warp's 32 that are valid (may be <= 0)
@@ -630,10 +647,24 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
               release_acc();  // the accumulator has been read completely: hand it back before the stores go out
               released = true;
             }
+            if (h == 0) {  // the previous tiled store (lane 0's) has read the staging tile
+              if (lane == 0) bulk_wait_read_all();
+              __syncwarp();
+            }
 #pragma unroll
             for (int j = 0; j < 4; ++j)
               *reinterpret_cast<uint4*>(stage_tile + lane * 128 + (((h * 4 + j) ^ (lane & 7)) << 4)) =
                   make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+          }
+          if (rows_here >= 32 && f0 + 64 <= n_feat) {
+            // a full 32-row x 64-feature box: one tiled bulk store (the staging layout is the 128-byte swizzle)
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(t.dense ? &omaps.o2 : &omaps.o, smem_u32(stage_tile), f0, t.row0 + warp * 32);
+              bulk_commit();
+            }
+            continue;
           }
           __syncwarp();
 #pragma unroll
@@ -652,6 +683,7 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       *abort_flag = 1;
       atomicCAS(p.status, kStOk, kStTimeout);
     }
+    if (!SWAP && lane == 0) bulk_wait_all();  // the tiled stores are complete before the staging tiles are given up
   }
 
   // ---- teardown
@@ -698,11 +730,11 @@ bool encode_map(CUtensorMap* map, const void* base, int rank, const uint64_t* di
 
 template <typename Kernel>
 cudaError_t launch_variant(Kernel kern, int threads, const CUtensorMap& mx, const CUtensorMap& mw,
-                           const CUtensorMap& mx2, const CUtensorMap& mw2, const TcParams& prm, int grid, size_t smem,
-                           cudaStream_t stream) {
+                           const CUtensorMap& mx2, const CUtensorMap& mw2, const OutMaps& om, const TcParams& prm,
+                           int grid, size_t smem, cudaStream_t stream) {
   cudaError_t err = ensure_dynamic_smem(kern, smem);
   if (err != cudaSuccess) return err;
-  kern<<<grid, threads, smem, stream>>>(mx, mw, mx2, mw2, prm);
+  kern<<<grid, threads, smem, stream>>>(mx, mw, mx2, mw2, om, prm);
   return cudaGetLastError();
 }
 
@@ -779,6 +811,20 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
     const uint32_t bw[3] = {box_k, (uint32_t)kWBoxRows, 1u};
     if (!encode_map(&mw2, dense->W, 3, dw, sw, bw, fp8)) return cudaErrorInvalidValue;
   }
+  OutMaps om;
+  {
+    const uint64_t d[2] = {(uint64_t)p.n_feat, (uint64_t)p.rows_cap};
+    const uint64_t st[1] = {(uint64_t)p.n_feat * 2};
+    const uint32_t bx[2] = {(uint32_t)(p.n_feat < 64 ? p.n_feat : 64), 32u};
+    if (!encode_map(&om.o, p.out, 2, d, st, bx)) return cudaErrorInvalidValue;
+    om.o2 = om.o;
+    if (dense != nullptr) {
+      const uint64_t d2[2] = {(uint64_t)dense->n_feat, (uint64_t)dense->rows};
+      const uint64_t st2[1] = {(uint64_t)dense->n_feat * 2};
+      const uint32_t bx2[2] = {(uint32_t)(dense->n_feat < 64 ? dense->n_feat : 64), 32u};
+      if (!encode_map(&om.o2, dense->out, 2, d2, st2, bx2)) return cudaErrorInvalidValue;
+    }
+  }
   TcParams prm;
   prm.gather_src = static_cast<const __nv_bfloat16*>(p.gather_src);
   prm.gather_src2 = dense ? static_cast<const __nv_bfloat16*>(dense->A) : nullptr;
@@ -823,19 +869,19 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
   if (grid < 1) grid = 1;
   cudaError_t err;
   if (gather)
-    err = launch_variant(grouped_gemm_tc_kernel<false, true, true, false>, kThreadsGather, mx, mw, mx2, mw2, prm, grid, smem, stream);
+    err = launch_variant(grouped_gemm_tc_kernel<false, true, true, false>, kThreadsGather, mx, mw, mx2, mw2, om, prm, grid, smem, stream);
   else if (fp8 && swap_ab)
-    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true, false, true>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
-                  : launch_variant(grouped_gemm_tc_kernel<true, false, false, true>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true, false, true>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream)
+                  : launch_variant(grouped_gemm_tc_kernel<true, false, false, true>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream);
   else if (fp8)
-    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true, false, true>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
-                  : launch_variant(grouped_gemm_tc_kernel<false, false, false, true>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true, false, true>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream)
+                  : launch_variant(grouped_gemm_tc_kernel<false, false, false, true>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream);
   else if (swap_ab)
-    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
-                  : launch_variant(grouped_gemm_tc_kernel<true, false, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, true, false, false>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream)
+                  : launch_variant(grouped_gemm_tc_kernel<true, false, false, false>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream);
   else
-    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream)
-                  : launch_variant(grouped_gemm_tc_kernel<false, false, false, false>, kThreads, mx, mw, mx2, mw2, prm, grid, smem, stream);
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<false, true, false, false>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream)
+                  : launch_variant(grouped_gemm_tc_kernel<false, false, false, false>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream);
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }
