@@ -112,3 +112,36 @@ def test_fp8_call_is_refused_on_a_bf16_context_and_the_other_way_round():
     with pytest.raises(B.MoeError):  # the CUDA-core check kernel has no FP8 form
         B.MoeContext(B.make_config(256, 8, 2, 128, 0, 32, gemm_variant=B.MOE_GEMM_VALIDATION,
                                    weight_format=B.MOE_WEIGHTS_FP8_E4M3))
+
+
+def test_fp8_decode_step_replays_from_a_cuda_graph_and_is_run_to_run_identical():
+    shape = wl.LayerShape("f8", T=48, H=512, E=16, k=4, I=256, shared_I=128, select_bias=True)
+    w8 = wl.make_weights_fp8(shape, 1, DEV)
+    a1, a2 = wl.make_activations(shape, 2, DEV), wl.make_activations(shape, 3, DEV)
+    sd = torch.cuda.Stream()
+    d = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 48, B.MOE_PHASE_DECODE,
+                                   weight_format=B.MOE_WEIGHTS_FP8_E4M3), stream=sd)
+    torch.cuda.synchronize()
+    eager1, _ = d.layer_fp8(a1["x"], a1["logits"], a1["bias"], w8)
+    eager2, _ = d.layer_fp8(a2["x"], a2["logits"], a2["bias"], w8)
+    again1, _ = d.layer_fp8(a1["x"], a1["logits"], a1["bias"], w8)   # the other buffer set, same bits
+    torch.cuda.synchronize()
+    assert torch.equal(again1, eager1)
+    x, logits, bias = a1["x"].clone(), a1["logits"].clone(), a1["bias"].clone()
+    bufs = B.alloc_step_buffers(48, 4, 16, DEV)
+    out = torch.empty(48, 512, dtype=torch.bfloat16, device=DEV)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=sd):
+        d.layer_fp8(x, logits, bias, w8, out=out, bufs=bufs)
+    out.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager1)
+    x.copy_(a2["x"]); logits.copy_(a2["logits"]); bias.copy_(a2["bias"])
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager2)
+    assert d.moe_ctx_status() == B.MOE_OK
+    del g
+    d.close()
