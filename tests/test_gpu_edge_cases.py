@@ -44,6 +44,8 @@ def _check(out, ref, label):
     (300, 128, 1, 1, 192, 0),    # a single expert: the layer is a dense MLP
     (129, 192, 3, 2, 320, 64),   # one row past a tile boundary; H, I not powers of two
     (200, 2560, 512, 8, 256, 0), # the paper's model shape: hidden 2,560, 512 routed experts, top-8 (I is not stated there)
+    (70, 128, 1024, 32, 64, 0),  # the largest E and k the library accepts (single-CTA layout)
+    (600, 128, 1024, 32, 64, 64),  # the same with 19200 routed rows: the multi-CTA layout with E = 1024
 ])
 def test_small_and_degenerate_shapes(phase, pname, T, H, E, k, I, shared_I):
     shape = wl.LayerShape("t", T=T, H=H, E=E, k=k, I=I, shared_I=shared_I, select_bias=True)
