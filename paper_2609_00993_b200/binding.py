@@ -298,7 +298,8 @@ class MoeContext:
             off = p.value - base
             return self.workspace[off:off + rows * cols * esz].view(dtype).view(rows, cols)
 
-        return {"x_perm": view(ptrs[0], N, c.hidden, torch.bfloat16), "act": view(ptrs[1], N, c.inter, torch.bfloat16),
+        fp8 = c.weight_format == MOE_WEIGHTS_FP8_E4M3  # such a context keeps no bf16 x_perm
+        return {"x_perm": None if fp8 else view(ptrs[0], N, c.hidden, torch.bfloat16), "act": view(ptrs[1], N, c.inter, torch.bfloat16),
                 "y_perm": view(ptrs[2], N, c.hidden, torch.bfloat16),
                 "y_shared": view(ptrs[3], c.max_tokens, c.hidden, torch.bfloat16) if c.n_shared else None,
                 "counts": view(ptrs[4], 1, c.n_experts, torch.int32), "offsets": view(ptrs[5], 1, c.n_experts + 1, torch.int32)}

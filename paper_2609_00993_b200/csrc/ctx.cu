@@ -66,8 +66,9 @@ size_t carve_set(const moe_config& c, char* base, BufferSet* out) {
     off += align_up(bytes ? bytes : 1, 256);
     return p;
   };
+  const size_t f8 = c.weight_format == MOE_WEIGHTS_FP8_E4M3 ? 1 : 0;
   BufferSet b;
-  b.x_perm = take(N * H * 2);
+  b.x_perm = take(f8 ? 0 : N * H * 2);  // an FP8 context moves quantised rows (xq) instead
   b.act = take(N * I * 2);
   b.y_perm = take(N * H * 2);
   b.act_shared = take(T * Is * 2);
@@ -82,7 +83,6 @@ size_t carve_set(const moe_config& c, char* base, BufferSet* out) {
   b.x_stage = take(T * H * 2);
   b.out_stage = take(T * H * 2);
   b.scan = reinterpret_cast<int32_t*>(take(moe::layout_scratch_ints((int64_t)N, (int)E) * 4));
-  const size_t f8 = c.weight_format == MOE_WEIGHTS_FP8_E4M3 ? 1 : 0;
   b.xq = take(f8 * N * H);
   b.sx = reinterpret_cast<float*>(take(f8 * N * 4));
   b.aq = take(f8 * N * I);
