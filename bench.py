@@ -554,15 +554,27 @@ def run_ours(args):
                "note": "W8A8: E4M3 weights with per-output-channel scales, bf16 rows quantised per row on the fly, "
                        "tcgen05 kind::f8f6f4; not the headline (the metric is quoted on bf16)"}
 
-    # ---- end to end: host buffers in, host buffer out, copies inside the timed region
-    e2e_value = None
+    # ---- end to end: pinned host buffers in, pinned host buffer out, every copy inside the timed region.
+    # Public API: moe_layer_host_submit / moe_layer_host_wait, four slots, so that the copies of one step overlap
+    # the kernels of its neighbours; the synchronous moe_layer_host (copy, compute, copy, sync) is timed beside it.
+    e2e_value = e2e_sync_value = None
     if not args.quick:
         hx = [a["x"].cpu().pin_memory() for a in acts]
         hl = [a["logits"].cpu().pin_memory() for a in acts]
-        hout = torch.empty(T, H, dtype=torch.bfloat16).pin_memory()
 
         def host_step(i):
-            ctx.moe_layer_host(hl[i % n_in], None, hx[i % n_in], *wargs, hout)
+            ctx.moe_layer_host(hl[i % n_in], None, hx[i % n_in], *wargs, hout[0])
+
+        n_slots = 4
+        hout = [torch.empty(T, H, dtype=torch.bfloat16).pin_memory() for _ in range(n_slots)]
+
+        def run_pipelined(n):
+            for i in range(n):
+                if i >= n_slots:
+                    ctx.moe_layer_host_wait(i % n_slots)
+                ctx.moe_layer_host_submit(i % n_slots, hl[i % n_in], None, hx[i % n_in], *wargs, hout[i % n_slots])
+            for sl in range(n_slots):
+                ctx.moe_layer_host_wait(sl)
 
         for i in range(max(3, args.warmup)):
             host_step(i)
@@ -571,8 +583,13 @@ def run_ours(args):
         for i in range(args.steps):
             host_step(i)
         torch.cuda.synchronize(dev)
-        e2e_s = max_over_ranks(time.perf_counter() - t0, dist, dev)
-        e2e_value = whole_job_rate(T * args.steps, world, e2e_s)
+        e2e_sync_value = whole_job_rate(T * args.steps, world, max_over_ranks(time.perf_counter() - t0, dist, dev))
+        run_pipelined(max(4, args.warmup))
+        barrier()
+        t0 = time.perf_counter()
+        run_pipelined(args.steps)
+        torch.cuda.synchronize(dev)
+        e2e_value = whole_job_rate(T * args.steps, world, max_over_ranks(time.perf_counter() - t0, dist, dev))
     assert ctx.moe_ctx_status() == B.MOE_OK
 
     if rank != 0:
@@ -631,7 +648,9 @@ def run_ours(args):
                        "l2": "inputs larger than L2: 1.2 GB of weights streamed per step, 4 rotating input batches",
                        "parallelism": f"replicas x{world} (no data-path collective)"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": T * E * 4 + T * H * 2,
-                    "d2h_bytes_per_step": T * H * 2},
+                    "d2h_bytes_per_step": T * H * 2,
+                    "api": "moe_layer_host_submit / moe_layer_host_wait, four slots in rotation (copies overlap kernels)",
+                    "synchronous_moe_layer_host": e2e_sync_value},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu_baseline,
             "stages": stages, "fused_row_gather": fused, "fp8_variant": fp8}
     ctx.close()

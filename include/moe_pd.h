@@ -14,10 +14,10 @@
  * Conventions for every call
  *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned,
  *     dense row-major.  The library never frees or keeps them beyond the stream work
- *     of the step they belong to.  Only `moe_layer_host` takes HOST pointers, and says so.
+ *     of the step they belong to.  Only `moe_layer_host` and `moe_layer_host_submit` take HOST pointers.
  *   - Calls validate on the host, enqueue kernels on the context's stream and return.
  *     They do not synchronise, allocate device memory or read device memory back
- *     (except `moe_ctx_status`, `moe_ctx_destroy` and `moe_layer_host`, which say so).
+ *     (except `moe_ctx_status`, `moe_ctx_destroy`, `moe_layer_host` and `moe_layer_host_wait`, which say so).
  *   - Every function returns a `moe_status`; no exception crosses the boundary.
  *     `moe_last_error` gives a human-readable reason for the last failure on a context.
  *   - Problems only the device can see (an expert index outside [0,E), a bounded wait
@@ -275,6 +275,24 @@ moe_status moe_dispatch_layout_static(const int32_t* topk_idx, int32_t T, int32_
 moe_status moe_layer_host(moe_ctx* ctx, const float* logits_host, const float* select_bias, const void* x_host,
                           int32_t T, const void* w_gate_up, const void* w_down, const void* ws_gate_up,
                           const void* ws_down, void* out_host);
+
+/* Pipelined form of moe_layer_host: MOE_HOST_SLOTS staging slots, so that the host<->device copies of one step
+ * overlap the kernels and the copies of others (host-to-device, kernels and device-to-host run as a three-stage
+ * pipeline; with three or more slots in rotation each stage stays busy).  moe_layer_host_submit(slot) enqueues the
+ * host-to-device copies of logits_host and x_host on a copy stream of the context, the step's kernels on the
+ * context's stream behind them, and the copy of the result to out_host on a second copy stream behind the
+ * kernels; it returns without synchronising.  moe_layer_host_wait(slot) blocks the calling thread until that
+ * slot's result has arrived in out_host (a no-op for a slot with nothing in flight).  A slot must be waited for
+ * before it is submitted again (MOE_ERR_STATE otherwise); the host buffers of a submitted slot must stay valid
+ * and untouched until its wait returns, and must be pinned for the copies to overlap anything.  Steps execute in
+ * submission order.  The two copy streams and the events are created by the first submit on a context (host
+ * resources, no device memory) and belong to that context alone; moe_ctx_destroy refuses while a slot is in
+ * flight.  Device-side arguments as for moe_layer_host.  Not for contexts created for FP8 weights. */
+#define MOE_HOST_SLOTS 4
+moe_status moe_layer_host_submit(moe_ctx* ctx, int32_t slot, const float* logits_host, const float* select_bias,
+                                 const void* x_host, int32_t T, const void* w_gate_up, const void* w_down,
+                                 const void* ws_gate_up, const void* ws_down, void* out_host);
+moe_status moe_layer_host_wait(moe_ctx* ctx, int32_t slot);
 
 /* Test/inspection only: device pointers into the buffer set of the step in progress (between steps: of
  * the step that finished last).  Rows

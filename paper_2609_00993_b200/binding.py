@@ -28,7 +28,7 @@ STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_CAPACITY", 3:
 # every symbol include/moe_pd.h declares
 EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_destroy", "moe_ctx_status",
            "moe_last_error", "moe_route", "moe_dispatch_layout", "moe_grouped_ffn", "moe_grouped_ffn_fp8", "moe_combine",
-           "moe_layer_host",
+           "moe_layer_host", "moe_layer_host_submit", "moe_layer_host_wait",
            "moe_ctx_debug_ptrs", "moe_ctx_debug_ptrs_fp8", "moe_ctx_launch_count", "moe_ctx_set_profiling", "moe_ctx_read_profile",
            "moe_dispatch_layout_static", "moe_ctx_set_segments", "moe_ctx_abandon_step", "moe_turnstile_create", "moe_turnstile_destroy",
            "moe_turnstile_set_span", "moe_turnstile_begin_epoch", "moe_turnstile_publish", "moe_turnstile_task_done",
@@ -98,6 +98,10 @@ def load_library() -> ctypes.CDLL:
     lib.moe_combine.argtypes = [vp, vp, vp, i32, vp]
     lib.moe_layer_host.restype = i32
     lib.moe_layer_host.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.moe_layer_host_submit.restype = i32
+    lib.moe_layer_host_submit.argtypes = [vp, i32, vp, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.moe_layer_host_wait.restype = i32
+    lib.moe_layer_host_wait.argtypes = [vp, i32]
     lib.moe_ctx_debug_ptrs.restype = i32
     lib.moe_ctx_debug_ptrs.argtypes = [vp] + [ctypes.POINTER(vp)] * 6
     lib.moe_ctx_abandon_step.restype = i32
@@ -202,6 +206,21 @@ class MoeContext:
             pass
 
     # -- the C entry points, same names
+    def moe_layer_host_submit(self, slot, logits_host, select_bias, x_host, w_gate_up, w_down, ws_gate_up, ws_down,
+                              out_host, T=None):
+        """Pipelined form of moe_layer_host: returns once the copies and kernels of the step are enqueued; the
+        host tensors (pinned) must stay untouched until moe_layer_host_wait(slot)."""
+        for n, t in (("logits_host", logits_host), ("x_host", x_host), ("out_host", out_host)):
+            if t.is_cuda:
+                raise ValueError(f"{n} must be a host tensor")
+        T = x_host.shape[0] if T is None else T
+        self._check(self.lib.moe_layer_host_submit(self.handle, slot, _ptr(logits_host), _ptr(select_bias),
+                                                   _ptr(x_host), T, _ptr(w_gate_up), _ptr(w_down), _ptr(ws_gate_up),
+                                                   _ptr(ws_down), _ptr(out_host)))
+
+    def moe_layer_host_wait(self, slot):
+        self._check(self.lib.moe_layer_host_wait(self.handle, slot))
+
     def moe_ctx_status(self) -> int:
         v = ctypes.c_int32(0)
         self._check(self.lib.moe_ctx_status(self.handle, ctypes.byref(v)))

@@ -95,6 +95,19 @@ size_t carve_set(const moe_config& c, char* base, BufferSet* out) {
   return off;
 }
 
+// One more staging slot of the pipelined host path (the first slots are the staging buffers of the context's
+// buffer sets); with base == nullptr it only measures.
+size_t carve_staging(const moe_config& c, char* base, BufferSet* out) {
+  const size_t T = (size_t)c.max_tokens, H = (size_t)c.hidden, E = (size_t)c.n_experts;
+  const size_t a = align_up(T * E * 4, 256), b = align_up(T * H * 2, 256);
+  if (base && out) {
+    out->logits = reinterpret_cast<float*>(base);
+    out->x_stage = base + a;
+    out->out_stage = base + a + b;
+  }
+  return a + 2 * b;
+}
+
 const char* validate_config(const moe_config* c) {
   if (!c) return "config is NULL";
   if (c->hidden <= 0 || c->hidden % 64) return "hidden must be a positive multiple of 64";
@@ -124,7 +137,8 @@ Layout measure(const moe_config& c) {
   Layout l;
   l.n_sets = (c.phase == MOE_PHASE_DECODE) ? 2 : 1;
   l.set_bytes = carve_set(c, nullptr, nullptr);
-  l.total_bytes = kStatusBlock + l.set_bytes * (size_t)l.n_sets;
+  l.total_bytes = kStatusBlock + l.set_bytes * (size_t)l.n_sets +
+                  (size_t)(MOE_HOST_SLOTS - l.n_sets) * carve_staging(c, nullptr, nullptr);
   return l;
 }
 
@@ -161,6 +175,16 @@ struct moe_ctx {
   struct Span { cudaEvent_t beg, end; int stage; };
   std::vector<Span> spans;
   size_t spans_used;
+  // pipelined host path: staging slots and two copy streams (created by the first moe_layer_host_submit)
+  struct HostSlot {
+    float* logits;
+    char* x;
+    char* out;
+    cudaEvent_t h2d, comp, done;
+    bool in_flight;
+  } slots[MOE_HOST_SLOTS];
+  cudaStream_t h2d_stream, d2h_stream;
+  bool host_pipeline;
   char err[256];
 };
 
@@ -346,6 +370,18 @@ moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspa
   ctx->err[0] = 0;
   ctx->status = reinterpret_cast<int*>(ctx->ws);
   for (int s = 0; s < l.n_sets; ++s) carve_set(*cfg, ctx->ws + kStatusBlock + (size_t)s * l.set_bytes, &ctx->sets[s]);
+  ctx->host_pipeline = false;
+  const size_t staging_bytes = carve_staging(*cfg, nullptr, nullptr);
+  for (int s = 0; s < MOE_HOST_SLOTS; ++s) {
+    BufferSet st = ctx->sets[s < l.n_sets ? s : 0];
+    if (s >= l.n_sets)
+      carve_staging(*cfg, ctx->ws + kStatusBlock + l.set_bytes * (size_t)l.n_sets + (size_t)(s - l.n_sets) * staging_bytes,
+                    &st);
+    ctx->slots[s].logits = st.logits;
+    ctx->slots[s].x = st.x_stage;
+    ctx->slots[s].out = st.out_stage;
+    ctx->slots[s].in_flight = false;
+  }
 
   {
     // Isolation is validated at construction: no two live contexts may share a mutable byte, and a
@@ -392,6 +428,19 @@ moe_status moe_ctx_destroy(moe_ctx* ctx) {
   cudaError_t q = cudaEventQuery(ctx->done);
   if (q == cudaErrorNotReady) return fail(ctx, MOE_ERR_STATE, "work is still in flight on the context's stream");
   if (q != cudaSuccess) (void)cudaGetLastError();
+  for (int s = 0; s < MOE_HOST_SLOTS; ++s)
+    if (ctx->slots[s].in_flight && cudaEventQuery(ctx->slots[s].done) == cudaErrorNotReady)
+      return fail(ctx, MOE_ERR_STATE, "a moe_layer_host_submit slot is still in flight");
+  (void)cudaGetLastError();
+  if (ctx->host_pipeline) {
+    for (int s = 0; s < MOE_HOST_SLOTS; ++s) {
+      cudaEventDestroy(ctx->slots[s].h2d);
+      cudaEventDestroy(ctx->slots[s].comp);
+      cudaEventDestroy(ctx->slots[s].done);
+    }
+    cudaStreamDestroy(ctx->h2d_stream);
+    cudaStreamDestroy(ctx->d2h_stream);
+  }
   {
     std::lock_guard<std::mutex> lock(g_registry_mutex);
     for (size_t i = 0; i < g_registry.size(); ++i)
@@ -694,6 +743,81 @@ moe_status moe_layer_host(moe_ctx* ctx, const float* logits_host, const float* s
   if (T > 0) e = cudaMemcpyAsync(out_host, b.out_stage, x_bytes, cudaMemcpyDeviceToHost, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "device-to-host copy");
+  return MOE_OK;
+}
+
+moe_status moe_layer_host_submit(moe_ctx* ctx, int32_t slot, const float* logits_host, const float* select_bias,
+                                 const void* x_host, int32_t T, const void* w_gate_up, const void* w_down,
+                                 const void* ws_gate_up, const void* ws_down, void* out_host) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= MOE_HOST_SLOTS) return fail(ctx, MOE_ERR_INVALID_ARG, "slot must be in [0, %d)", MOE_HOST_SLOTS);
+  if (ctx->cfg.weight_format != MOE_WEIGHTS_BF16)
+    return fail(ctx, MOE_ERR_STATE, "the host path serves contexts created for BF16 weights");
+  if (ctx->state != ST_IDLE) return fail(ctx, MOE_ERR_STATE, "moe_layer_host_submit called in the middle of a step");
+  if (ctx->slots[slot].in_flight) return fail(ctx, MOE_ERR_STATE, "slot %d has not been waited for", slot);
+  if (T < 0) return fail(ctx, MOE_ERR_INVALID_ARG, "T < 0");
+  if (T > ctx->cfg.max_tokens) return fail(ctx, MOE_ERR_CAPACITY, "T = %d exceeds max_tokens = %d", T, ctx->cfg.max_tokens);
+  if (T > 0 && (!logits_host || !x_host || !out_host)) return fail(ctx, MOE_ERR_INVALID_ARG, "NULL host pointer");
+  DeviceGuard guard(ctx->device);
+  cudaError_t e = cudaSuccess;
+  if (!ctx->host_pipeline) {
+    constexpr int kEvents = 3 * MOE_HOST_SLOTS;
+    cudaEvent_t ev[kEvents] = {};
+    cudaStream_t st[2] = {};
+    for (int i = 0; i < kEvents && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) e = cudaStreamCreateWithFlags(&st[i], cudaStreamNonBlocking);
+    if (e != cudaSuccess) {
+      for (int i = 0; i < kEvents; ++i)
+        if (ev[i]) cudaEventDestroy(ev[i]);
+      for (int i = 0; i < 2; ++i)
+        if (st[i]) cudaStreamDestroy(st[i]);
+      return cuda_fail(ctx, e, "moe_layer_host_submit set-up");
+    }
+    for (int s = 0; s < MOE_HOST_SLOTS; ++s) {
+      ctx->slots[s].h2d = ev[3 * s];
+      ctx->slots[s].comp = ev[3 * s + 1];
+      ctx->slots[s].done = ev[3 * s + 2];
+    }
+    ctx->h2d_stream = st[0];
+    ctx->d2h_stream = st[1];
+    ctx->host_pipeline = true;
+  }
+  moe_ctx::HostSlot& hs = ctx->slots[slot];
+  BufferSet& b = ctx->sets[ctx->cur];
+  const moe_config& c = ctx->cfg;
+  const size_t x_bytes = (size_t)T * c.hidden * 2;
+  if (T > 0) {
+    e = cudaMemcpyAsync(hs.logits, logits_host, (size_t)T * c.n_experts * 4, cudaMemcpyHostToDevice, ctx->h2d_stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(hs.x, x_host, x_bytes, cudaMemcpyHostToDevice, ctx->h2d_stream);
+  }
+  if (e == cudaSuccess) e = cudaEventRecord(hs.h2d, ctx->h2d_stream);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->stream, hs.h2d, 0);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "host-to-device copy");
+  moe_status st = moe_route(ctx, hs.logits, select_bias, T, b.topk_idx, b.topk_w);
+  if (st == MOE_OK) st = moe_dispatch_layout(ctx, b.topk_idx, T, hs.x, nullptr, nullptr, nullptr, nullptr);
+  if (st == MOE_OK) st = moe_grouped_ffn(ctx, w_gate_up, w_down, hs.x, ws_gate_up, ws_down, T);
+  if (st == MOE_OK) st = moe_combine(ctx, b.topk_w, nullptr, T, hs.out);
+  if (st != MOE_OK) {
+    ctx->state = ST_IDLE;
+    return st;
+  }
+  e = cudaEventRecord(hs.comp, ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->d2h_stream, hs.comp, 0);
+  if (e == cudaSuccess && T > 0) e = cudaMemcpyAsync(out_host, hs.out, x_bytes, cudaMemcpyDeviceToHost, ctx->d2h_stream);
+  if (e == cudaSuccess) e = cudaEventRecord(hs.done, ctx->d2h_stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "device-to-host copy");
+  hs.in_flight = true;
+  return MOE_OK;
+}
+
+moe_status moe_layer_host_wait(moe_ctx* ctx, int32_t slot) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= MOE_HOST_SLOTS) return fail(ctx, MOE_ERR_INVALID_ARG, "slot must be in [0, %d)", MOE_HOST_SLOTS);
+  if (!ctx->slots[slot].in_flight) return MOE_OK;
+  DeviceGuard guard(ctx->device);
+  cudaError_t e = cudaEventSynchronize(ctx->slots[slot].done);
+  ctx->slots[slot].in_flight = false;
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_layer_host_wait");
   return MOE_OK;
 }
 

@@ -43,7 +43,9 @@ def test_a_stream_serves_one_phase_only():
 
 
 def test_decode_context_holds_two_buffer_sets():
-    assert B.moe_ctx_workspace_bytes(_cfg(B.MOE_PHASE_DECODE)) > 1.9 * B.moe_ctx_workspace_bytes(_cfg()) - 4096
+    staging = 32 * 8 * 4 + 2 * 32 * 256 * 2  # one extra host-staging slot (P carves three, D two)
+    assert (B.moe_ctx_workspace_bytes(_cfg(B.MOE_PHASE_DECODE)) - 2 * staging
+            > 1.9 * (B.moe_ctx_workspace_bytes(_cfg()) - 3 * staging) - 4096)
     ctx = B.MoeContext(_cfg(B.MOE_PHASE_DECODE))
     shape = wl.LayerShape("t", T=32, H=256, E=8, k=2, I=128)
     w, a = wl.make_weights(shape, 1, DEV), wl.make_activations(shape, 2, DEV)
@@ -116,6 +118,45 @@ def test_an_abandoned_step_leaves_the_context_usable_and_rests_its_buffer_set():
         ref = oracle.layer(wl.bits(a2["x"]), np_f32(a2["logits"]), None, 2, wl.bits(w["w_gate_up"]),
                            wl.bits(w["w_down"]))
         check_layer(out, ref["out"], label="after an abandoned step")
+        ctx.close()
+
+
+def test_pipelined_host_path_overlaps_steps_and_matches_the_device_path():
+    """moe_layer_host_submit / moe_layer_host_wait: results equal the device path's bit for bit, in submission
+    order, on both phases; a slot cannot be resubmitted before it was waited for."""
+    shape = wl.LayerShape("t", T=32, H=256, E=8, k=2, I=128, shared_I=64, select_bias=True)
+    w = wl.make_weights(shape, 1, DEV)
+    acts = [wl.make_activations(shape, 10 + i, DEV) for i in range(5)]
+    wargs = (w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+    torch.cuda.synchronize()
+    for phase in (B.MOE_PHASE_PREFILL, B.MOE_PHASE_DECODE):
+        ctx = B.MoeContext(_cfg(phase, shared_inter=64), stream=torch.cuda.Stream())
+        ref = []
+        for a in acts:
+            o, _ = ctx.layer(a["x"], a["logits"], a["bias"], *wargs)
+            ref.append(o.clone())
+        torch.cuda.synchronize()
+        hx = [a["x"].cpu().pin_memory() for a in acts]
+        hl = [a["logits"].cpu().pin_memory() for a in acts]
+        hout = [torch.zeros(32, 256, dtype=torch.bfloat16).pin_memory() for _ in acts]
+        n_slots = 3  # any number up to MOE_HOST_SLOTS = 4
+        for i in range(n_slots):
+            ctx.moe_layer_host_submit(i, hl[i], acts[i]["bias"], hx[i], *wargs, hout[i])
+        with pytest.raises(B.MoeError) as ei:  # slot 1 has not been waited for
+            ctx.moe_layer_host_submit(1, hl[3], acts[3]["bias"], hx[3], *wargs, hout[3])
+        assert ei.value.status == B.MOE_ERR_STATE
+        with pytest.raises(B.MoeError) as ei:
+            ctx.moe_layer_host_submit(4, hl[3], acts[3]["bias"], hx[3], *wargs, hout[3])
+        assert ei.value.status == B.MOE_ERR_INVALID_ARG
+        for i in range(n_slots, 5):
+            ctx.moe_layer_host_wait(i % n_slots)
+            assert torch.equal(hout[i - n_slots], ref[i - n_slots].cpu())
+            ctx.moe_layer_host_submit(i % n_slots, hl[i], acts[i]["bias"], hx[i], *wargs, hout[i])
+        for sl in range(4):
+            ctx.moe_layer_host_wait(sl)  # slot 3 never had anything in flight: a no-op
+        for i in range(5):
+            assert torch.equal(hout[i], ref[i].cpu())
+        assert ctx.moe_ctx_status() == B.MOE_OK
         ctx.close()
 
 
