@@ -151,7 +151,9 @@ moe_status moe_route(moe_ctx* ctx, const float* logits, const float* select_bias
  * With flat slot f = t*k + j and N = T*k:
  *   counts[e]  = #{f : topk_idx[f] == e};   offsets[0] = 0, offsets[e+1] = offsets[e] + counts[e]
  *   perm[p] = f and inv_perm[f] = p, where slots of one expert keep ascending f (stable)
- *   x_perm[p,:] = x[perm[p] / k, :]   (bit copy into the context's workspace)
+ *   x_perm[p,:] = x[perm[p] / k, :]   (bit copy into the context's workspace; with row_gather = 1 the copy is
+ *                 skipped and GEMM1 reads x through perm; a context created for FP8 weights quantises each row
+ *                 of x once and moves the E4M3 codes and the row scales instead, see moe_grouped_ffn_fp8)
  * topk_idx [T,k] int32 (the caller's own routing is welcome; moe_route is optional);
  * x [T,H] bf16, or NULL to build the layout only (then moe_grouped_ffn is not allowed);
  * counts [E], offsets [E+1], perm [N], inv_perm [N] int32 -- each may be NULL, in which
