@@ -410,6 +410,11 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm):
     res["serial_us"] = {"p50": percentile(ser_us, 50), "p99": percentile(ser_us, 99),
                         "note": "D ready at the start of an unsegmented P batch, runs after it"}
     res["prefill_serial_tokens_per_s"] = wl.C4_P.T / ((p_alone_ms + res["alone_us"]["p50"] * 1e-3) * 1e-3)
+    # how much of a P batch plus one D step the turnstile run hides by running them at the same time: 0 % means
+    # strict time slicing (the turnstile admits D between P segments and P waits for it), 100 % would hide all of D
+    t_p, t_d = p_alone_ms * 1e-3, res["alone_us"]["p50"] * 1e-6
+    t_conc = wl.C4_P.T / res["prefill_concurrent_tokens_per_s"]  # seconds per P batch while D steps run
+    res["overlap_pct"] = 100.0 * (t_p + t_d - t_conc) / t_d
     res["iterations"] = iters
     res["workload"] = "C4: P T=4096 on stream P || D T=64 on stream D (high priority), DeepSeek-V3-shaped layer"
     ctx_p.close(); ctx_d.close()
