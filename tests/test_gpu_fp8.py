@@ -145,3 +145,51 @@ def test_fp8_decode_step_replays_from_a_cuda_graph_and_is_run_to_run_identical()
     assert d.moe_ctx_status() == B.MOE_OK
     del g
     d.close()
+
+
+_V3_FP8 = {}
+
+
+def _v3_fp8_weights():
+    """One copy of the V3-shaped FP8 weights (11.4 GB) for both phases' tests."""
+    if not _V3_FP8:
+        shape = wl.C4_D
+        w8 = wl.make_weights_fp8(shape, 21, DEV, std=1.0)
+        for name, fan in (("sw_gate_up", shape.H), ("sws_gate_up", shape.H), ("sw_down", shape.I),
+                          ("sws_down", shape.shared_I)):
+            w8[name] = (w8[name] / fan ** 0.5).contiguous()
+        _V3_FP8.update(w8)
+    return _V3_FP8
+
+
+@pytest.mark.parametrize("shape,phase", [(wl.C4_D, B.MOE_PHASE_DECODE), (wl.C4_P, B.MOE_PHASE_PREFILL)],
+                         ids=["decode-T64", "prefill-T4096"])
+def test_fp8_at_the_v3_layer_shape_on_sampled_tokens(shape, phase):
+    """Both batches of config 4 on the DeepSeek-V3-shaped layer (H=7168, E=256, top-8, I=2048, shared expert) with
+    FP8 weights: 56 k-blocks per GEMM1 tile, the small-M kernel for D and the large-M kernel for P, the shared
+    expert riding along.  The oracle follows sampled tokens through their eight experts (only those experts'
+    codes leave the GPU)."""
+    T, H, E, k, I, Is = shape.T, shape.H, shape.E, shape.k, shape.I, shape.shared_I
+    w8 = _v3_fp8_weights()
+    a = wl.make_activations(shape, 22, DEV)
+    ctx = B.MoeContext(B.make_config(H, E, k, I, Is, T, phase, weight_format=B.MOE_WEIGHTS_FP8_E4M3))
+    torch.cuda.synchronize()
+    out, bufs = ctx.layer_fp8(a["x"], a["logits"], a["bias"], w8)
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_OK
+    idx_ref, w_ref = oracle.route(np_f32(a["logits"]), np_f32(a["bias"]), k)
+    assert np.array_equal(np_i32(bufs["topk_idx"]), idx_ref)
+    x_bits = wl.bits(a["x"])
+    shared = [_np_u8(w8["wsq_gate_up"]), np_f32(w8["sws_gate_up"]), _np_u8(w8["wsq_down"]), np_f32(w8["sws_down"])]
+    out_gpu = np_f32(out)
+    for t in (0, (17 * T) // 64, T - 1):
+        acc = oracle.ffn_fp8(x_bits[t:t + 1], *shared)[0].astype(np.float64)
+        for j in range(k):
+            e = int(idx_ref[t, j])
+            y = oracle.ffn_fp8(x_bits[t:t + 1], _np_u8(w8["wq_gate_up"][e]), np_f32(w8["sw_gate_up"][e]),
+                               _np_u8(w8["wq_down"][e]), np_f32(w8["sw_down"][e]))[0]
+            acc += float(w_ref[t, j]) * y.astype(np.float64)
+        rel = np.linalg.norm(out_gpu[t] - acc) / np.linalg.norm(acc)
+        print(f"[fp8 parity V3 shape T={T}, token {t}] rel_l2={rel:.4g}")
+        assert rel <= 1e-2, (t, rel)
+    ctx.close()
