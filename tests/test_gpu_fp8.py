@@ -86,14 +86,15 @@ def test_fp8_stages_against_the_oracle(T, H, E, k, I, shared_I, phase, variant):
     # elements; where that moves an element across an E4M3 rounding boundary its code changes by one step
     # (2^-3 relative at worst), which happens to a fraction ~2^-8 / 2^-4 = 6 % of the differing elements.  With
     # at most every element differing, the relative L2 error of y is bounded by sqrt(0.06) * 2^-4 / sqrt(3)
-    # ~ 0.9 %, hence the 1e-2 below (measured: 0.23 %).
+    # ~ 0.9 % in the worst case.  Measured: 0.23 %, which is the bf16 rounding of the output itself, so the
+    # layer's own tolerance (relative L2 <= 5e-3) is asserted here too.
     ref = oracle.layer_fp8(wl.bits(a["x"]), np_f32(a["logits"]), np_f32(a["bias"]), k, h["wq_gate_up"], h["sw_gate_up"],
                            h["wq_down"], h["sw_down"], h["wsq_gate_up"], h["sws_gate_up"], h["wsq_down"], h["sws_down"])
     for name in ("topk_idx", "counts", "offsets", "perm", "inv_perm"):
         assert np.array_equal(np_i32(bufs[name]).reshape(-1), np.asarray(ref[name]).reshape(-1)), name
     rel = np.linalg.norm(np_f32(out) - ref["out"]) / np.linalg.norm(ref["out"])
     print(f"[fp8 parity T={T} H={H} E={E}] rel_l2={rel:.4g}")
-    assert rel <= 1e-2, rel
+    assert rel <= 5e-3, rel
     ctx.close()
 
 
@@ -191,5 +192,5 @@ def test_fp8_at_the_v3_layer_shape_on_sampled_tokens(shape, phase):
             acc += float(w_ref[t, j]) * y.astype(np.float64)
         rel = np.linalg.norm(out_gpu[t] - acc) / np.linalg.norm(acc)
         print(f"[fp8 parity V3 shape T={T}, token {t}] rel_l2={rel:.4g}")
-        assert rel <= 1e-2, (t, rel)
+        assert rel <= 5e-3, (t, rel)
     ctx.close()
