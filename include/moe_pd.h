@@ -195,8 +195,9 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
  * the same way from the quantised x with its own codes and scales.
  * wq_gate_up [E,2I,H] uint8, sw_gate_up [E,2I] fp32, wq_down [E,H,I] uint8, sw_down [E,H] fp32;
  * wsq_gate_up [2I_s,H], sws_gate_up [2I_s], wsq_down [H,I_s], sws_down [H] (required iff S = 1).
- * H, I and I_s may not exceed 8192.  The row gather, prefill segmentation and moe_layer_host do not apply to
- * an FP8 context.  Errors as for moe_grouped_ffn; MOE_ERR_STATE if the context was created for BF16 weights. */
+ * H, I and I_s may not exceed 8192.  Prefill segmentation (moe_ctx_set_segments) applies as to moe_grouped_ffn,
+ * the quantisation of the activation being one more segment between the two passes; the row gather and the
+ * host-buffer entry points do not apply to an FP8 context.  Errors as for moe_grouped_ffn; MOE_ERR_STATE if the context was created for BF16 weights. */
 moe_status moe_grouped_ffn_fp8(moe_ctx* ctx, const void* wq_gate_up, const float* sw_gate_up, const void* wq_down,
                                const float* sw_down, const void* wsq_gate_up, const float* sws_gate_up,
                                const void* wsq_down, const float* sws_down, int32_t T);

@@ -658,31 +658,75 @@ moe_status moe_grouped_ffn_fp8(moe_ctx* ctx, const void* wq_gate_up, const float
   int n = 0;
   cudaError_t e = cudaSuccess;
   if (T > 0) {
-    // GEMM1 + SwiGLU on the rows moe_dispatch_layout quantised -> quantise the activation -> GEMM2; the shared
-    // expert's passes ride in the routed launches
+    // GEMM1 + SwiGLU on the rows moe_dispatch_layout quantised -> quantise the activation -> GEMM2.
+    // Unsegmented: the shared expert's passes ride in the routed launches.  Segmented (moe_ctx_set_segments): one
+    // launch per group of experts and pass, the shared expert's passes and the activation's quantisation are
+    // segments of their own, and the boundary hook runs after each.
+    const int span = (ctx->seg_experts > 0 && ctx->seg_experts < c.n_experts) ? ctx->seg_experts : c.n_experts;
+    const int routed_segs = (c.n_experts + span - 1) / span;
+    const bool fuse_shared = shared && ctx->seg_experts == 0;
+    const int n_bound = 2 * routed_segs + 1 + ((shared && !fuse_shared) ? 2 : 0);
+    int bound = 0;
+    auto boundary = [&]() {
+      if (ctx->seg_experts > 0 && ctx->boundary_fn) {
+        if (!capturing(ctx)) cudaEventRecord(ctx->done, ctx->stream);
+        ctx->boundary_fn(ctx->boundary_user, bound, n_bound);
+      }
+      ++bound;
+    };
     moe::GemmProblem g1{b.xq, wq_gate_up, b.act, ctx->offsets, 0, Ncap, N, c.n_experts, c.inter, c.hidden, true};
     g1.fp8 = true;
     g1.row_scale = b.sx;
     g1.w_scale = sw_gate_up;
-    moe::GemmDenseGroup s1{b.xq_tok, wsq_gate_up, b.act_shared, T, c.shared_inter, c.hidden, b.sx_tok, sws_gate_up};
-    {
-      StageTimer tm(ctx, 3);
-      e = run_gemm(ctx, g1, shared ? &s1 : nullptr, T, &n);
-    }
-    if (e == cudaSuccess) {
-      StageTimer tm(ctx, 9);
-      e = moe::launch_quantize_rows(b.act, N, c.inter, b.aq, b.sa, ctx->stream, &n);
-      if (e == cudaSuccess && shared)
-        e = moe::launch_quantize_rows(b.act_shared, T, c.shared_inter, b.aq_shared, b.sa_shared, ctx->stream, &n);
-    }
     moe::GemmProblem g2{b.aq, wq_down, b.y_perm, ctx->offsets, 0, Ncap, N, c.n_experts, c.hidden, c.inter, false};
     g2.fp8 = true;
     g2.row_scale = b.sa;
     g2.w_scale = sw_down;
+    moe::GemmDenseGroup s1{b.xq_tok, wsq_gate_up, b.act_shared, T, c.shared_inter, c.hidden, b.sx_tok, sws_gate_up};
     moe::GemmDenseGroup s2{b.aq_shared, wsq_down, b.y_shared, T, c.hidden, c.shared_inter, b.sa_shared, sws_down};
-    if (e == cudaSuccess) {
-      StageTimer tm(ctx, 4);
-      e = run_gemm(ctx, g2, shared ? &s2 : nullptr, T, &n);
+    auto dense_problem = [&](const moe::GemmDenseGroup& d, bool gated) {
+      moe::GemmProblem q{d.A, d.W, d.out, nullptr, T, T, T, 1, d.n_feat, d.K, gated};
+      q.fp8 = true;
+      q.row_scale = d.row_scale;
+      q.w_scale = d.w_scale;
+      return q;
+    };
+    for (int pass = 0; pass < 2 && e == cudaSuccess; ++pass) {
+      moe::GemmProblem& g = pass == 0 ? g1 : g2;
+      for (int e0 = 0; e0 < c.n_experts && e == cudaSuccess; e0 += span) {
+        g.e_begin = e0;
+        g.e_end = e0 + span < c.n_experts ? e0 + span : c.n_experts;
+        {
+          StageTimer tm(ctx, pass == 0 ? 3 : 4);
+          e = run_gemm(ctx, g, fuse_shared ? (pass == 0 ? &s1 : &s2) : nullptr, T, &n);
+        }
+        if (e == cudaSuccess) boundary();
+      }
+      if (pass == 0 && e == cudaSuccess && shared && !fuse_shared) {
+        moe::GemmProblem d1 = dense_problem(s1, true);
+        {
+          StageTimer tm(ctx, 5);
+          e = run_gemm(ctx, d1, nullptr, T, &n);
+        }
+        if (e == cudaSuccess) boundary();
+      }
+      if (pass == 0 && e == cudaSuccess) {
+        {
+          StageTimer tm(ctx, 9);
+          e = moe::launch_quantize_rows(b.act, N, c.inter, b.aq, b.sa, ctx->stream, &n);
+          if (e == cudaSuccess && shared)
+            e = moe::launch_quantize_rows(b.act_shared, T, c.shared_inter, b.aq_shared, b.sa_shared, ctx->stream, &n);
+        }
+        if (e == cudaSuccess) boundary();
+      }
+    }
+    if (e == cudaSuccess && shared && !fuse_shared) {
+      moe::GemmProblem d2 = dense_problem(s2, false);
+      {
+        StageTimer tm(ctx, 6);
+        e = run_gemm(ctx, d2, nullptr, T, &n);
+      }
+      if (e == cudaSuccess) boundary();
     }
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_grouped_ffn_fp8");

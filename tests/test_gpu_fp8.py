@@ -194,3 +194,22 @@ def test_fp8_at_the_v3_layer_shape_on_sampled_tokens(shape, phase):
         print(f"[fp8 parity V3 shape T={T}, token {t}] rel_l2={rel:.4g}")
         assert rel <= 5e-3, (t, rel)
     ctx.close()
+
+
+def test_fp8_prefill_segments_are_bit_identical_and_boundaries_are_counted():
+    shape = wl.LayerShape("f8", T=300, H=512, E=6, k=3, I=192, shared_I=128, select_bias=True)
+    w8, a = wl.make_weights_fp8(shape, 5, DEV), wl.make_activations(shape, 6, DEV)
+    ctx = B.MoeContext(B.make_config(512, 6, 3, 192, 128, 300, B.MOE_PHASE_PREFILL,
+                                     weight_format=B.MOE_WEIGHTS_FP8_E4M3))
+    torch.cuda.synchronize()
+    whole, _ = ctx.layer_fp8(a["x"], a["logits"], a["bias"], w8)
+    whole = whole.clone()
+    seen = []
+    ctx.moe_ctx_set_segments(2, lambda i, n: seen.append((i, n)))
+    cut, _ = ctx.layer_fp8(a["x"], a["logits"], a["bias"], w8)
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_OK
+    assert torch.equal(cut, whole)
+    # 3 routed segments per pass, the shared expert's two passes and the activation's quantisation
+    assert seen == [(i, 9) for i in range(9)]
+    ctx.close()
