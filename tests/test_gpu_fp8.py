@@ -213,3 +213,24 @@ def test_fp8_prefill_segments_are_bit_identical_and_boundaries_are_counted():
     # 3 routed segments per pass, the shared expert's two passes and the activation's quantisation
     assert seen == [(i, 9) for i in range(9)]
     ctx.close()
+
+
+def test_entry_points_that_do_not_serve_an_fp8_context_say_so():
+    shape = wl.LayerShape("f8", T=16, H=256, E=4, k=2, I=128)
+    w16, a = wl.make_weights(shape, 1, DEV), wl.make_activations(shape, 2, DEV)
+    ctx = B.MoeContext(B.make_config(256, 4, 2, 128, 0, 16, weight_format=B.MOE_WEIGHTS_FP8_E4M3))
+    hx, hl = a["x"].cpu().pin_memory(), a["logits"].cpu().pin_memory()
+    hout = torch.empty(16, 256, dtype=torch.bfloat16).pin_memory()
+    for call in (lambda: ctx.moe_layer_host_submit(0, hl, None, hx, w16["w_gate_up"], w16["w_down"], None, None, hout),
+                 lambda: ctx.moe_layer_host(hl, None, hx, w16["w_gate_up"], w16["w_down"], None, None, hout)):
+        with pytest.raises(B.MoeError) as ei:
+            call()
+        assert ei.value.status == B.MOE_ERR_STATE
+    # the context is between steps after either refusal and still runs an FP8 step
+    w8 = wl.make_weights_fp8(shape, 3, DEV)
+    out, _ = ctx.layer_fp8(a["x"], a["logits"], None, w8)
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_OK and torch.isfinite(out.float()).all()
+    with pytest.raises(B.MoeError):  # the row gather has no FP8 form
+        B.MoeContext(B.make_config(256, 4, 2, 128, 0, 16, row_gather=1, weight_format=B.MOE_WEIGHTS_FP8_E4M3))
+    ctx.close()
