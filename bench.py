@@ -626,7 +626,14 @@ def run_ours(args):
     bytes_permute = 2.0 * T * H + 2.0 * N * H + 4.0 * N
     bytes_combine = 2.0 * N * H + 2.0 * T * H + 8.0 * N
     gemm2_flops = 2.0 * N * H * I
+    # Bracketing every stage with its own pair of timing events drains the stream at each boundary, which the plain
+    # timed region does not do: the sum of the bracketed stages exceeds the plain step by this much per stage
+    # (the per-stage figures below are the bracketed, pessimistic ones).
+    n_br = sum(1 for n in ("route", "layout", "permute", "gemm1_swiglu", "gemm2", "combine") if stage_us.get(n))
+    bracket_overhead = (sum(stage_us[n] for n in ("route", "layout", "permute", "gemm1_swiglu", "gemm2", "combine")
+                            if stage_us.get(n)) - 1e3 * ms_per_step) / max(n_br, 1)
     stages = {
+        "event_bracket_overhead_us_per_stage": bracket_overhead,
         "route_us": stage_us["route"], "layout_us": stage_us["layout"],
         "layout": {"us": stage_us["layout"], "launches": 3, "launch_floor_us_per_launch": launch_floor_us,
                    "note": "counts + scan + placement move 1.3 MB at this size: three dependent launches of chained small loads, bound by latency, not by HBM"},
