@@ -69,3 +69,34 @@ def test_random_shape(case):
     e = layer_errors(out, ref["out"])
     assert e["rel_l2"] <= 5e-3, e
     ctx.close()
+
+
+@pytest.mark.parametrize("case", CASES[:15], ids=lambda c: f"fp8-{c[0]}-T{c[1]}-H{c[2]}-E{c[3]}-k{c[4]}-I{c[5]}-S{c[6]}-{c[8]}")
+def test_random_shape_fp8(case):
+    """The FP8 (E4M3) precision variant on the same list, against the oracle's statement of its recipe."""
+    i, T, H, E, k, I, shared_I, skew, mode = case
+    shape = wl.LayerShape("r8", T=T, H=H, E=E, k=k, I=I, shared_I=shared_I, select_bias=True)
+    w8 = wl.make_weights_fp8(shape, 700 + i, DEV, std=1.0)
+    for name, fan in (("sw_gate_up", H), ("sws_gate_up", H), ("sw_down", I), ("sws_down", shared_I)):
+        if w8[name] is not None:
+            w8[name] = (w8[name] / fan ** 0.5).contiguous()
+    a = wl.make_activations(shape, 800 + i, DEV)
+    if skew:
+        a["logits"] = (a["logits"] + wl.zipf_log_weight(E, 1.2, 900 + i, DEV)).contiguous()
+    phase = B.MOE_PHASE_PREFILL if T >= 130 else B.MOE_PHASE_DECODE
+    variant = {"large": B.MOE_GEMM_LARGE_M, "small": B.MOE_GEMM_SMALL_M}.get(mode, B.MOE_GEMM_AUTO)
+    ctx = B.MoeContext(B.make_config(H, E, k, I, shared_I, T, phase, 0, variant, weight_format=B.MOE_WEIGHTS_FP8_E4M3))
+    if mode == "segments":
+        ctx.moe_ctx_set_segments(max(1, E // 3))
+    torch.cuda.synchronize()
+    out, bufs = ctx.layer_fp8(a["x"], a["logits"], a["bias"], w8)
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_OK
+    h = {n: (None if v is None else v.cpu().numpy()) for n, v in w8.items()}
+    ref = oracle.layer_fp8(wl.bits(a["x"]), np_f32(a["logits"]), np_f32(a["bias"]), k, h["wq_gate_up"], h["sw_gate_up"],
+                           h["wq_down"], h["sw_down"], h["wsq_gate_up"], h["sws_gate_up"], h["wsq_down"], h["sws_down"])
+    for name in ("topk_idx", "counts", "offsets", "perm", "inv_perm"):
+        assert np.array_equal(np_i32(bufs[name]).reshape(-1), np.asarray(ref[name]).reshape(-1)), name
+    e = layer_errors(out, ref["out"])
+    assert e["rel_l2"] <= 5e-3, e
+    ctx.close()
