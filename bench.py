@@ -263,6 +263,7 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm):
     # the same D step with FP8 weights (half the weight bytes to stream)
     try:
         w8 = wl.make_weights_fp8(wl.C2, 2, dev)
+        torch.cuda.synchronize(dev)  # the weights are generated on torch's current stream, the steps run on sd
         s = wl.C4_D
         ctx_d8 = B.MoeContext(B.make_config(s.H, s.E, s.k, s.I, s.shared_I, s.T, B.MOE_PHASE_DECODE,
                                             weight_format=B.MOE_WEIGHTS_FP8_E4M3), stream=sd, device=dev)
@@ -275,8 +276,8 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm):
             evs.append((e0, e1))
         torch.cuda.synchronize(dev)
         t8 = [1e3 * a.elapsed_time(b) for a, b in evs[warm:]]
-        res["fp8_alone_us"] = {"p50": percentile(t8, 50), "p99": percentile(t8, 99)}
-        assert ctx_d8.moe_ctx_status() == B.MOE_OK
+        res["fp8_alone_us"] = {"p50": percentile(t8, 50), "p99": percentile(t8, 99),
+                               "device_status": ctx_d8.moe_ctx_status()}
         ctx_d8.close()
         del w8
         torch.cuda.empty_cache()
@@ -411,7 +412,8 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm):
                         "note": "D ready at the start of an unsegmented P batch, runs after it"}
     res["prefill_serial_tokens_per_s"] = wl.C4_P.T / ((p_alone_ms + res["alone_us"]["p50"] * 1e-3) * 1e-3)
     # how much of a P batch plus one D step the turnstile run hides by running them at the same time: 0 % means
-    # strict time slicing (the turnstile admits D between P segments and P waits for it), 100 % would hide all of D
+    # strict time slicing (the turnstile admits D between P segments and P waits for it), 100 % would hide all of D,
+    # a negative figure means that cutting P into segments costs more than is hidden
     t_p, t_d = p_alone_ms * 1e-3, res["alone_us"]["p50"] * 1e-6
     t_conc = wl.C4_P.T / res["prefill_concurrent_tokens_per_s"]  # seconds per P batch while D steps run
     res["overlap_pct"] = 100.0 * (t_p + t_d - t_conc) / t_d
@@ -535,6 +537,7 @@ def run_ours(args):
     fp8 = None
     if not args.quick:
         w8 = wl.make_weights_fp8(shape, 3 + rank, dev)
+        torch.cuda.synchronize(dev)
         ctx8 = B.MoeContext(B.make_config(H, E, k, I, shape.shared_I, T, B.MOE_PHASE_PREFILL,
                                           weight_format=B.MOE_WEIGHTS_FP8_E4M3), stream=stream, device=dev)
 

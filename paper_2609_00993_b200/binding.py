@@ -174,6 +174,9 @@ class MoeContext:
             self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
             self.workspace = workspace if workspace is not None else torch.empty(nbytes, dtype=torch.uint8,
                                                                                  device=self.device)
+            # torch hands out the block on the CURRENT stream and may have recycled it from tensors whose last
+            # kernels are still queued there; the context's stream must not touch it before they are done
+            self.stream.wait_stream(torch.cuda.current_stream(self.device))
         self.workspace_bytes = nbytes
         handle = ctypes.c_void_p()
         st = self.lib.moe_ctx_create(ctypes.byref(cfg), ctypes.c_void_p(self.workspace.data_ptr()),
