@@ -338,13 +338,28 @@ class MoeContext:
         off = p.value - self.workspace.data_ptr()
         return self.workspace[off:off + n * esz].view(dtype).view(*shape)
 
+    def _step_tensors(self, T, k, E, device, bufs, out):
+        """Allocates the step's arrays and output when the caller passes none.  torch allocates on its current
+        stream; when the context runs on another one, that stream first waits for the current one (a recycled
+        block may still be written there) and the tensors are marked as in use on the context's stream."""
+        fresh = []
+        if bufs is None:
+            bufs = alloc_step_buffers(T, k, E, device)
+            fresh += list(bufs.values())
+        if out is None:
+            out = torch.empty(T, self.cfg.hidden, dtype=torch.bfloat16, device=device)
+            fresh.append(out)
+        cur = torch.cuda.current_stream(self.device)
+        if fresh and cur != self.stream:
+            self.stream.wait_stream(cur)
+            for t in fresh:
+                t.record_stream(self.stream)
+        return bufs, out
+
     # -- convenience: one whole step on device tensors (calls the four entry points in order)
     def layer(self, x, logits, select_bias, w_gate_up, w_down, ws_gate_up=None, ws_down=None, out=None, bufs=None):
         T, k, E = x.shape[0], self.cfg.top_k, self.cfg.n_experts
-        if bufs is None:
-            bufs = alloc_step_buffers(T, k, E, x.device)
-        if out is None:
-            out = torch.empty(T, self.cfg.hidden, dtype=torch.bfloat16, device=x.device)
+        bufs, out = self._step_tensors(T, k, E, x.device, bufs, out)
         self.moe_route(logits, select_bias, bufs["topk_idx"], bufs["topk_w"], T=T)
         self.moe_dispatch_layout(bufs["topk_idx"], x, bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"],
                                  T=T)
@@ -356,10 +371,7 @@ class MoeContext:
         """One step with FP8 weights; `w8` holds wq_gate_up, sw_gate_up, wq_down, sw_down and, with a shared
         expert, wsq_gate_up, sws_gate_up, wsq_down, sws_down (see workloads.make_weights_fp8)."""
         T, k, E = x.shape[0], self.cfg.top_k, self.cfg.n_experts
-        if bufs is None:
-            bufs = alloc_step_buffers(T, k, E, x.device)
-        if out is None:
-            out = torch.empty(T, self.cfg.hidden, dtype=torch.bfloat16, device=x.device)
+        bufs, out = self._step_tensors(T, k, E, x.device, bufs, out)
         self.moe_route(logits, select_bias, bufs["topk_idx"], bufs["topk_w"], T=T)
         self.moe_dispatch_layout(bufs["topk_idx"], x, bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"],
                                  T=T)
