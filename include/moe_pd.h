@@ -107,7 +107,9 @@ size_t moe_ctx_workspace_bytes(const moe_config* cfg);
  * allocated (256-byte aligned) and keeps alive until moe_ctx_destroy.  The range is
  * registered process-wide: a range overlapping a live context's, or a stream already bound
  * to a live context of the other phase, is refused with MOE_ERR_STATE (construction
- * validates isolation before any kernel runs).  Enqueues one memset on the stream. */
+ * validates isolation before any kernel runs).  Enqueues one memset on the stream; if the workspace was
+ * allocated or last used on another stream (a stream-ordered or caching allocator may hand out a block that
+ * still has work pending there), order the two streams before this call. */
 moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspace_bytes, void* cuda_stream,
                           moe_ctx** out);
 
