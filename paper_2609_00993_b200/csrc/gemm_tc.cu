@@ -20,8 +20,8 @@
 // accumulator by the row's and the weight row's scale before SwiGLU / the bf16 store.
 // An expert's row tile may run past the end of its segment: TMA needs no alignment on the row coordinate, so
 // segments are NOT padded; rows that belong to the next expert are computed and simply not stored.  A last tile
-// of at most 32 rows fetches only a 32-row box of token rows (whatever else lies in the stage is multiplied and
-// dropped).
+// of at most 96 rows fetches only a 32-, 64- or 96-row box of token rows (whatever else lies in the stage is
+// multiplied and dropped).
 //
 // Warp roles (192 threads): warps 0-3 epilogue (TMEM lanes 32w..32w+31), warp 4 TMA producer, warp 5 MMA
 // issuer and TMEM owner.  The optional row-gather instantiation adds warps 6-9, which fetch the routed
@@ -215,11 +215,10 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 // Output tensor maps (large-M epilogue): [rows, n_feat] bf16 with boxes of 64 features x 32 rows, 128-byte swizzle
 struct OutMaps {
   CUtensorMap o, o2;
-  // large-M: the token rows again with 32-row boxes, for an expert's last tile when it holds at most 32 rows
-  // (the other 96 rows of the X tile are never stored, so nothing needs to be fetched for them)
-  CUtensorMap xs, xs2;
+  // large-M: the token rows again with 32-, 64- and 96-row boxes, for an expert's last tile when it holds no
+  // more rows than that (the other rows of the X tile are never stored, so nothing needs to be fetched for them)
+  CUtensorMap xs[3], xs2[3];
 };
-constexpr int kTailRows = 32;
 // Tiled bulk store shared -> global of one box, tracked in the issuing thread's bulk groups
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src_smem, int c0, int c1) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src_smem),
@@ -415,13 +414,14 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         const CUtensorMap* mx = t.dense ? &map_x2 : &map_x;
         const int w_e = t.dense ? 0 : p.e_base + t.e;
         const int num_kb = t.dense ? num_kb2 : num_kb1;
-        const bool short_x = !SWAP && !GATHER && t.rows <= kTailRows;
-        const CUtensorMap* mxs = t.dense ? &omaps.xs2 : &omaps.xs;
+        const uint32_t x_rows = (uint32_t)((t.rows + 31) & ~31);  // rows worth fetching, in steps of 32
+        const bool short_x = !SWAP && !GATHER && x_rows < 128u;
+        const CUtensorMap* mxs = (t.dense ? omaps.xs2 : omaps.xs) + (short_x ? x_rows / 32u - 1u : 0u);
         for (int kb = 0, k0 = 0; kb < num_kb; ++kb, k0 += kbk) {
           if (!mbar_wait(bar_empty + 8u * ring.stage, ring.phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t full = bar_full + 8u * ring.stage;
           const uint32_t st = base_addr + ring.stage * (uint32_t)stage_bytes;
-          mbar_expect_tx(full, GATHER ? 2u * kWBoxBytes : (short_x ? 2u * kWBoxBytes + kTailRows * 128u : (uint32_t)stage_bytes));
+          mbar_expect_tx(full, GATHER ? 2u * kWBoxBytes : (short_x ? 2u * kWBoxBytes + x_rows * 128u : (uint32_t)stage_bytes));
           tma_load_3d(st, mw, full, k0, w_row0, w_e);
           tma_load_3d(st + kWBoxBytes, mw, full, k0, w_row1, w_e);
           if (!GATHER) tma_load_2d(st + 2 * kWBoxBytes, short_x ? mxs : mx, full, k0, t.row0);
@@ -833,18 +833,22 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bo
       if (!encode_map(&om.o2, dense->out, 2, d2, st2, bx2)) return cudaErrorInvalidValue;
     }
   }
-  om.xs = mx;
-  om.xs2 = mx2;
+  for (int m = 0; m < 3; ++m) {
+    om.xs[m] = mx;
+    om.xs2[m] = mx2;
+  }
   if (!swap_ab && !gather) {
-    const uint64_t dims[2] = {(uint64_t)p.K, (uint64_t)p.rows_bound};
-    const uint64_t str[1] = {(uint64_t)p.K * esz};
-    const uint32_t box[2] = {box_k, (uint32_t)kTailRows};
-    if (!encode_map(&om.xs, p.A, 2, dims, str, box, fp8)) return cudaErrorInvalidValue;
-    om.xs2 = om.xs;
-    if (dense != nullptr) {
-      const uint64_t dx[2] = {(uint64_t)dense->K, (uint64_t)dense->rows};
-      const uint64_t sx[1] = {(uint64_t)dense->K * esz};
-      if (!encode_map(&om.xs2, dense->A, 2, dx, sx, box, fp8)) return cudaErrorInvalidValue;
+    for (int m = 0; m < 3; ++m) {
+      const uint64_t dims[2] = {(uint64_t)p.K, (uint64_t)p.rows_bound};
+      const uint64_t str[1] = {(uint64_t)p.K * esz};
+      const uint32_t box[2] = {box_k, (uint32_t)(32 * (m + 1))};
+      if (!encode_map(&om.xs[m], p.A, 2, dims, str, box, fp8)) return cudaErrorInvalidValue;
+      om.xs2[m] = om.xs[m];
+      if (dense != nullptr) {
+        const uint64_t dx[2] = {(uint64_t)dense->K, (uint64_t)dense->rows};
+        const uint64_t sx[1] = {(uint64_t)dense->K * esz};
+        if (!encode_map(&om.xs2[m], dense->A, 2, dx, sx, box, fp8)) return cudaErrorInvalidValue;
+      }
     }
   }
   TcParams prm;
