@@ -18,6 +18,9 @@
  *   - Calls validate on the host, enqueue kernels on the context's stream and return.
  *     They do not synchronise, allocate device memory or read device memory back
  *     (except `moe_ctx_status`, `moe_ctx_destroy`, `moe_layer_host` and `moe_layer_host_wait`, which say so).
+ *   - Host threads: calls on ONE context must not overlap in time (a context is not locked; give each phase's
+ *     context to one thread, or serialise).  Calls on different contexts, creation and destruction included,
+ *     may run concurrently from different threads; the turnstile controller is thread-safe by itself.
  *   - Every function returns a `moe_status`; no exception crosses the boundary.
  *     `moe_last_error` gives a human-readable reason for the last failure on a context.
  *   - Problems only the device can see (an expert index outside [0,E), a bounded wait
