@@ -92,3 +92,23 @@ def sample_tokens(T, counts, offsets, perm, k, n, seed=0):
             toks.add(int(perm[offsets[e]] // k))
             toks.add(int(perm[offsets[e + 1] - 1] // k))
     return sorted(toks)
+
+
+def check_against_storage_precision(out_gpu, out_ref, out_emul, label=""):
+    """The GPU result is as accurate as the specified storage precisions allow: its error against the unrounded
+    oracle is compared with that of the oracle's own bf16-storage emulation (activation, expert outputs and layer
+    output rounded to bf16 where a bf16 pipeline stores them) and with the rounding of the exact result alone."""
+    g = np_f32(out_gpu).astype(np.float64)
+    r = np.asarray(out_ref, np.float64)
+    m = np.asarray(out_emul, np.float64)
+    r_bf16 = torch.from_numpy(np.asarray(out_ref, np.float32)).to(torch.bfloat16).double().numpy()
+    m_bf16 = torch.from_numpy(np.asarray(out_emul, np.float32)).to(torch.bfloat16).double().numpy()  # + the output's own rounding
+    floor_round = float(np.abs(r_bf16 - r).max())
+    floor_emul = float(np.abs(m_bf16 - r).max())
+    rel_emul = float(np.linalg.norm(m_bf16 - r) / max(np.linalg.norm(r), 1e-30))
+    max_abs = float(np.abs(g - r).max())
+    rel = float(np.linalg.norm(g - r) / max(np.linalg.norm(r), 1e-30))
+    print(f"[storage floors {label}] gpu max_abs={max_abs:.4g} rel_l2={rel:.4g} | bf16 of the exact result: "
+          f"{floor_round:.4g} | bf16-storage emulation: max_abs={floor_emul:.4g} rel_l2={rel_emul:.4g}")
+    assert max_abs <= 1.5 * floor_emul, f"{label}: max abs {max_abs} against emulation floor {floor_emul}"
+    assert rel <= 1.1 * rel_emul, f"{label}: rel L2 {rel} against emulation {rel_emul}"

@@ -9,7 +9,8 @@ import pytest
 import torch
 
 import oracle
-from helpers import (check_layer, check_topk_w, np_f32, np_i32, oracle_tokens_from_device, sample_tokens)
+from helpers import (check_against_storage_precision, check_layer, check_topk_w, np_f32, np_i32,
+                     oracle_tokens_from_device, sample_tokens)
 from paper_2609_00993_b200 import binding as B
 from paper_2609_00993_b200 import workloads as wl
 
@@ -104,6 +105,9 @@ def test_c2_decode_v3_shaped(v3_weights):
     toks = sample_tokens(shape.T, counts, offsets, perm, shape.k, 12, seed=2)
     ref, mag = oracle_tokens_from_device(a["x"], bufs["topk_idx"], bufs["topk_w"], v3_weights, toks)
     check_layer(out[toks], ref, mag, literal=False, label="C2")
+    emul = oracle_tokens_from_device(a["x"], bufs["topk_idx"], bufs["topk_w"], v3_weights, toks, want_term_abs=False,
+                                     emulate_bf16=True)
+    check_against_storage_precision(out[toks], ref, emul, label="C2")
     # a second step lands in the other buffer set of the D context and gives the same bits
     out2, _ = _step(ctx, a, v3_weights)
     assert torch.equal(out, out2)
@@ -145,6 +149,9 @@ def test_c4_prefill_and_decode_contexts_concurrently(v3_weights):
         toks = sample_tokens(shape.T, counts, offsets, perm, shape.k, 6, seed=4)
         ref, mag = oracle_tokens_from_device(a["x"], bufs["topk_idx"], bufs["topk_w"], w, toks)
         check_layer(out[toks], ref, mag, literal=False, label=name)
+        emul = oracle_tokens_from_device(a["x"], bufs["topk_idx"], bufs["topk_w"], w, toks, want_term_abs=False,
+                                         emulate_bf16=True)
+        check_against_storage_precision(out[toks], ref, emul, label=name)
     ctx_p.close(); ctx_d.close()
 
 
