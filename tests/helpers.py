@@ -36,7 +36,9 @@ def layer_errors(out_gpu, out_ref, term_abs=None):
     g = np_f32(out_gpu).astype(np.float64)
     r = np.asarray(out_ref, np.float64)
     d = g - r
-    res = {"max_abs": float(np.abs(d).max()) if d.size else 0.0,
+    tok_rel = (np.linalg.norm(d, axis=-1) / np.maximum(np.linalg.norm(r, axis=-1), 1e-30)) if d.ndim == 2 and d.size else np.zeros(1)
+    res = {"worst_token_rel_l2": float(tok_rel.max()),
+           "max_abs": float(np.abs(d).max()) if d.size else 0.0,
            "rel_l2": float(np.linalg.norm(d) / max(np.linalg.norm(r), 1e-30)) if d.size else 0.0,
            "frac_gt": float((np.abs(d) > MAX_ABS).mean()) if d.size else 0.0}
     if term_abs is not None:
@@ -46,9 +48,11 @@ def layer_errors(out_gpu, out_ref, term_abs=None):
 
 def check_layer(out_gpu, out_ref, term_abs=None, literal=True, label=""):
     e = layer_errors(out_gpu, out_ref, term_abs)
-    print(f"[parity {label}] max_abs={e['max_abs']:.4g} rel_l2={e['rel_l2']:.4g} frac>2e-2={e['frac_gt']:.3g}"
+    print(f"[parity {label}] max_abs={e['max_abs']:.4g} rel_l2={e['rel_l2']:.4g} worst token rel_l2={e['worst_token_rel_l2']:.4g} "
+          f"frac>2e-2={e['frac_gt']:.3g}"
           + (f" scaled_max={e['scaled_max']:.4g}" if "scaled_max" in e else ""))
     assert e["rel_l2"] <= REL_L2_MAX, f"{label}: rel L2 {e['rel_l2']}"
+    assert e["worst_token_rel_l2"] <= REL_L2_MAX, f"{label}: worst token rel L2 {e['worst_token_rel_l2']}"
     if literal:
         assert e["max_abs"] <= MAX_ABS, f"{label}: max abs {e['max_abs']}"
     else:
