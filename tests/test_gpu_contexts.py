@@ -423,3 +423,54 @@ ctx.close()
     assert r.returncode == 0, r.stderr[-2000:]
     assert f"STATUS {B.MOE_ERR_TIMEOUT}" in r.stdout and f"STATUS_AFTER_READ {B.MOE_OK}" in r.stdout
     assert "ALIVE 8.0" in r.stdout
+
+
+@pytest.mark.parametrize("phase,fmt", [(B.MOE_PHASE_PREFILL, B.MOE_WEIGHTS_BF16), (B.MOE_PHASE_DECODE, B.MOE_WEIGHTS_BF16),
+                                       (B.MOE_PHASE_PREFILL, B.MOE_WEIGHTS_FP8_E4M3), (B.MOE_PHASE_DECODE, B.MOE_WEIGHTS_FP8_E4M3)])
+def test_nothing_is_written_outside_the_workspace_and_the_callers_arrays(phase, fmt):
+    """Guard bands of a known pattern on both sides of the workspace and of every array the caller passes must
+    survive whole steps (ragged T, shared expert, segments on the prefill side): no kernel writes out of bounds."""
+    T, H, E, k, I, Is = 333, 320, 11, 3, 192, 128
+    shape = wl.LayerShape("g", T=T, H=H, E=E, k=k, I=I, shared_I=Is, select_bias=True)
+    cfg = B.make_config(H, E, k, I, Is, T, phase, weight_format=fmt)
+    nbytes = B.moe_ctx_workspace_bytes(cfg)
+    guard = 4096
+    pattern = 0xA5
+
+    def guarded(n_bytes):
+        raw = torch.full((n_bytes + 2 * guard,), pattern, dtype=torch.uint8, device=DEV)
+        return raw, raw[guard:guard + n_bytes]
+
+    raw_ws, ws = guarded((nbytes + 255) // 256 * 256)
+    N = T * k
+    raws = {}
+    views = {}
+    for name, n_el, dt in (("topk_idx", N, torch.int32), ("topk_w", N, torch.float32), ("counts", E, torch.int32),
+                           ("offsets", E + 1, torch.int32), ("perm", N, torch.int32), ("inv_perm", N, torch.int32),
+                           ("out", T * H, torch.bfloat16)):
+        esz = torch.empty(0, dtype=dt).element_size()
+        nb = (n_el * esz + 255) // 256 * 256
+        raws[name], v = guarded(nb)
+        views[name] = v[:n_el * esz].view(dt)
+    bufs = {"topk_idx": views["topk_idx"].view(T, k), "topk_w": views["topk_w"].view(T, k), "counts": views["counts"],
+            "offsets": views["offsets"], "perm": views["perm"], "inv_perm": views["inv_perm"]}
+    out = views["out"].view(T, H)
+    a = wl.make_activations(shape, 5, DEV)
+    torch.cuda.synchronize()
+    ctx = B.MoeContext(cfg, workspace=ws)
+    for seg in (0, 4):
+        if phase == B.MOE_PHASE_PREFILL:
+            ctx.moe_ctx_set_segments(seg)
+        for _ in range(2):  # a decode context visits both of its buffer sets
+            if fmt == B.MOE_WEIGHTS_FP8_E4M3:
+                ctx.layer_fp8(a["x"], a["logits"], a["bias"], wl.make_weights_fp8(shape, 6, DEV), out=out, bufs=bufs)
+            else:
+                w = wl.make_weights(shape, 6, DEV)
+                ctx.layer(a["x"], a["logits"], a["bias"], w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"],
+                          out=out, bufs=bufs)
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_OK
+    for name, raw in [("workspace", raw_ws)] + list(raws.items()):
+        assert bool((raw[:guard] == pattern).all()) and bool((raw[-guard:] == pattern).all()), f"{name}: guard band overwritten"
+    assert torch.isfinite(out.float()).all()
+    ctx.close()
