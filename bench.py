@@ -240,6 +240,15 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm):
     time_d(warm)
     alone = time_d(iters)
     res["alone_us"] = {"p50": percentile(alone, 50), "p99": percentile(alone, 99), "max": max(alone)}
+    # the same step as the host sees it: from the first enqueue to the end of a stream synchronisation
+    wall = []
+    for i in range(max(20, iters // 4)):
+        t0 = time.perf_counter()
+        with torch.cuda.stream(sd):
+            d_step(i)
+        sd.synchronize()
+        wall.append(1e6 * (time.perf_counter() - t0))
+    res["alone_host_wall_us"] = {"p50": percentile(wall, 50), "p99": percentile(wall, 99)}
 
     # the same D step replayed from a CUDA graph (stable phase-owned addresses): launch overhead off the path
     try:
