@@ -146,3 +146,39 @@ def test_fp8_layer_stays_within_the_quantisation_error_of_the_bf16_layer():
     # E4M3 keeps 3 mantissa bits: rounding error uniform within half a step is ~2.6 % rms per operand, ~3.7 % per
     # product and (random signs) per dot product, ~5.5 % after silu(g) * u, ~6.6 % after the second quantised GEMM
     assert 3e-2 < rel < 1e-1, rel
+
+
+def _read_fp8_golden():
+    import os
+    vals = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "fp8_hand_example.txt")) as fh:
+        for line in fh:
+            line = line.split("#")[0].strip()
+            if "=" in line:
+                name, rhs = line.split("=")
+                vals[name.strip()] = [int(v, 16) if v.lower().startswith("0x") else float(v) for v in rhs.split()]
+    return vals
+
+
+def test_hand_derived_fp8_example():
+    """tests/golden/fp8_hand_example.txt: rows quantised by hand (exact codes, a rounding case, both tie cases, the
+    all-zero row) and one expert followed through GEMM1, SwiGLU, the bf16 store, the re-quantisation and GEMM2."""
+    g = _read_fp8_golden()
+    rows = np.array(g["rows"], np.float32).reshape(4, 4)
+    bits = _bf16_bits(rows)
+    assert np.array_equal(oracle.bf16_to_f32(bits), rows)  # the example's inputs are bf16 values
+    q, s = oracle.quantize_rows(bits)
+    assert [int(c) for c in q.reshape(-1)] == g["codes"]
+    assert np.array_equal(s, np.array(g["scales"], np.float64).astype(np.float32))
+    wq1 = np.array(g["gate_up_codes"], np.uint8).reshape(2, 4)
+    sw1 = np.array(g["gate_up_scale"], np.float32)
+    act = oracle.gemm1_fp8(q[:1], s[:1], wq1, sw1)
+    assert [int(v) for v in act.reshape(-1)] == g["act_bf16"]
+    aq, sa = oracle.quantize_rows(act)
+    assert int(aq[0, 0]) == 0xFE and sa[0] == np.float32(0.453125) / np.float32(448.0)
+    wq2 = np.array(g["down_codes"], np.uint8).reshape(4, 1)
+    sw2 = np.array(g["down_scale"], np.float32)
+    y = oracle.gemm2_fp8(aq, sa, wq2, sw2)
+    assert np.allclose(y[0], np.array(g["y"], np.float64), rtol=1e-6, atol=0)
+    y_all = oracle.ffn_fp8(bits[:1], wq1, sw1, wq2, sw2)
+    assert np.array_equal(y_all, y)
