@@ -347,3 +347,73 @@ def test_layer_hand_derived_example():
             0.5 * sm1 + 0.5 * (0.5 * 2 * s1), 0.5 * sm1,
             sig(1.0) * (2 * s1) + sig(-1.0) * (0.5 * s2), sig(1.0) * (-s1)]
     assert np.allclose(gold["out"], want, rtol=1e-12)
+    # the term magnitude A = sum_j |w_j y_j| and the bf16-storage emulation, both from the same hand derivation
+    out, mag = oracle.layer_tokens(_bf16_bits(x), r["topk_idx"], r["topk_w"], _bf16_bits(wgu), _bf16_bits(wd),
+                                   want_term_abs=True)
+    assert np.allclose(out.ravel(), gold["out"], rtol=1e-6)
+    assert np.allclose(mag.ravel(), gold["term_abs"], rtol=1e-6)
+    want_mag = [0.5 * 4 * s1 + 0.5 * 3 * s2, 0.5 * 2 * s1 + 0.5 * 3 * s2, 0.5 * -sm1 + 0.5 * s1, 0.5 * -sm1,
+                sig(1.0) * 2 * s1 + sig(-1.0) * 0.5 * s2, sig(1.0) * s1]
+    assert np.allclose(gold["term_abs"], want_mag, rtol=1e-12)
+    assert not np.allclose(gold["term_abs"], np.abs(gold["out"]), rtol=1e-3)  # mixed signs: A is not |out|
+    emu = oracle.layer_tokens(_bf16_bits(x), r["topk_idx"], r["topk_w"], _bf16_bits(wgu), _bf16_bits(wd),
+                              emulate_bf16=True)
+    assert np.allclose(emu.ravel(), gold["out_bf16_storage"], rtol=1e-6)
+    staged = oracle.layer(_bf16_bits(x), logits, None, 2, _bf16_bits(wgu), _bf16_bits(wd), emulate_bf16=True)
+    assert np.allclose(staged["out"].ravel(), gold["out_bf16_storage"], rtol=1e-6)
+    assert not np.allclose(gold["out_bf16_storage"], gold["out"], rtol=1e-4)  # the rounding of a bites
+
+
+def _bf16_round(v):
+    """Round to nearest even onto 8 significant bits with torch's own bfloat16 (a library routine)."""
+    return float(torch.tensor(v, dtype=torch.float64).to(torch.float32).to(torch.bfloat16).double())
+
+
+def test_layer_hand_derived_example_with_shared_expert():
+    """tests/golden/hand_example_shared.txt: a shared expert, down weights that make an expert output's bf16
+    rounding bite, the term magnitude A including |y_shared|, and the bf16-storage emulation of all three."""
+    gold = _read_golden(os.path.join(GOLDEN, "hand_example_shared.txt"))
+    x = torch.tensor(gold["x"].reshape(2, 2), dtype=torch.float32)
+    logits = gold["logits"].reshape(2, 3).astype(np.float32)
+    wgu = torch.tensor(gold["w_gate_up"].reshape(3, 2, 2), dtype=torch.float32)
+    wd = torch.tensor(gold["w_down"].reshape(3, 2, 1), dtype=torch.float32)
+    wsgu = torch.tensor(gold["ws_gate_up"].reshape(2, 2), dtype=torch.float32)
+    wsd = torch.tensor(gold["ws_down"].reshape(2, 1), dtype=torch.float32)
+    args = (_bf16_bits(x), logits, None, 2, _bf16_bits(wgu), _bf16_bits(wd), _bf16_bits(wsgu), _bf16_bits(wsd))
+    r = oracle.layer(*args)
+    assert np.array_equal(r["topk_idx"].ravel(), gold["topk_idx"].astype(np.int32))
+    assert np.allclose(r["topk_w"].ravel(), gold["topk_w"], rtol=1e-6)
+    assert np.allclose(r["out"].ravel(), gold["out"], rtol=1e-6)
+    out, mag = oracle.layer_tokens(args[0], r["topk_idx"], r["topk_w"], args[4], args[5], args[6], args[7],
+                                   want_term_abs=True)
+    assert np.allclose(out.ravel(), gold["out"], rtol=1e-6)
+    assert np.allclose(mag.ravel(), gold["term_abs"], rtol=1e-6)
+    emu, emag = oracle.layer_tokens(args[0], r["topk_idx"], r["topk_w"], args[4], args[5], args[6], args[7],
+                                    emulate_bf16=True, want_term_abs=True)
+    assert np.allclose(emu.ravel(), gold["out_bf16_storage"], rtol=1e-6)
+    assert np.allclose(emag.ravel(), gold["term_abs_bf16_storage"], rtol=1e-6)
+    assert np.allclose(oracle.layer(*args, emulate_bf16=True)["out"].ravel(), gold["out_bf16_storage"], rtol=1e-6)
+
+    # the stored values again, from the closed forms of the derivation (no oracle code involved)
+    sig = lambda z: 1.0 / (1.0 + math.exp(-z))
+    silu = lambda z: z * sig(z)
+    w0 = (sig(1.0), sig(-1.0))
+
+    def rows(rnd):
+        ffn = lambda g, u, down: [rnd(rnd(silu(g) * u) * d) for d in down]
+        t0 = (w0, ffn(2, 3, (1, 3)), ffn(3, 1, (0.5, -3)), ffn(-1, 2, (-1, 0.5)))
+        t1 = ((0.5, 0.5), ffn(2, -1, (3, -1)), ffn(1, 2, (0.5, -3)), ffn(3, -1, (-1, 0.5)))
+        out = [w[0] * ya[c] + w[1] * yb[c] + ys[c] for (w, ya, yb, ys) in (t0, t1) for c in range(2)]
+        mag = [abs(w[0] * ya[c]) + abs(w[1] * yb[c]) + abs(ys[c]) for (w, ya, yb, ys) in (t0, t1) for c in range(2)]
+        return out, mag
+
+    out_x, mag_x = rows(lambda v: v)
+    out_r, mag_r = rows(_bf16_round)
+    assert np.allclose(gold["out"], out_x, rtol=1e-12) and np.allclose(gold["term_abs"], mag_x, rtol=1e-12)
+    assert np.allclose(gold["out_bf16_storage"], out_r, rtol=1e-12)
+    assert np.allclose(gold["term_abs_bf16_storage"], mag_r, rtol=1e-12)
+    # plausible mistakes in A are far outside the pin: dropped shared term, unweighted terms, doubled
+    no_shared = [abs(w0[0] * 3 * silu(2)) + abs(w0[1] * 0.5 * silu(3))]
+    assert abs(gold["term_abs"][0] - no_shared[0]) > 0.1
+    # y = 3 a is not a power-of-two multiple: the rounding of y bites (15.84375 is a tie and goes to even, 15.875)
+    assert _bf16_round(3 * _bf16_round(3 * silu(2))) == 15.875
