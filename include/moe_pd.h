@@ -65,12 +65,17 @@ typedef enum {
   MOE_ERR_BAD_INDEX = 7    /* device: an expert index was outside [0, E)                  */
 } moe_status;
 
-/* GEMM kernel variants.  AUTO follows the phase: large-M for P, small-M for D. */
+/* GEMM kernel variants.  AUTO: a DECODE context uses small-M; a PREFILL context chooses per step from the
+ * step's rows per expert (T * top_k / n_experts <= 256: small-M, else large-M) -- a function of T alone, so a
+ * step captured in a CUDA graph replays the kernel it was captured with. */
 typedef enum {
   MOE_GEMM_AUTO = 0,
-  MOE_GEMM_LARGE_M = 1,  /* tokens fill the 128-row MMA dimension; tensor-bound at prefill sizes */
-  MOE_GEMM_SMALL_M = 2,  /* swap-AB: weight rows fill the MMA M dimension, an expert's few tokens
-                            sit in N; streams the weights once -- HBM-bound by design          */
+  MOE_GEMM_LARGE_M = 1,  /* tokens fill the 128-row MMA dimension; for experts of many hundreds of rows,
+                            where the pass is bound by the tensor cores                            */
+  MOE_GEMM_SMALL_M = 2,  /* swap-AB: weight rows fill the MMA M dimension, an expert's tokens sit in N
+                            (16..256 per tile, following the expert's row count), so each expert's
+                            weights enter an SM once per 256 tokens -- for experts of few rows, where
+                            the pass is bound by streaming the weights                             */
   MOE_GEMM_VALIDATION = 3 /* plain CUDA-core kernel, slow; exists to localise tensor-core bugs   */
 } moe_gemm_variant;
 
@@ -129,6 +134,18 @@ moe_status moe_ctx_destroy(moe_ctx* ctx);
  * set, so the abandoned step's buffers are written again only after one more whole step has been enqueued
  * behind them on the stream.  Enqueues nothing and does not synchronise. */
 moe_status moe_ctx_abandon_step(moe_ctx* ctx);
+
+/* Time limit of every bounded device-side wait of this context's kernels, in microseconds (0 restores the
+ * default of 2 s).  A wait that runs out makes the kernel record MOE_ERR_TIMEOUT in the status word and return
+ * (the paper's controller likewise detects protocol violations instead of waiting forever, Section "Rank-Aligned
+ * Segment Boundaries"); a service that prefers to fail fast on a wedged device sets a few milliseconds. */
+moe_status moe_ctx_set_wait_limit(moe_ctx* ctx, int64_t limit_us);
+
+/* Test hook of the failure-detection path (the paper has no counterpart): while enabled, the copy-issuing warp
+ * of this context's GEMM kernels issues nothing, so every consumer wait runs into the limit set by
+ * moe_ctx_set_wait_limit, the kernels report MOE_ERR_TIMEOUT through the status word, free their tensor
+ * memory and return.  The outputs of such a step are undefined.  Use a short limit with it. */
+moe_status moe_ctx_debug_inject_stall(moe_ctx* ctx, int32_t enabled);
 
 /* Synchronises the context's stream and returns the device status word (a moe_status:
  * MOE_OK, MOE_ERR_TIMEOUT or MOE_ERR_BAD_INDEX) in *device_status, then clears it. */

@@ -32,7 +32,8 @@ EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_
            "moe_ctx_debug_ptrs", "moe_ctx_debug_ptrs_fp8", "moe_ctx_launch_count", "moe_ctx_set_profiling", "moe_ctx_read_profile",
            "moe_dispatch_layout_static", "moe_ctx_set_segments", "moe_ctx_abandon_step", "moe_turnstile_create", "moe_turnstile_destroy",
            "moe_turnstile_set_span", "moe_turnstile_begin_epoch", "moe_turnstile_publish", "moe_turnstile_task_done",
-           "moe_turnstile_d_enter", "moe_turnstile_d_release", "moe_turnstile_state")
+           "moe_turnstile_d_enter", "moe_turnstile_d_release", "moe_turnstile_state", "moe_ctx_set_wait_limit",
+           "moe_ctx_debug_inject_stall")
 
 BOUNDARY_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32)
 
@@ -119,6 +120,10 @@ def load_library() -> ctypes.CDLL:
                        ("moe_turnstile_state", [vp, ctypes.POINTER(i64)] + [ctypes.POINTER(i32)] * 4)):
         getattr(lib, name).restype = i32
         getattr(lib, name).argtypes = args
+    lib.moe_ctx_set_wait_limit.restype = i32
+    lib.moe_ctx_set_wait_limit.argtypes = [vp, i64]
+    lib.moe_ctx_debug_inject_stall.restype = i32
+    lib.moe_ctx_debug_inject_stall.argtypes = [vp, i32]
     lib.moe_ctx_set_segments.restype = i32
     lib.moe_ctx_set_segments.argtypes = [vp, i32, BOUNDARY_FN, vp]
     lib.moe_dispatch_layout_static.restype = i32
@@ -231,6 +236,12 @@ class MoeContext:
 
     def moe_ctx_abandon_step(self):
         self._check(self.lib.moe_ctx_abandon_step(self.handle))
+
+    def moe_ctx_set_wait_limit(self, limit_us: int):
+        self._check(self.lib.moe_ctx_set_wait_limit(self.handle, int(limit_us)))
+
+    def moe_ctx_debug_inject_stall(self, enabled: bool):
+        self._check(self.lib.moe_ctx_debug_inject_stall(self.handle, int(bool(enabled))))
 
     def moe_ctx_launch_count(self) -> int:
         return int(self.lib.moe_ctx_launch_count(self.handle))

@@ -11,7 +11,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmoe_pd.so")
 OBJ_DIR = os.path.join(HERE, "build")
-SOURCES = ["ctx.cu", "route.cu", "layout.cu", "rows.cu", "gemm_validation.cu", "gemm_tc.cu", "quant.cu", "turnstile.cu"]
+SOURCES = ["ctx.cu", "route.cu", "layout.cu", "rows.cu", "gemm_validation.cu", "gemm_tc.cu", "gemm_stream.cu", "quant.cu", "turnstile.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
               "-Xptxas", "-v"]
 

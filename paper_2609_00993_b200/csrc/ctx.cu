@@ -185,6 +185,8 @@ struct moe_ctx {
   } slots[MOE_HOST_SLOTS];
   cudaStream_t h2d_stream, d2h_stream;
   bool host_pipeline;
+  unsigned long long wait_limit_ns;  // time limit of every bounded device-side wait (0 = the kernels' default)
+  bool debug_stall;                  // failure-detection hook: the GEMM producers issue no copies
   char err[256];
 };
 
@@ -265,24 +267,35 @@ int gemm_ctas(const moe_ctx* ctx) {
   return (ctx->cfg.sm_budget > 0 && ctx->cfg.sm_budget < ctx->n_sms) ? ctx->cfg.sm_budget : ctx->n_sms;
 }
 
-// Token tile of the small-M variant: the smallest power of two >= T, within [16, 128].
-int small_m_tile(int T) {
-  int t = 16;
-  while (t < T && t < 128) t <<= 1;
-  return t;
-}
+// Experts of up to this many rows on average go to the small-M (weight-streaming) variant: below it a pass is
+// bound by the bytes of weights the SMs take in, and the small-M kernel takes in the fewest (one tile of up to
+// 256 tokens per expert and feature tile); above it the pass is bound by the tensor cores and the large-M kernel's
+// double-buffered accumulators and bulk-store epilogue win.
+constexpr int64_t kSmallMRowsPerExpert = 256;
 
-int gemm_variant_of(const moe_ctx* ctx) {
+// AUTO: a DECODE context always streams; a PREFILL context chooses per step from the rows per expert of that
+// step's batch (T tokens): the choice is a function of T alone, so it is the same on every replay of a graph.
+int gemm_variant_of(const moe_ctx* ctx, int T) {
   const int v = ctx->cfg.gemm_variant;
-  return v != MOE_GEMM_AUTO ? v : (ctx->cfg.phase == MOE_PHASE_DECODE ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M);
+  if (v != MOE_GEMM_AUTO) return v;
+  if (ctx->cfg.phase == MOE_PHASE_DECODE) return MOE_GEMM_SMALL_M;
+  if (ctx->cfg.row_gather == 1) return MOE_GEMM_LARGE_M;  // only the large-M kernel gathers its rows itself
+  const int64_t rows = (int64_t)T * ctx->cfg.top_k;
+  return rows <= kSmallMRowsPerExpert * ctx->cfg.n_experts ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M;
 }
 
 // GEMM1 gathers its rows itself only on the large-M tensor-core variant.
-bool gathers_rows(const moe_ctx* ctx) { return ctx->cfg.row_gather == 1 && gemm_variant_of(ctx) == MOE_GEMM_LARGE_M; }
+bool gathers_rows(const moe_ctx* ctx) {
+  const int v = ctx->cfg.gemm_variant;
+  return ctx->cfg.row_gather == 1 &&
+         (v == MOE_GEMM_LARGE_M || (v == MOE_GEMM_AUTO && ctx->cfg.phase == MOE_PHASE_PREFILL));
+}
 
 // `dense` (the shared expert's pass, or nullptr) rides in the same launch on the tensor-core path.
-cudaError_t run_gemm(moe_ctx* ctx, const moe::GemmProblem& p, const moe::GemmDenseGroup* dense, int T, int* n) {
-  const int variant = gemm_variant_of(ctx);
+cudaError_t run_gemm(moe_ctx* ctx, moe::GemmProblem p, const moe::GemmDenseGroup* dense, int T, int* n) {
+  const int variant = gemm_variant_of(ctx, T);
+  p.wait_limit_ns = ctx->wait_limit_ns;
+  p.debug_stall = ctx->debug_stall;
   if (variant == MOE_GEMM_VALIDATION) {
     cudaError_t e = moe::launch_gemm_validation(p, ctx->stream, n);
     if (e == cudaSuccess && dense != nullptr) {
@@ -292,9 +305,8 @@ cudaError_t run_gemm(moe_ctx* ctx, const moe::GemmProblem& p, const moe::GemmDen
     }
     return e;
   }
-  const bool swap = (variant == MOE_GEMM_SMALL_M);
-  return moe::launch_gemm_tc(p, dense, swap, swap ? small_m_tile(T) : 128, gemm_ctas(ctx), ctx->status, ctx->stream,
-                             n);
+  if (variant == MOE_GEMM_SMALL_M) return moe::launch_gemm_stream(p, dense, gemm_ctas(ctx), ctx->status, ctx->stream, n);
+  return moe::launch_gemm_tc(p, dense, gemm_ctas(ctx), ctx->status, ctx->stream, n);
 }
 
 }  // namespace
@@ -371,6 +383,8 @@ moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspa
   ctx->status = reinterpret_cast<int*>(ctx->ws);
   for (int s = 0; s < l.n_sets; ++s) carve_set(*cfg, ctx->ws + kStatusBlock + (size_t)s * l.set_bytes, &ctx->sets[s]);
   ctx->host_pipeline = false;
+  ctx->wait_limit_ns = 0;
+  ctx->debug_stall = false;
   const size_t staging_bytes = carve_staging(*cfg, nullptr, nullptr);
   for (int s = 0; s < MOE_HOST_SLOTS; ++s) {
     BufferSet st = ctx->sets[s < l.n_sets ? s : 0];
@@ -540,11 +554,11 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
   if (e == cudaSuccess && x != nullptr && fp8) {
     StageTimer tm(ctx, 2);
     e = moe::launch_permute(b.xq_tok, ctx->inv_perm, b.xq, T, ctx->cfg.top_k, ctx->cfg.hidden / 2, ctx->status,
-                            ctx->stream, &n, b.sx_tok, b.sx);
+                            ctx->stream, &n, b.sx_tok, b.sx, ctx->wait_limit_ns);
   } else if (e == cudaSuccess && x != nullptr && !gathers_rows(ctx)) {
     StageTimer tm(ctx, 2);
     e = moe::launch_permute(x, ctx->inv_perm, b.x_perm, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->status, ctx->stream,
-                            &n);
+                            &n, nullptr, nullptr, ctx->wait_limit_ns);
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_dispatch_layout");
   ctx->T = T;
@@ -749,7 +763,8 @@ moe_status moe_combine(moe_ctx* ctx, const float* topk_w, const int32_t* inv_per
   {
     StageTimer tm(ctx, 7);
     e = moe::launch_combine(b.y_perm, ctx->cfg.n_shared ? b.y_shared : nullptr, inv_perm ? inv_perm : ctx->inv_perm,
-                            topk_w, out, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->status, ctx->stream, &n);
+                            topk_w, out, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->status, ctx->stream, &n,
+                            ctx->wait_limit_ns);
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_combine");
   ctx->state = ST_IDLE;
@@ -872,6 +887,19 @@ moe_status moe_ctx_set_segments(moe_ctx* ctx, int32_t experts_per_segment, moe_b
   ctx->seg_experts = experts_per_segment;
   ctx->boundary_fn = fn;
   ctx->boundary_user = user;
+  return MOE_OK;
+}
+
+moe_status moe_ctx_set_wait_limit(moe_ctx* ctx, int64_t limit_us) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (limit_us < 0) return fail(ctx, MOE_ERR_INVALID_ARG, "limit_us < 0");
+  ctx->wait_limit_ns = (unsigned long long)limit_us * 1000ull;
+  return MOE_OK;
+}
+
+moe_status moe_ctx_debug_inject_stall(moe_ctx* ctx, int32_t enabled) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  ctx->debug_stall = enabled != 0;
   return MOE_OK;
 }
 

@@ -37,11 +37,13 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
 // ---- a5 permute, a9 combine ----------------------------------------------------------------
 // H counts 2-byte columns (a row of H E4M3 codes is H/2 of them).  row_val / row_val_perm (optional): one fp32
 // value per source row is copied to each of its destination rows.
+// wait_limit_ns: time limit of the kernels' bounded waits (0 = the default of 2 s).
 cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm, int T, int k, int H, int* status,
                            cudaStream_t stream, int* n_launches, const float* row_val = nullptr,
-                           float* row_val_perm = nullptr);
+                           float* row_val_perm = nullptr, unsigned long long wait_limit_ns = 0);
 cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32_t* inv_perm, const float* topk_w,
-                           void* out, int T, int k, int H, int* status, cudaStream_t stream, int* n_launches);
+                           void* out, int T, int k, int H, int* status, cudaStream_t stream, int* n_launches,
+                           unsigned long long wait_limit_ns = 0);
 
 // ---- a6-a8 grouped GEMM --------------------------------------------------------------------
 // One grouped GEMM pass:  out[r, :] = epilogue( A[r, :] . W[e]^T )  for r in expert e's segment.
@@ -72,6 +74,10 @@ struct GemmProblem {
   bool fp8 = false;
   const float* row_scale = nullptr;
   const float* w_scale = nullptr;
+  // Bounded waits of the tensor-core kernels: time limit in nanoseconds (0 = the default of 2 s), and the
+  // failure-detection hook (the TMA producer issues nothing, so every consumer wait runs into the limit).
+  unsigned long long wait_limit_ns = 0;
+  bool debug_stall = false;
 };
 
 // A dense group (the shared expert) that rides in the same launch as a grouped problem: its tiles are added
@@ -94,12 +100,16 @@ cudaError_t launch_quantize_rows(const void* x, int64_t rows, int n, void* q, fl
 
 cudaError_t launch_gemm_validation(const GemmProblem& p, cudaStream_t stream, int* n_launches);
 
-// Tensor-core path (tcgen05 + TMEM + TMA).  `swap_ab` selects the small-M variant; `row_tile` is the
-// token tile (128 for large-M; 16..128 for small-M); `max_ctas` caps the persistent grid.
-// Returns cudaErrorNotSupported for shapes it does not handle.
+// Tensor-core path (tcgen05 + TMEM + TMA), large-M variant: 128 tokens fill the MMA M dimension.  `max_ctas`
+// caps the persistent grid.  Returns cudaErrorNotSupported for shapes it does not handle.
 // `dense` (optional) is computed in the same launch with the same `gated` epilogue.
-cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, bool swap_ab, int row_tile,
-                           int max_ctas, int* status, cudaStream_t stream, int* n_launches);
+cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, int max_ctas, int* status,
+                           cudaStream_t stream, int* n_launches);
+// Weight-streaming variant (swap-AB with the MMA N following each expert's row count, up to 256 tokens per tile,
+// operands in a byte ring): the variant for experts of up to a few hundred rows, where the step is bound by the
+// bytes the SMs ingest.  Same contract as launch_gemm_tc; no row gather.
+cudaError_t launch_gemm_stream(const GemmProblem& p, const GemmDenseGroup* dense, int max_ctas, int* status,
+                               cudaStream_t stream, int* n_launches);
 // One-time driver entry-point lookup for tensor-map encoding; returns false (with a reason) if unavailable.
 bool gemm_tc_init(const char** why);
 

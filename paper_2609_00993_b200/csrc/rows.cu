@@ -9,6 +9,10 @@
 // Every mbarrier wait is bounded; on expiry the kernel records a timeout in the status word and stops.
 #include <cuda_bf16.h>
 
+#include <map>
+#include <mutex>
+#include <tuple>
+
 #include "kernels.h"
 
 namespace moe {
@@ -26,8 +30,8 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// Bounded wait: gives up after kWaitLimitNs of wall time (global timer, read every 256 polls).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait: gives up after limit_ns of wall time (global timer, read every 256 polls).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
   unsigned long long t0 = 0;
   for (uint32_t i = 0;; ++i) {
     uint32_t ok;
@@ -44,7 +48,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         unsigned long long now;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
         if (t0 == 0) t0 = now;
-        else if (now - t0 > kWaitLimitNs) return false;
+        else if (now - t0 > limit_ns) return false;
       }
       __nanosleep(64);
     }
@@ -69,6 +73,11 @@ __device__ __forceinline__ void bulk_wait_read() {
 __device__ __forceinline__ void flag_timeout(int* status) {
   if (status != nullptr) atomicCAS(status, kStOk, kStTimeout);
 }
+// After a wait has run out: copies this CTA issued may still be landing in its shared memory, so give them
+// time before the CTA exits and the memory is handed to the next one.
+__device__ __forceinline__ void linger_after_timeout() {
+  for (int i = 0; i < 64; ++i) __nanosleep(1000);
+}
 
 // ------------------------------------------------------------------------------------------- a5 permute
 constexpr int kPermuteSlots = 4;
@@ -80,7 +89,8 @@ constexpr int kPermuteChunkCols = 4096;  // bf16 columns per item: at most 8 KB 
 __global__ void __launch_bounds__(32)
 permute_rows_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ inv_perm,
                     __nv_bfloat16* __restrict__ x_perm, int T, int k, int H, int col_blocks, int slot_bytes,
-                    const float* __restrict__ row_val, float* __restrict__ row_val_perm, int* status) {
+                    const float* __restrict__ row_val, float* __restrict__ row_val_perm, int* status,
+                    unsigned long long wait_limit_ns) {
   extern __shared__ __align__(128) uint8_t smem[];
   const uint32_t slots = smem_u32(smem);
   const uint32_t bar_full = slots + (uint32_t)(kPermuteSlots * slot_bytes);
@@ -114,7 +124,7 @@ permute_rows_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restri
     const uint32_t s = (uint32_t)(n % kPermuteSlots), ph = (uint32_t)((n / kPermuteSlots) & 1);
     int dst_row = -1;
     if (lane < k) dst_row = __ldg(inv_perm + (size_t)t * k + lane);  // in flight while the row chunk arrives
-    ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8u * s, ph));
+    ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8u * s, ph, wait_limit_ns));
     if (!ok) break;
     if (dst_row >= 0) bulk_store(x_perm + (size_t)dst_row * H + c0, slots + s * (uint32_t)slot_bytes, bytes);
     bulk_commit();
@@ -125,7 +135,10 @@ permute_rows_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restri
     if (lane == 0 && n >= 1) issue_load(n - 1 + kPermuteSlots);
   }
   bulk_wait_read<0>();
-  if (!ok && lane == 0) flag_timeout(status);
+  if (!ok) {
+    if (lane == 0) flag_timeout(status);
+    linger_after_timeout();
+  }
 }
 
 // ------------------------------------------------------------------------------------------- a9 combine
@@ -152,7 +165,8 @@ template <int KT>
 __global__ void __launch_bounds__(kCombineThreads)
 combine_kernel(const __nv_bfloat16* __restrict__ y_perm, const __nv_bfloat16* __restrict__ y_shared,
                const int32_t* __restrict__ inv_perm, const float* __restrict__ topk_w, __nv_bfloat16* __restrict__ out,
-               int T, int k, int H, int col_blocks, int chunk_bytes, int stage_bytes, int n_stages, int* status) {
+               int T, int k, int H, int col_blocks, int chunk_bytes, int stage_bytes, int n_stages, int* status,
+               unsigned long long wait_limit_ns) {
   extern __shared__ __align__(128) uint8_t smem[];
   const uint32_t base = smem_u32(smem);
   const uint32_t bar_full = base + (uint32_t)(n_stages * stage_bytes);
@@ -185,7 +199,7 @@ combine_kernel(const __nv_bfloat16* __restrict__ y_perm, const __nv_bfloat16* __
         row = __ldg(inv_perm + (size_t)t * k + lane);
         wv = __ldg(topk_w + (size_t)t * k + lane);
       }
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8u * s, ph ^ 1u));
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8u * s, ph ^ 1u, wait_limit_ns));
       if (!ok) break;
       uint8_t* st = smem + (size_t)s * stage_bytes;
       const unsigned valid = __ballot_sync(0xffffffffu, row >= 0);
@@ -199,7 +213,10 @@ combine_kernel(const __nv_bfloat16* __restrict__ y_perm, const __nv_bfloat16* __
       if (row >= 0) bulk_load(dst + (uint32_t)(lane * chunk_bytes), y_perm + (size_t)row * H + c0, bytes, full);
       if (shared && lane == 0) bulk_load(dst + (uint32_t)(k * chunk_bytes), y_shared + (size_t)t * H + c0, bytes, full);
     }
-    if (!ok && lane == 0) flag_timeout(status);
+    if (!ok) {
+      if (lane == 0) flag_timeout(status);
+      linger_after_timeout();
+    }
   } else {
     // ============================================================ consumer warps: one 16-byte vector each
     bool ok = true;
@@ -209,7 +226,7 @@ combine_kernel(const __nv_bfloat16* __restrict__ y_perm, const __nv_bfloat16* __
       const int t = (int)(it / col_blocks), c0 = (int)(it % col_blocks) * kCombineChunkCols;
       const int cols = min(kCombineChunkCols, H - c0);
       const uint32_t s = (uint32_t)(n % n_stages), ph = (uint32_t)((n / n_stages) & 1);
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8u * s, ph));
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8u * s, ph, wait_limit_ns));
       if (!ok) break;
       const uint8_t* st = smem + (size_t)s * stage_bytes;
       const float* wts = reinterpret_cast<const float*>(st + meta_off);
@@ -236,23 +253,36 @@ combine_kernel(const __nv_bfloat16* __restrict__ y_perm, const __nv_bfloat16* __
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_empty + 8u * s);
     }
-    if (!ok && lane == 0) flag_timeout(status);
+    if (!ok) {
+      if (lane == 0) flag_timeout(status);
+      linger_after_timeout();
+    }
   }
 }
 
-// CTAs of `kern` that fit on the device at once (one resident wave for a persistent grid).
+// CTAs of `kern` that fit on the device at once (one resident wave for a persistent grid); looked up once per
+// kernel, device and shared-memory size, so that steady-state launches make no driver call besides the launch.
 int resident_ctas(const void* kern, int threads, size_t smem) {
-  int dev = 0, sms = 148, per_sm = 1;
+  static std::mutex mu;
+  static std::map<std::tuple<const void*, int, size_t>, int> known;
+  int dev = 0;
   cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
-  return sms * (per_sm > 0 ? per_sm : 1);
+  std::lock_guard<std::mutex> lock(mu);
+  int& v = known[std::make_tuple(kern, dev, smem)];
+  if (v == 0) {
+    int sms = 148, per_sm = 1;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
+    v = sms * (per_sm > 0 ? per_sm : 1);
+  }
+  return v;
 }
 
 }  // namespace
 
 cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm, int T, int k, int H, int* status,
-                           cudaStream_t stream, int* n_launches, const float* row_val, float* row_val_perm) {
+                           cudaStream_t stream, int* n_launches, const float* row_val, float* row_val_perm,
+                           unsigned long long wait_limit_ns) {
   if (T <= 0) return cudaSuccess;
   if (k > 32) return cudaErrorNotSupported;  // one storing lane per destination
   const int col_blocks = (H + kPermuteChunkCols - 1) / kPermuteChunkCols;
@@ -265,14 +295,16 @@ cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm,
   const int grid = (int)(n_items < cap ? n_items : cap);
   permute_rows_kernel<<<grid, 32, smem, stream>>>(static_cast<const __nv_bfloat16*>(x), inv_perm,
                                                   static_cast<__nv_bfloat16*>(x_perm), T, k, H, col_blocks, slot_bytes,
-                                                  row_val, row_val_perm, status);
+                                                  row_val, row_val_perm, status,
+                                                  wait_limit_ns ? wait_limit_ns : kWaitLimitNs);
   err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }
 
 cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32_t* inv_perm, const float* topk_w,
-                           void* out, int T, int k, int H, int* status, cudaStream_t stream, int* n_launches) {
+                           void* out, int T, int k, int H, int* status, cudaStream_t stream, int* n_launches,
+                           unsigned long long wait_limit_ns) {
   if (T <= 0) return cudaSuccess;
   if (k > 32) return cudaErrorNotSupported;  // one gathering lane per row
   const int col_blocks = (H + kCombineChunkCols - 1) / kCombineChunkCols;
@@ -290,7 +322,8 @@ cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32
     const int grid = (int)(n_items < cap ? n_items : cap);
     kern<<<grid, kCombineThreads, smem, stream>>>(
         static_cast<const __nv_bfloat16*>(y_perm), static_cast<const __nv_bfloat16*>(y_shared), inv_perm, topk_w,
-        static_cast<__nv_bfloat16*>(out), T, k, H, col_blocks, chunk_bytes, stage_bytes, stages, status);
+        static_cast<__nv_bfloat16*>(out), T, k, H, col_blocks, chunk_bytes, stage_bytes, stages, status,
+        wait_limit_ns ? wait_limit_ns : kWaitLimitNs);
     return cudaSuccess;
   };
   cudaError_t err = k == 8 ? launch(combine_kernel<8>) : k == 4 ? launch(combine_kernel<4>)

@@ -395,34 +395,32 @@ def test_turnstile_controller_drives_two_contexts_from_two_host_threads():
     p.close(); d.close()
 
 
-def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable():
-    """Failure detection without faulting the GPU: in a child process the GEMM's producer is told (on the host) to
-    issue nothing, so the consumers' bounded waits expire; the kernels return, the status word says
-    MOE_ERR_TIMEOUT (and is cleared by the read), the CUDA context is still alive and the MoE context closes."""
-    import subprocess
-    import sys
-    code = r"""
-import os, sys, torch
-sys.path.insert(0, os.getcwd())
-from paper_2609_00993_b200 import binding as B, workloads as wl
-shape = wl.LayerShape("t", T=64, H=256, E=8, k=2, I=128)
-w, a = wl.make_weights(shape, 1, "cuda"), wl.make_activations(shape, 2, "cuda")
-ctx = B.MoeContext(B.make_config(256, 8, 2, 128, 0, 64, B.MOE_PHASE_PREFILL))
-torch.cuda.synchronize()
-ctx.layer(a["x"], a["logits"], None, w["w_gate_up"], w["w_down"])
-torch.cuda.synchronize()
-print("STATUS", ctx.moe_ctx_status())
-print("STATUS_AFTER_READ", ctx.moe_ctx_status())
-t = torch.ones(4, device="cuda") * 2   # the CUDA context is alive
-print("ALIVE", float(t.sum().item()))
-ctx.close()
-"""
-    env = dict(os.environ, MOE_PD_INJECT_PRODUCER_STALL="1")
-    r = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, env=env, timeout=120,
-                       cwd=os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
-    assert r.returncode == 0, r.stderr[-2000:]
-    assert f"STATUS {B.MOE_ERR_TIMEOUT}" in r.stdout and f"STATUS_AFTER_READ {B.MOE_OK}" in r.stdout
-    assert "ALIVE 8.0" in r.stdout
+@pytest.mark.parametrize("variant", [B.MOE_GEMM_LARGE_M, B.MOE_GEMM_SMALL_M])
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(variant):
+    """Failure detection without faulting the GPU: the context is told (on the host) that its GEMM producers
+    issue nothing, so the consumers' bounded waits expire (after 20 ms here: a shared GPU is held for
+    milliseconds); the kernels return, the status word says MOE_ERR_TIMEOUT (and is cleared by the read), the
+    CUDA context is still alive, and with the hook off the very same context computes a correct step again."""
+    shape = wl.LayerShape("t", T=64, H=256, E=8, k=2, I=128)
+    w, a = wl.make_weights(shape, 1, DEV), wl.make_activations(shape, 2, DEV)
+    ctx = B.MoeContext(B.make_config(256, 8, 2, 128, 0, 64, B.MOE_PHASE_PREFILL, gemm_variant=variant), device=DEV)
+    torch.cuda.synchronize()
+    good, _ = ctx.layer(a["x"], a["logits"], None, w["w_gate_up"], w["w_down"])
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_OK
+    ctx.moe_ctx_set_wait_limit(20_000)
+    ctx.moe_ctx_debug_inject_stall(True)
+    ctx.layer(a["x"], a["logits"], None, w["w_gate_up"], w["w_down"])
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_ERR_TIMEOUT
+    assert ctx.moe_ctx_status() == B.MOE_OK          # the read cleared it
+    assert float((torch.ones(4, device=DEV) * 2).sum().item()) == 8.0   # the CUDA context is alive
+    ctx.moe_ctx_debug_inject_stall(False)
+    ctx.moe_ctx_set_wait_limit(0)
+    again, _ = ctx.layer(a["x"], a["logits"], None, w["w_gate_up"], w["w_down"])
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_OK and torch.equal(again, good)
+    ctx.close()
 
 
 @pytest.mark.parametrize("phase,fmt", [(B.MOE_PHASE_PREFILL, B.MOE_WEIGHTS_BF16), (B.MOE_PHASE_DECODE, B.MOE_WEIGHTS_BF16),

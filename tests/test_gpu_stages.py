@@ -173,7 +173,8 @@ def _oracle_step(a, w, k, emulate=False):
 VARIANTS = [(B.MOE_GEMM_VALIDATION, B.MOE_PHASE_PREFILL, "validation", 0),
             (B.MOE_GEMM_LARGE_M, B.MOE_PHASE_PREFILL, "large-M", 0),
             (B.MOE_GEMM_LARGE_M, B.MOE_PHASE_PREFILL, "large-M-gather", 1),  # GEMM1 gathers its rows; no x_perm
-            (B.MOE_GEMM_SMALL_M, B.MOE_PHASE_DECODE, "small-M", 0)]
+            (B.MOE_GEMM_SMALL_M, B.MOE_PHASE_DECODE, "small-M", 0),
+            (B.MOE_GEMM_SMALL_M, B.MOE_PHASE_PREFILL, "small-M-P", 0)]
 
 SHAPES = [
     # T,   H,    E,  k, I,   shared_I
@@ -181,6 +182,8 @@ SHAPES = [
     (300, 512, 16, 4, 192, 128),   # several row tiles, ragged tails, I not a multiple of 128, shared expert
     (33, 1024, 64, 8, 128, 0),     # a few rows per expert; some experts empty
     (700, 320, 4, 2, 64, 64),      # H not a multiple of 128/256: partial feature tiles; K = 320 (5 k-blocks)
+    (400, 512, 8, 4, 256, 128),    # ~200 rows per expert: tiles of 129..256 tokens
+    (1100, 256, 3, 2, 128, 0),     # ~730 rows per expert: several token chunks per expert
 ]
 
 
