@@ -65,9 +65,10 @@ typedef enum {
   MOE_ERR_BAD_INDEX = 7    /* device: an expert index was outside [0, E)                  */
 } moe_status;
 
-/* GEMM kernel variants.  AUTO: a DECODE context uses small-M; a PREFILL context chooses per step from the
- * step's rows per expert (T * top_k / n_experts <= 256: small-M, else large-M) -- a function of T alone, so a
- * step captured in a CUDA graph replays the kernel it was captured with. */
+/* GEMM kernel variants.  AUTO: a DECODE context uses small-M; a PREFILL context chooses per step and pass from
+ * the step's rows per expert R = T * top_k / n_experts (small-M up to R = 1024 for the gated pass, 384 for the
+ * down pass, 256 with FP8 weights; large-M above) -- a function of T alone, so a step captured in a CUDA graph
+ * replays the kernels it was captured with. */
 typedef enum {
   MOE_GEMM_AUTO = 0,
   MOE_GEMM_LARGE_M = 1,  /* tokens fill the 128-row MMA dimension; for experts of many hundreds of rows,

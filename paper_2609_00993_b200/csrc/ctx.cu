@@ -267,21 +267,26 @@ int gemm_ctas(const moe_ctx* ctx) {
   return (ctx->cfg.sm_budget > 0 && ctx->cfg.sm_budget < ctx->n_sms) ? ctx->cfg.sm_budget : ctx->n_sms;
 }
 
-// Experts of up to this many rows on average go to the small-M (weight-streaming) variant: below it a pass is
-// bound by the bytes of weights the SMs take in, and the small-M kernel takes in the fewest (one tile of up to
-// 256 tokens per expert and feature tile); above it the pass is bound by the tensor cores and the large-M kernel's
-// double-buffered accumulators and bulk-store epilogue win.
-constexpr int64_t kSmallMRowsPerExpert = 256;
+// Steps of up to this many rows per expert on average go to the small-M variant, per pass.  Measured on a B200
+// (DeepSeek-V3- and Qwen3-30B-shaped layers, uniform and Zipf routing): with tiles of up to 256 tokens the small-M
+// kernel moves fewer bytes through shared memory per flop than the large-M kernel (one CTA's MMA operands come
+// from shared memory, whose bandwidth is what both kernels end up waiting for).  The gated pass (long K on the
+// V3 shape, SwiGLU in the epilogue) is ahead with small-M by 5-13 % up to ~512 rows per expert and level with
+// large-M around 1024; the down pass (short K, so the exposed epilogue of its tiles of more than 128 tokens
+// weighs more) and the FP8 passes (half the operand bytes per flop, so the issue cost of two MMAs per 16
+// K-elements shows) change over near 256-384 rows per expert.
+constexpr int64_t kSmallMRowsGated = 1024, kSmallMRowsDown = 384, kSmallMRowsFp8 = 256;
 
-// AUTO: a DECODE context always streams; a PREFILL context chooses per step from the rows per expert of that
-// step's batch (T tokens): the choice is a function of T alone, so it is the same on every replay of a graph.
-int gemm_variant_of(const moe_ctx* ctx, int T) {
+// AUTO: a DECODE context always streams; a PREFILL context chooses per launch from the rows per expert of the
+// problem (T * top_k rows over n_experts; T rows over one group for the shared expert by itself): the choice is
+// a function of T alone, so it is the same on every replay of a graph.
+int gemm_variant_of(const moe_ctx* ctx, const moe::GemmProblem& p) {
   const int v = ctx->cfg.gemm_variant;
   if (v != MOE_GEMM_AUTO) return v;
   if (ctx->cfg.phase == MOE_PHASE_DECODE) return MOE_GEMM_SMALL_M;
   if (ctx->cfg.row_gather == 1) return MOE_GEMM_LARGE_M;  // only the large-M kernel gathers its rows itself
-  const int64_t rows = (int64_t)T * ctx->cfg.top_k;
-  return rows <= kSmallMRowsPerExpert * ctx->cfg.n_experts ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M;
+  const int64_t limit = p.fp8 ? kSmallMRowsFp8 : (p.gated ? kSmallMRowsGated : kSmallMRowsDown);
+  return p.rows_bound <= limit * p.E ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M;  // p.E = 1 for a dense problem
 }
 
 // GEMM1 gathers its rows itself only on the large-M tensor-core variant.
@@ -293,7 +298,7 @@ bool gathers_rows(const moe_ctx* ctx) {
 
 // `dense` (the shared expert's pass, or nullptr) rides in the same launch on the tensor-core path.
 cudaError_t run_gemm(moe_ctx* ctx, moe::GemmProblem p, const moe::GemmDenseGroup* dense, int T, int* n) {
-  const int variant = gemm_variant_of(ctx, T);
+  const int variant = gemm_variant_of(ctx, p);
   p.wait_limit_ns = ctx->wait_limit_ns;
   p.debug_stall = ctx->debug_stall;
   if (variant == MOE_GEMM_VALIDATION) {

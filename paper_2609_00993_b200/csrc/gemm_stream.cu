@@ -34,13 +34,22 @@ namespace {
 using namespace tc;
 
 #ifndef MOE_STREAM_ISSUERS
-#define MOE_STREAM_ISSUERS 2
+#define MOE_STREAM_ISSUERS 1
 #endif
-constexpr int kIssuers = MOE_STREAM_ISSUERS;  // MMA-issuing threads: one per weight box (2) or one for both (1)
-constexpr int kThreads = 192 + 32 * (kIssuers - 1);
-constexpr int kEpilogueWarps = 4;
-constexpr int kProducerWarp = 4;
-constexpr int kMmaWarp = 5;  // issuer of box 0 and TMEM owner; warp 6 issues box 1 when kIssuers == 2
+#ifndef MOE_STREAM_EPI_WARPS
+#define MOE_STREAM_EPI_WARPS 8
+#endif
+// MMA-issuing threads: one for both weight boxes (1) or one per box (2).  Two were measured and are no faster:
+// what the issuer waits for is the tensor pipe, which in turn waits for shared-memory bandwidth.
+constexpr int kIssuers = MOE_STREAM_ISSUERS;
+// Epilogue warps: 4 (each owns 32 TMEM lanes = 32 weight rows) or 8 (two warps per lane group, one taking the
+// even and one the odd 16-token chunks), which halves the time a tile of more than 128 tokens keeps the MMA
+// issuer waiting for its single accumulator.
+constexpr int kEpilogueWarps = MOE_STREAM_EPI_WARPS;
+constexpr int kProducerWarp = kEpilogueWarps;
+constexpr int kMmaWarp = kEpilogueWarps + 1;  // issuer of box 0 and TMEM owner; the next warp issues box 1 when kIssuers == 2
+constexpr int kThreads = 32 * (kEpilogueWarps + 1 + kIssuers);
+constexpr int kSortMaxExperts = 512;  // the tile list is ordered by expert size up to this many experts
 constexpr int kSlotBytes = 2048;                        // ring granularity: 16 token rows of one k-block
 constexpr int kWSlots = 2 * kWBoxBytes / kSlotBytes;    // 16 slots: the two weight boxes
 constexpr int kMaxTileRows = 256;                       // largest MMA N
@@ -97,10 +106,16 @@ __device__ __forceinline__ void chunking(int cnt, int& tiles, int& chunk) {
   chunk = tiles > 0 ? (((cnt + tiles - 1) / tiles) + 15) & ~15 : 0;
 }
 
+// Position of a CTA's w-th tile in the tile list: the list is dealt in waves of n_units tiles, alternately
+// forwards and backwards, so that with tiles ordered by cost no CTA always gets the costliest tile of a wave.
+__device__ __forceinline__ int snake_tile(int w, int unit, int n_units) {
+  return w * n_units + ((w & 1) ? n_units - 1 - unit : unit);
+}
+
 // tile -> (expert, first row, valid rows, feature tile).  The dense group's tiles come first (chunk major),
-// then the experts': prefix[e] = chunks of experts < e.
+// then the experts' in the order `order` (largest first): prefix[i] = chunks of the experts at positions < i.
 __device__ __forceinline__ STile decode_tile(int tile, int dense_tiles, int n_ft2, int rows2, int n_ft, int E,
-                                             const int* prefix, const int* seg) {
+                                             const int* prefix, const int* order, const int* beg, const int* cnts) {
   STile t;
   int tiles, chunk;
   if (tile < dense_tiles) {
@@ -115,17 +130,17 @@ __device__ __forceinline__ STile decode_tile(int tile, int dense_tiles, int n_ft
   }
   tile -= dense_tiles;
   const int rt = tile / n_ft;
-  int lo = 0, hi = E;  // largest e in [0,E) with prefix[e] <= rt
+  int lo = 0, hi = E;  // largest position in [0,E) with prefix[position] <= rt
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
     if (prefix[mid] <= rt) lo = mid; else hi = mid;
   }
-  const int cnt = seg[lo + 1] - seg[lo];
+  const int e = order[lo], cnt = cnts[e];
   chunking(cnt, tiles, chunk);
   const int mt = rt - prefix[lo];
-  t.e = lo;
+  t.e = e;
   t.ft = tile - rt * n_ft;
-  t.row0 = seg[lo] + mt * chunk;
+  t.row0 = beg[e] + mt * chunk;
   t.rows = min(chunk, cnt - mt * chunk);
   t.dense = false;
   return t;
@@ -138,7 +153,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   constexpr int kbk = FP8 ? 2 * kBlockK : kBlockK;  // K elements per k-block
   extern __shared__ uint8_t smem_raw[];
   // carve: ring (ring_slots x 2 KB) | full[kNB] empty[kNB] tfull[2] tempty[2] | tmem slot | abort | sizes[kNB]
-  //        | prefix[E+1] | seg[E+1]
+  //        | prefix[E+1] | order[E] | beg[E] | cnts[E]
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
   uint8_t* base = smem_raw + (base_addr - raw_addr);
@@ -151,7 +166,9 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* sizes = reinterpret_cast<int*>(tmem_slot + 2);  // slots held by the k-blocks in flight (producer only)
   int* prefix = sizes + kNB;
-  int* seg = prefix + (p.E + 1);
+  int* order = prefix + (p.E + 1);
+  int* beg = order + p.E;
+  int* cnts = beg + p.E;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int unit = (int)blockIdx.x, n_units = (int)gridDim.x;
@@ -162,19 +179,33 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   const int dense_tiles = p.rows2 > 0 ? ((p.rows2 + kMaxTileRows - 1) / kMaxTileRows) * n_ft2 : 0;
   const unsigned long long limit = p.wait_limit_ns;
 
-  // ---- set-up: tile list, barriers, TMEM
+  // ---- set-up: tile list (experts ordered by size, largest first), barriers, TMEM
+  for (int e = threadIdx.x; e < p.E; e += kThreads) {
+    const int b = p.offsets ? p.offsets[e] : 0;
+    int c = p.offsets ? p.offsets[e + 1] - b : p.fixed_rows;
+    if (c < 0) c = 0;
+    beg[e] = b;
+    cnts[e] = c;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < p.E; e += kThreads) {
+    int rank = e;  // more than kSortMaxExperts experts: the natural order
+    if (p.E <= kSortMaxExperts) {
+      const int c = cnts[e];
+      rank = 0;
+      for (int j = 0; j < p.E; ++j) {
+        const int cj = cnts[j];
+        rank += (cj > c || (cj == c && j < e)) ? 1 : 0;
+      }
+    }
+    order[rank] = e;
+  }
+  __syncthreads();
   if (warp == 0) {
     int carry = 0;
     for (int b = 0; b < p.E; b += 32) {
-      const int e = b + lane;
-      int beg = 0, cnt = 0;
-      if (e < p.E) {
-        beg = p.offsets ? p.offsets[e] : 0;
-        cnt = p.offsets ? p.offsets[e + 1] - beg : p.fixed_rows;
-        if (cnt < 0) cnt = 0;
-        seg[e] = beg;
-        if (e == p.E - 1) seg[p.E] = beg + cnt;
-      }
+      const int i = b + lane;
+      const int cnt = i < p.E ? cnts[order[i]] : 0;
       const int tiles = (cnt + kMaxTileRows - 1) / kMaxTileRows;
       int incl = tiles;
 #pragma unroll
@@ -182,12 +213,12 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
         const int n = __shfl_up_sync(0xffffffffu, incl, off);
         if (lane >= off) incl += n;
       }
-      if (e < p.E) prefix[e] = carry + incl - tiles;
+      if (i < p.E) prefix[i] = carry + incl - tiles;
       carry += __shfl_sync(0xffffffffu, incl, 31);
     }
     if (lane == 0) prefix[p.E] = carry;
   }
-  if (threadIdx.x == 32) {
+  if (threadIdx.x == 32 * kProducerWarp) {
     for (int s = 0; s < kNB; ++s) {
       mbar_init(bar_full + 8u * s, 1);
       mbar_init(bar_empty + 8u * s, kIssuers);
@@ -215,8 +246,10 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       bool ok = true;
       [[maybe_unused]] long long prof_wait_empty = 0, prof_tiles = 0;
       [[maybe_unused]] const long long prof_start = clock64();
-      for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
-        const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, seg);
+      for (int w = 0; w * n_units < total_tiles && ok; ++w) {
+        const int tile = snake_tile(w, unit, n_units);
+        if (tile >= total_tiles) break;
+        const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
         const uint32_t n = (uint32_t)((t.rows + 15) & ~15);
         const uint32_t s = (uint32_t)kWSlots + (n >> 4);
         const int w_row0 = t.ft * kFeatPerTile;
@@ -273,8 +306,10 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       const uint32_t desc_hi = (uint32_t)(umma_smem_desc(0) >> 32);
       const uint32_t lo_base = (uint32_t)umma_smem_desc(base_addr);  // slot 0
       constexpr uint32_t lo_slot = (uint32_t)kSlotBytes >> 4, lo_box = (uint32_t)kWBoxBytes >> 4;
-      for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
-        const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, seg);
+      for (int w = 0; w * n_units < total_tiles && ok; ++w) {
+        const int tile = snake_tile(w, unit, n_units);
+        if (tile >= total_tiles) break;
+        const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
         const uint32_t n = (uint32_t)((t.rows + 15) & ~15);
         const uint32_t s = (uint32_t)kWSlots + (n >> 4);
         const bool big = n > 128u;
@@ -357,11 +392,15 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
     // lane = weight row (output feature) of each box, TMEM column = token
     uint32_t use0 = 0, use1 = 0, next_half = 0;
     bool ok = true;
-    const uint32_t lane_base = ((uint32_t)(warp * 32)) << 16;
-    const int fl = warp * 32 + lane;
+    const int lg = warp & 3;                         // TMEM lane group of this warp: lanes 32 lg .. 32 lg + 31
+    const int c_first = kEpilogueWarps == 8 ? 16 * (warp >> 2) : 0, c_step = kEpilogueWarps == 8 ? 32 : 16;
+    const uint32_t lane_base = ((uint32_t)(lg * 32)) << 16;
+    const int fl = lg * 32 + lane;
     const bool even = (lane & 1) == 0;
-    for (int tile = unit; tile < total_tiles && ok; tile += n_units) {
-      const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, seg);
+    for (int w = 0; w * n_units < total_tiles && ok; ++w) {
+      const int tile = snake_tile(w, unit, n_units);
+      if (tile >= total_tiles) break;
+      const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
       const uint32_t n = (uint32_t)((t.rows + 15) & ~15);
       const bool big = n > 128u;
       uint32_t h = 0, d_a, d_b;
@@ -400,7 +439,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       // values for them (features f, f+1 of one token are one 4-byte store); the odd lane does the same for
       // the odd tokens.  n_feat is a multiple of 8, so a pair is inside the row or outside it as a whole.
       const int f_pair = (GATED ? f_a : 0) & ~1;
-      for (int c = 0; c < t.rows; c += 16) {
+      for (int c = c_first; c < t.rows; c += c_step) {
         uint32_t ra[16], rb[16];
         tmem_ld16(d_a + (uint32_t)c, ra);
         tmem_ld16(d_b + (uint32_t)c, rb);
@@ -560,7 +599,7 @@ cudaError_t launch_gemm_stream(const GemmProblem& p, const GemmDenseGroup* dense
   prm.w_scale2 = dense ? dense->w_scale : nullptr;
 
   const size_t tail = (2 * kNB + 4) * sizeof(uint64_t) + 2 * sizeof(uint32_t) + kNB * sizeof(int) +
-                      2 * (size_t)(prm.E + 1) * sizeof(int);
+                      4 * (size_t)(prm.E + 1) * sizeof(int);
   const int slots = (int)((kSmemBudget - 1024 - (int)tail) / kSlotBytes);
   if (slots < 2 * (kWSlots + kMaxTileRows / 16)) return cudaErrorNotSupported;
   prm.ring_slots = slots;
