@@ -28,8 +28,8 @@
  *     context's device status word; nothing traps.  `moe_ctx_status` reads it.
  *   - bf16 tensors are passed as `const void*` / `void*`.
  *
- * Per step, in order:  moe_route (optional) -> moe_dispatch_layout -> moe_grouped_ffn
- * -> moe_combine.  Any other order returns MOE_ERR_STATE.
+ * Per step, in order:  moe_route (optional) -> moe_dispatch_layout (or its two halves moe_dispatch_notify ->
+ * moe_dispatch_move) -> moe_grouped_ffn -> moe_combine.  Any other order returns MOE_ERR_STATE.
  *
  * CUDA graphs.  The four step calls only enqueue kernels, so a step may be recorded while the
  * context's stream is being captured and replayed later (D keeps stable graph addresses: the
@@ -188,6 +188,33 @@ moe_status moe_route(moe_ctx* ctx, const float* logits, const float* select_bias
 moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T, const void* x, int32_t* counts,
                                int32_t* offsets, int32_t* perm, int32_t* inv_perm);
 
+/* Split-phase dispatch.  The paper splits a normal (prefill) dispatch AFTER notification: expert notification and
+ * the receive counts come first; the routed data movement happens only after the counts are there AND the
+ * boundary controller has given its permit, so that a ready decode iteration can be ordered in between; the backend
+ * keeps a pending-dispatch record (the tensors and the stream state the second half needs), allows at most one
+ * pending dispatch per prefill buffer and makes every transition explicit (Section "Exposing a Safe Prefill
+ * Boundary").  On one GPU the two halves of moe_dispatch_layout are:
+ *   moe_dispatch_notify   stages a2-a4 only (counts, exclusive scan, stable permutation; arguments as for
+ *                         moe_dispatch_layout without x).  The context then holds a pending dispatch: the arrays, T
+ *                         and the stream position of this half.  With prefill segmentation on, the boundary hook is
+ *                         called here as boundary 0 of 1 + (the boundaries of moe_grouped_ffn), which then
+ *                         reports its own as 1, 2, ...: the first safe point of a prefill step lies before any
+ *                         row has moved.
+ *   moe_dispatch_move     stage a5, the routed data movement of the pending dispatch (x [T,H] bf16; an FP8 context
+ *                         quantises and moves codes, a row_gather context moves nothing).  The counts need no
+ *                         host round trip here -- they stay on the device and the stream orders the two halves --
+ *                         so calling this function IS the permit.  Afterwards the step continues with
+ *                         moe_grouped_ffn as after moe_dispatch_layout.
+ * Transitions: idle/routed --notify--> pending --move--> laid out.  A second moe_dispatch_notify or a
+ * moe_dispatch_layout while a dispatch is pending returns MOE_ERR_STATE, as does moe_dispatch_move without one;
+ * moe_ctx_abandon_step retires a pending dispatch together with the step (kernels already enqueued still run).
+ * If moe_dispatch_move fails the dispatch stays pending.  moe_ctx_pending_dispatch reports whether a dispatch is
+ * pending, its T, and whether the first half has already finished on the device (an event query; no wait). */
+moe_status moe_dispatch_notify(moe_ctx* ctx, const int32_t* topk_idx, int32_t T, int32_t* counts, int32_t* offsets,
+                               int32_t* perm, int32_t* inv_perm);
+moe_status moe_dispatch_move(moe_ctx* ctx, const void* x);
+moe_status moe_ctx_pending_dispatch(moe_ctx* ctx, int32_t* pending, int32_t* tokens, int32_t* notified_done);
+
 /* Stages a6-a8 -- grouped SwiGLU expert FFN over the permuted rows, plus the shared expert:
  *   act[p,i]    = silu(x_perm[p,:] . W_gate_up[e,i,:]) * (x_perm[p,:] . W_gate_up[e,I+i,:])
  *   y_perm[p,c] = act[p,:] . W_down[e,c,:]          for p in expert e's segment
@@ -284,6 +311,8 @@ moe_status moe_combine(moe_ctx* ctx, const float* topk_w, const int32_t* inv_per
  * The call allocates nothing and frees nothing.  It works on the device that is current when it is called:
  * the pointers and the stream must belong to that device.  The first call on each device looks up the
  * array's device address (a host-side set-up step); make that first call before any stream capture begins.
+ * A call with more experts than any earlier call on that device (single-launch path, T*top_k <= 16384) also
+ * raises a kernel's shared-memory limit on the host, so it too should come before capture.
  * All calls on one device share the array: two calls whose kernels can overlap on the GPU (different
  * streams without an ordering between them) race on it -- order them.  Nothing in the array needs clearing
  * between calls: every cell is written before it is read within a call.

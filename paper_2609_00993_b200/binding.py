@@ -33,7 +33,7 @@ EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_
            "moe_dispatch_layout_static", "moe_ctx_set_segments", "moe_ctx_abandon_step", "moe_turnstile_create", "moe_turnstile_destroy",
            "moe_turnstile_set_span", "moe_turnstile_begin_epoch", "moe_turnstile_publish", "moe_turnstile_task_done",
            "moe_turnstile_d_enter", "moe_turnstile_d_release", "moe_turnstile_state", "moe_ctx_set_wait_limit",
-           "moe_ctx_debug_inject_stall")
+           "moe_ctx_debug_inject_stall", "moe_dispatch_notify", "moe_dispatch_move", "moe_ctx_pending_dispatch")
 
 BOUNDARY_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32)
 
@@ -120,6 +120,12 @@ def load_library() -> ctypes.CDLL:
                        ("moe_turnstile_state", [vp, ctypes.POINTER(i64)] + [ctypes.POINTER(i32)] * 4)):
         getattr(lib, name).restype = i32
         getattr(lib, name).argtypes = args
+    lib.moe_dispatch_notify.restype = i32
+    lib.moe_dispatch_notify.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    lib.moe_dispatch_move.restype = i32
+    lib.moe_dispatch_move.argtypes = [vp, vp]
+    lib.moe_ctx_pending_dispatch.restype = i32
+    lib.moe_ctx_pending_dispatch.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.moe_ctx_set_wait_limit.restype = i32
     lib.moe_ctx_set_wait_limit.argtypes = [vp, i64]
     lib.moe_ctx_debug_inject_stall.restype = i32
@@ -276,6 +282,25 @@ class MoeContext:
         T = topk_idx.shape[0] if T is None else T
         self._check(self.lib.moe_dispatch_layout(self.handle, _ptr(topk_idx), T, _ptr(x), _ptr(counts), _ptr(offsets),
                                                  _ptr(perm), _ptr(inv_perm)))
+
+    def moe_dispatch_notify(self, topk_idx, counts=None, offsets=None, perm=None, inv_perm=None, T=None):
+        """First half of a split dispatch (counts, scan, permutation); the context then holds a pending dispatch."""
+        _dev(topk_idx, torch.int32, "topk_idx")
+        for n, t in (("counts", counts), ("offsets", offsets), ("perm", perm), ("inv_perm", inv_perm)):
+            _dev(t, torch.int32, n)
+        T = topk_idx.shape[0] if T is None else T
+        self._check(self.lib.moe_dispatch_notify(self.handle, _ptr(topk_idx), T, _ptr(counts), _ptr(offsets),
+                                                 _ptr(perm), _ptr(inv_perm)))
+
+    def moe_dispatch_move(self, x):
+        """Second half: the routed data movement of the pending dispatch."""
+        _dev(x, torch.bfloat16, "x")
+        self._check(self.lib.moe_dispatch_move(self.handle, _ptr(x)))
+
+    def moe_ctx_pending_dispatch(self) -> dict:
+        p, t, d = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+        self._check(self.lib.moe_ctx_pending_dispatch(self.handle, ctypes.byref(p), ctypes.byref(t), ctypes.byref(d)))
+        return {"pending": bool(p.value), "tokens": int(t.value), "notified_done": bool(d.value)}
 
     def moe_grouped_ffn(self, w_gate_up, w_down, x, ws_gate_up=None, ws_down=None, T=None):
         for n, t in (("w_gate_up", w_gate_up), ("w_down", w_down), ("x", x), ("ws_gate_up", ws_gate_up),

@@ -16,7 +16,9 @@
 
 namespace {
 
-enum StepState { ST_IDLE = 0, ST_ROUTED = 1, ST_LAID_OUT = 2, ST_LAYOUT_ONLY = 3, ST_FFN_DONE = 4 };
+// ST_NOTIFIED: the first half of a split dispatch has been enqueued (counts, scan, permutation) and the routed
+// data movement is pending; ST_LAYOUT_ONLY: a layout without rows (moe_dispatch_layout with x == NULL).
+enum StepState { ST_IDLE = 0, ST_ROUTED = 1, ST_LAID_OUT = 2, ST_LAYOUT_ONLY = 3, ST_FFN_DONE = 4, ST_NOTIFIED = 5 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -166,6 +168,11 @@ struct moe_ctx {
   int32_t* inv_perm;
   cudaEvent_t done;  // recorded after the last enqueue of every call
   int64_t launches;
+  // pending-dispatch record of a split dispatch: what the second half needs (the arrays above, T) and the
+  // stream position of the first half; at most one per context
+  bool pending_dispatch;
+  cudaEvent_t notified;
+  bool split_step;   // the step in progress went through the split entry points (boundary numbering)
   // prefill segmentation (off by default)
   int seg_experts;
   moe_boundary_fn boundary_fn;
@@ -379,6 +386,8 @@ moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspa
   ctx->state = ST_IDLE;
   ctx->T = 0;
   ctx->launches = 0;
+  ctx->pending_dispatch = false;
+  ctx->split_step = false;
   ctx->profiling = false;
   ctx->spans_used = 0;
   ctx->seg_experts = 0;
@@ -423,6 +432,10 @@ moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspa
   int sms = 0;
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->done, cudaEventDisableTiming);
+  if (e == cudaSuccess) {
+    e = cudaEventCreateWithFlags(&ctx->notified, cudaEventDisableTiming);
+    if (e != cudaSuccess) cudaEventDestroy(ctx->done);
+  }
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ws, 0, kStatusBlock, ctx->stream);
   if (e == cudaSuccess) e = cudaEventRecord(ctx->done, ctx->stream);
   if (e != cudaSuccess) {
@@ -469,6 +482,7 @@ moe_status moe_ctx_destroy(moe_ctx* ctx) {
       }
   }
   cudaEventDestroy(ctx->done);
+  cudaEventDestroy(ctx->notified);
   for (auto& sp : ctx->spans) {
     cudaEventDestroy(sp.beg);
     cudaEventDestroy(sp.end);
@@ -482,6 +496,8 @@ moe_status moe_ctx_abandon_step(moe_ctx* ctx) {
   if (ctx->state == ST_IDLE) return MOE_OK;
   ctx->state = ST_IDLE;
   ctx->T = 0;
+  ctx->pending_dispatch = false;  // a pending dispatch is retired with the step
+  ctx->split_step = false;
   if (ctx->n_sets == 2) ctx->cur ^= 1;  // D: the abandoned step's buffer set rests for one whole step
   return MOE_OK;
 }
@@ -526,18 +542,18 @@ moe_status moe_route(moe_ctx* ctx, const float* logits, const float* select_bias
   return MOE_OK;
 }
 
-moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T, const void* x, int32_t* counts,
-                               int32_t* offsets, int32_t* perm, int32_t* inv_perm) {
-  if (!ctx) return MOE_ERR_INVALID_ARG;
-  if (ctx->state != ST_IDLE && ctx->state != ST_ROUTED && ctx->state != ST_LAYOUT_ONLY)
-    return fail(ctx, MOE_ERR_STATE, "moe_dispatch_layout called in the middle of a step");
+}  // extern "C"
+
+namespace {
+
+// First half of a dispatch: counts, exclusive scan, stable permutation (no rows move).
+moe_status enqueue_layout(moe_ctx* ctx, const char* who, const int32_t* topk_idx, int32_t T, int32_t* counts,
+                          int32_t* offsets, int32_t* perm, int32_t* inv_perm) {
   if (T < 0) return fail(ctx, MOE_ERR_INVALID_ARG, "T < 0");
   if (T > ctx->cfg.max_tokens) return fail(ctx, MOE_ERR_CAPACITY, "T = %d exceeds max_tokens = %d", T, ctx->cfg.max_tokens);
   if (T > 0 && !topk_idx) return fail(ctx, MOE_ERR_INVALID_ARG, "topk_idx is NULL");
-  if (misaligned(topk_idx) || misaligned(x) || misaligned(counts) || misaligned(offsets) || misaligned(perm) ||
-      misaligned(inv_perm))
+  if (misaligned(topk_idx) || misaligned(counts) || misaligned(offsets) || misaligned(perm) || misaligned(inv_perm))
     return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
-  DeviceGuard guard(ctx->device);
   BufferSet& b = ctx->sets[ctx->cur];
   ctx->counts = counts ? counts : b.counts;
   ctx->offsets = offsets ? offsets : b.offsets;
@@ -550,25 +566,120 @@ moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T,
     e = moe::launch_layout(topk_idx, (int64_t)T * ctx->cfg.top_k, ctx->cfg.n_experts, ctx->counts, ctx->offsets,
                            ctx->perm, ctx->inv_perm, b.scan, ctx->status, ctx->stream, &n);
   }
+  if (e != cudaSuccess) return cuda_fail(ctx, e, who);
+  ctx->T = T;
+  ctx->launches += n;
+  return MOE_OK;
+}
+
+// Second half: the routed data movement (an FP8 context quantises each token row once and moves the codes).
+moe_status enqueue_row_movement(moe_ctx* ctx, const char* who, const void* x) {
+  BufferSet& b = ctx->sets[ctx->cur];
+  const int32_t T = ctx->T;
   const bool fp8 = ctx->cfg.weight_format == MOE_WEIGHTS_FP8_E4M3;
-  if (e == cudaSuccess && x != nullptr && fp8) {
-    // FP8 variant: quantise each token row once, then move the codes (half the bytes) and the row scales
-    StageTimer tm(ctx, 8);
-    e = moe::launch_quantize_rows(x, T, ctx->cfg.hidden, b.xq_tok, b.sx_tok, ctx->stream, &n);
-  }
-  if (e == cudaSuccess && x != nullptr && fp8) {
-    StageTimer tm(ctx, 2);
-    e = moe::launch_permute(b.xq_tok, ctx->inv_perm, b.xq, T, ctx->cfg.top_k, ctx->cfg.hidden / 2, ctx->status,
-                            ctx->stream, &n, b.sx_tok, b.sx, ctx->wait_limit_ns);
-  } else if (e == cudaSuccess && x != nullptr && !gathers_rows(ctx)) {
+  int n = 0;
+  cudaError_t e = cudaSuccess;
+  if (T > 0 && fp8) {
+    {
+      StageTimer tm(ctx, 8);
+      e = moe::launch_quantize_rows(x, T, ctx->cfg.hidden, b.xq_tok, b.sx_tok, ctx->stream, &n);
+    }
+    if (e == cudaSuccess) {
+      StageTimer tm(ctx, 2);
+      e = moe::launch_permute(b.xq_tok, ctx->inv_perm, b.xq, T, ctx->cfg.top_k, ctx->cfg.hidden / 2, ctx->status,
+                              ctx->stream, &n, b.sx_tok, b.sx, ctx->wait_limit_ns);
+    }
+  } else if (T > 0 && !gathers_rows(ctx)) {
     StageTimer tm(ctx, 2);
     e = moe::launch_permute(x, ctx->inv_perm, b.x_perm, T, ctx->cfg.top_k, ctx->cfg.hidden, ctx->status, ctx->stream,
                             &n, nullptr, nullptr, ctx->wait_limit_ns);
   }
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_dispatch_layout");
-  ctx->T = T;
+  if (e != cudaSuccess) return cuda_fail(ctx, e, who);
+  ctx->launches += n;
+  return MOE_OK;
+}
+
+// Boundaries moe_grouped_ffn / moe_grouped_ffn_fp8 report with the current segmentation.
+int ffn_boundaries(const moe_ctx* ctx) {
+  const moe_config& c = ctx->cfg;
+  const bool shared = c.n_shared != 0;
+  const int span = (ctx->seg_experts > 0 && ctx->seg_experts < c.n_experts) ? ctx->seg_experts : c.n_experts;
+  const int routed_segs = (c.n_experts + span - 1) / span;
+  const bool fuse_shared = shared && ctx->seg_experts == 0;
+  if (c.weight_format == MOE_WEIGHTS_FP8_E4M3) return 2 * routed_segs + 1 + ((shared && !fuse_shared) ? 2 : 0);
+  return 2 * routed_segs + (shared ? 2 : 0);
+}
+
+}  // namespace
+
+extern "C" {
+
+moe_status moe_dispatch_layout(moe_ctx* ctx, const int32_t* topk_idx, int32_t T, const void* x, int32_t* counts,
+                               int32_t* offsets, int32_t* perm, int32_t* inv_perm) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->state == ST_NOTIFIED)
+    return fail(ctx, MOE_ERR_STATE, "a dispatch is pending on this context: move its rows or abandon the step");
+  if (ctx->state != ST_IDLE && ctx->state != ST_ROUTED && ctx->state != ST_LAYOUT_ONLY)
+    return fail(ctx, MOE_ERR_STATE, "moe_dispatch_layout called in the middle of a step");
+  if (misaligned(x)) return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+  DeviceGuard guard(ctx->device);
+  moe_status st = enqueue_layout(ctx, "moe_dispatch_layout", topk_idx, T, counts, offsets, perm, inv_perm);
+  if (st == MOE_OK && x != nullptr) st = enqueue_row_movement(ctx, "moe_dispatch_layout", x);
+  if (st != MOE_OK) return st;
   ctx->state = (x != nullptr || T == 0) ? ST_LAID_OUT : ST_LAYOUT_ONLY;  // an empty batch has no rows to move
-  mark(ctx, n);
+  ctx->split_step = false;
+  mark(ctx, 0);
+  return MOE_OK;
+}
+
+moe_status moe_dispatch_notify(moe_ctx* ctx, const int32_t* topk_idx, int32_t T, int32_t* counts, int32_t* offsets,
+                               int32_t* perm, int32_t* inv_perm) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->pending_dispatch || ctx->state == ST_NOTIFIED)
+    return fail(ctx, MOE_ERR_STATE, "a dispatch is already pending on this context (at most one per context)");
+  if (ctx->state != ST_IDLE && ctx->state != ST_ROUTED)
+    return fail(ctx, MOE_ERR_STATE, "moe_dispatch_notify called in the middle of a step");
+  DeviceGuard guard(ctx->device);
+  moe_status st = enqueue_layout(ctx, "moe_dispatch_notify", topk_idx, T, counts, offsets, perm, inv_perm);
+  if (st != MOE_OK) return st;
+  ctx->state = ST_NOTIFIED;
+  ctx->pending_dispatch = true;
+  ctx->split_step = true;
+  mark(ctx, 0);
+  if (!capturing(ctx)) cudaEventRecord(ctx->notified, ctx->stream);  // the record's stream position
+  // boundary 0 of a segmented step: after notification, before any row moves
+  if (ctx->seg_experts > 0 && ctx->boundary_fn) ctx->boundary_fn(ctx->boundary_user, 0, 1 + ffn_boundaries(ctx));
+  return MOE_OK;
+}
+
+moe_status moe_dispatch_move(moe_ctx* ctx, const void* x) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->state != ST_NOTIFIED || !ctx->pending_dispatch)
+    return fail(ctx, MOE_ERR_STATE, "moe_dispatch_move needs a pending dispatch (moe_dispatch_notify) on this context");
+  if (ctx->T > 0 && !x) return fail(ctx, MOE_ERR_INVALID_ARG, "x is NULL");
+  if (misaligned(x)) return fail(ctx, MOE_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+  DeviceGuard guard(ctx->device);
+  moe_status st = enqueue_row_movement(ctx, "moe_dispatch_move", x);
+  if (st != MOE_OK) return st;  // the dispatch stays pending: retry, or abandon the step
+  ctx->state = ST_LAID_OUT;
+  ctx->pending_dispatch = false;
+  mark(ctx, 0);
+  return MOE_OK;
+}
+
+moe_status moe_ctx_pending_dispatch(moe_ctx* ctx, int32_t* pending, int32_t* tokens, int32_t* notified_done) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (pending) *pending = ctx->pending_dispatch ? 1 : 0;
+  if (tokens) *tokens = ctx->pending_dispatch ? ctx->T : 0;
+  if (notified_done) {
+    *notified_done = 0;
+    if (ctx->pending_dispatch) {
+      DeviceGuard guard(ctx->device);
+      const cudaError_t q = cudaEventQuery(ctx->notified);
+      if (q == cudaSuccess) *notified_done = 1;
+      else (void)cudaGetLastError();
+    }
+  }
   return MOE_OK;
 }
 
@@ -597,8 +708,9 @@ moe_status moe_grouped_ffn(moe_ctx* ctx, const void* w_gate_up, const void* w_do
     // One launch per pass, or one per group of seg_experts experts with a boundary call after each.
     const int span = (ctx->seg_experts > 0 && ctx->seg_experts < c.n_experts) ? ctx->seg_experts : c.n_experts;
     const int routed_segs = (c.n_experts + span - 1) / span;
-    const int n_bound = 2 * routed_segs + (shared ? 2 : 0);
-    int bound = 0;
+    const int first = ctx->split_step ? 1 : 0;  // a split dispatch reported boundary 0 after its notification
+    const int n_bound = first + 2 * routed_segs + (shared ? 2 : 0);
+    int bound = first;
     auto boundary = [&]() {
       if (ctx->seg_experts > 0 && ctx->boundary_fn) {
         if (!capturing(ctx)) cudaEventRecord(ctx->done, ctx->stream);
@@ -684,8 +796,9 @@ moe_status moe_grouped_ffn_fp8(moe_ctx* ctx, const void* wq_gate_up, const float
     const int span = (ctx->seg_experts > 0 && ctx->seg_experts < c.n_experts) ? ctx->seg_experts : c.n_experts;
     const int routed_segs = (c.n_experts + span - 1) / span;
     const bool fuse_shared = shared && ctx->seg_experts == 0;
-    const int n_bound = 2 * routed_segs + 1 + ((shared && !fuse_shared) ? 2 : 0);
-    int bound = 0;
+    const int first = ctx->split_step ? 1 : 0;
+    const int n_bound = first + 2 * routed_segs + 1 + ((shared && !fuse_shared) ? 2 : 0);
+    int bound = first;
     auto boundary = [&]() {
       if (ctx->seg_experts > 0 && ctx->boundary_fn) {
         if (!capturing(ctx)) cudaEventRecord(ctx->done, ctx->stream);
@@ -773,6 +886,7 @@ moe_status moe_combine(moe_ctx* ctx, const float* topk_w, const int32_t* inv_per
   }
   if (e != cudaSuccess) return cuda_fail(ctx, e, "moe_combine");
   ctx->state = ST_IDLE;
+  ctx->split_step = false;
   if (ctx->n_sets == 2) ctx->cur ^= 1;  // D: the next step works in the other buffer set
   mark(ctx, n);
   return MOE_OK;

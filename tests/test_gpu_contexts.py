@@ -2,11 +2,12 @@
 import ctypes
 import os
 
+import numpy as np
 import pytest
 import torch
 
 import oracle
-from helpers import check_layer, np_f32
+from helpers import check_layer, layer_errors, np_f32, np_i32
 from paper_2609_00993_b200 import binding as B
 from paper_2609_00993_b200 import workloads as wl
 
@@ -273,6 +274,130 @@ def test_decode_step_admitted_at_a_prefill_boundary():
     assert torch.equal(p_out, p_alone) and torch.equal(d_out, d_alone)
     assert p.moe_ctx_status() == B.MOE_OK and d.moe_ctx_status() == B.MOE_OK
     p.moe_ctx_set_segments(0)
+    p.close(); d.close()
+
+
+def test_split_dispatch_state_transitions():
+    """Notification and row movement as two calls: at most one pending dispatch per context, explicit transitions,
+    an abandoned step retires the pending dispatch, and the one-call and two-call forms give the same bits."""
+    shape = wl.LayerShape("t", T=300, H=256, E=8, k=2, I=128, shared_I=64)
+    w, a = wl.make_weights(shape, 1, DEV), wl.make_activations(shape, 2, DEV)
+    ctx = B.MoeContext(B.make_config(256, 8, 2, 128, 64, 300, B.MOE_PHASE_PREFILL))
+    wargs = (w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+    torch.cuda.synchronize()
+    whole, wb = ctx.layer(a["x"], a["logits"], None, *wargs)
+    torch.cuda.synchronize()
+    bufs = B.alloc_step_buffers(300, 2, 8, DEV)
+    out = torch.empty_like(whole)
+    assert ctx.moe_ctx_pending_dispatch() == {"pending": False, "tokens": 0, "notified_done": False}
+    with pytest.raises(B.MoeError) as ei:      # no pending dispatch to move
+        ctx.moe_dispatch_move(a["x"])
+    assert ei.value.status == B.MOE_ERR_STATE
+    ctx.moe_route(a["logits"], None, bufs["topk_idx"], bufs["topk_w"])
+    ctx.moe_dispatch_notify(bufs["topk_idx"], bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"])
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_pending_dispatch() == {"pending": True, "tokens": 300, "notified_done": True}
+    # the integer results are complete after the first half
+    ref = oracle.layout(np_i32(bufs["topk_idx"]).reshape(-1), 8)
+    for name, want in zip(("counts", "offsets", "perm", "inv_perm"), ref):
+        assert np.array_equal(np_i32(bufs[name]), want), name
+    for call in (lambda: ctx.moe_dispatch_notify(bufs["topk_idx"]),                 # a second notification
+                 lambda: ctx.moe_dispatch_layout(bufs["topk_idx"], a["x"]),         # the one-call form
+                 lambda: ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"], w["ws_gate_up"], w["ws_down"]),
+                 lambda: ctx.moe_route(a["logits"], None, bufs["topk_idx"], bufs["topk_w"])):
+        with pytest.raises(B.MoeError) as ei:
+            call()
+        assert ei.value.status == B.MOE_ERR_STATE
+    assert ctx.moe_ctx_pending_dispatch()["pending"]
+    ctx.moe_dispatch_move(a["x"])
+    assert not ctx.moe_ctx_pending_dispatch()["pending"]
+    ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"], w["ws_gate_up"], w["ws_down"])
+    ctx.moe_combine(bufs["topk_w"], bufs["inv_perm"], out)
+    torch.cuda.synchronize()
+    assert torch.equal(out, whole) and torch.equal(bufs["perm"], wb["perm"])
+    # abandoning a step retires its pending dispatch; the context then takes a new notification
+    ctx.moe_dispatch_notify(bufs["topk_idx"])
+    ctx.moe_ctx_abandon_step()
+    assert not ctx.moe_ctx_pending_dispatch()["pending"]
+    ctx.moe_dispatch_notify(bufs["topk_idx"], bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"])
+    ctx.moe_dispatch_move(a["x"])
+    ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"], w["ws_gate_up"], w["ws_down"])
+    ctx.moe_combine(bufs["topk_w"], bufs["inv_perm"], out)
+    torch.cuda.synchronize()
+    assert torch.equal(out, whole) and ctx.moe_ctx_status() == B.MOE_OK
+    # with segmentation on, the notification is boundary 0 and the FFN's boundaries follow it
+    seen = []
+    ctx.moe_ctx_set_segments(4, lambda i, n: seen.append((i, n)))
+    ctx.moe_dispatch_notify(bufs["topk_idx"], bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"])
+    assert seen == [(0, 7)]                       # 1 + 2 * 2 routed segments + 2 shared-expert passes
+    ctx.moe_dispatch_move(a["x"])
+    ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"], w["ws_gate_up"], w["ws_down"])
+    ctx.moe_combine(bufs["topk_w"], bufs["inv_perm"], out)
+    torch.cuda.synchronize()
+    assert seen == [(i, 7) for i in range(7)] and torch.equal(out, whole)
+    ctx.moe_ctx_set_segments(0)
+    ctx.close()
+
+
+@pytest.mark.parametrize("fmt", [B.MOE_WEIGHTS_BF16, B.MOE_WEIGHTS_FP8_E4M3])
+def test_decode_step_admitted_between_notification_and_row_movement(fmt):
+    """The first safe point of a prefill step: P has enqueued its layout (notification, counts, permutation) and
+    holds a pending dispatch; the controller admits a whole D step there and gives P's row movement its permit
+    only afterwards.  Both phases give the bits they give alone, and those match the oracle."""
+    shape = wl.LayerShape("t", T=40, H=512, E=16, k=4, I=256, shared_I=128, select_bias=True)
+    pshape = shape.with_tokens(1500)
+    fp8 = fmt == B.MOE_WEIGHTS_FP8_E4M3
+    w = wl.make_weights_fp8(shape, 1, DEV) if fp8 else wl.make_weights(shape, 1, DEV)
+    ad, ap = wl.make_activations(shape, 2, DEV), wl.make_activations(pshape, 3, DEV)
+    sp, sd = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    d = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 40, B.MOE_PHASE_DECODE, weight_format=fmt), stream=sd)
+    p = B.MoeContext(B.make_config(512, 16, 4, 256, 128, 1500, B.MOE_PHASE_PREFILL, weight_format=fmt), stream=sp)
+
+    def ffn(ctx, a, T):
+        if fp8:
+            ctx.moe_grouped_ffn_fp8(w["wq_gate_up"], w["sw_gate_up"], w["wq_down"], w["sw_down"], w["wsq_gate_up"],
+                                    w["sws_gate_up"], w["wsq_down"], w["sws_down"], T=T)
+        else:
+            ctx.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"], w["ws_gate_up"], w["ws_down"])
+
+    def whole_step(ctx, a, out, bufs):
+        T = a["x"].shape[0]
+        ctx.moe_route(a["logits"], a["bias"], bufs["topk_idx"], bufs["topk_w"])
+        ctx.moe_dispatch_layout(bufs["topk_idx"], a["x"], bufs["counts"], bufs["offsets"], bufs["perm"], bufs["inv_perm"])
+        ffn(ctx, a, T)
+        ctx.moe_combine(bufs["topk_w"], bufs["inv_perm"], out)
+
+    bd, bp = B.alloc_step_buffers(40, 4, 16, DEV), B.alloc_step_buffers(1500, 4, 16, DEV)
+    d_alone, p_alone = torch.empty(40, 512, dtype=torch.bfloat16, device=DEV), torch.empty(1500, 512, dtype=torch.bfloat16, device=DEV)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(sd):
+        whole_step(d, ad, d_alone, bd)
+    with torch.cuda.stream(sp):
+        whole_step(p, ap, p_alone, bp)
+    torch.cuda.synchronize()
+    d_out, p_out = torch.zeros_like(d_alone), torch.zeros_like(p_alone)
+    torch.cuda.synchronize()
+    # P: route + notification; then the D step is admitted; then P's rows move behind it
+    p.moe_route(ap["logits"], ap["bias"], bp["topk_idx"], bp["topk_w"])
+    p.moe_dispatch_notify(bp["topk_idx"], bp["counts"], bp["offsets"], bp["perm"], bp["inv_perm"])
+    assert p.moe_ctx_pending_dispatch()["pending"]
+    with torch.cuda.stream(sd):
+        whole_step(d, ad, d_out, bd)
+        ev = torch.cuda.Event()
+        ev.record(sd)
+    sp.wait_event(ev)                 # the permit: P's data movement is ordered after the D step
+    p.moe_dispatch_move(ap["x"])
+    ffn(p, ap, 1500)
+    p.moe_combine(bp["topk_w"], bp["inv_perm"], p_out)
+    torch.cuda.synchronize()
+    assert p.moe_ctx_status() == B.MOE_OK and d.moe_ctx_status() == B.MOE_OK
+    assert torch.equal(p_out, p_alone) and torch.equal(d_out, d_alone)
+    if not fp8:
+        for a, out, shp in ((ap, p_out, pshape), (ad, d_out, shape)):
+            ref = oracle.layer(wl.bits(a["x"]), np_f32(a["logits"]), np_f32(a["bias"]), 4, wl.bits(w["w_gate_up"]),
+                               wl.bits(w["w_down"]), wl.bits(w["ws_gate_up"]), wl.bits(w["ws_down"]))
+            e = layer_errors(out, ref["out"])
+            assert e["rel_l2"] <= 5e-3 and e["max_abs"] <= 2e-2, e
     p.close(); d.close()
 
 
