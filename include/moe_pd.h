@@ -264,6 +264,27 @@ moe_status moe_grouped_ffn_fp8(moe_ctx* ctx, const void* wq_gate_up, const float
 typedef void (*moe_boundary_fn)(void* user, int32_t boundary, int32_t n_boundaries);
 moe_status moe_ctx_set_segments(moe_ctx* ctx, int32_t experts_per_segment, moe_boundary_fn fn, void* user);
 
+/* Preemption of a prefill step at tile granularity -- boundaries without cutting P into many launches.
+ * The paper lets successive D iterations advance through one long P execution at backend-provided boundaries
+ * (Section "In-Place P/D Execution"); on one GPU, where P and D compete for the same SMs and the same HBM, the
+ * finest boundary that costs nothing while no D is waiting is the end of a GEMM tile.  With preemption on (PREFILL
+ * contexts only), every GEMM pass of moe_grouped_ffn uses the small-M kernel, whose CTAs look at a yield request
+ * before each tile (tens of microseconds apart).  moe_ctx_request_yield(ctx, 1) -- callable from any host thread,
+ * typically the one about to enqueue a D step -- raises the request: every CTA finishes the tile it is in, saves
+ * its position and exits, so the SMs are free within one tile's time.  moe_grouped_ffn, which in this mode WAITS
+ * ON THE HOST for each of its launches (eager variable-length P; it cannot be captured in a graph and costs a
+ * host round trip of ~10 us per launch), then calls the boundary hook as fn(user, MOE_BOUNDARY_YIELD, 0) and,
+ * when the hook returns, launches the pass again: every CTA resumes where it stopped.  The hook is the permit
+ * wait: it should return once the D step has finished on the device and the request has been lowered
+ * (moe_ctx_request_yield(ctx, 0)); a request still up is honoured again (up to 64 launches per pass, after which
+ * the pass runs to its end regardless).  Results are bit-identical to the unpreempted pass.  The first
+ * moe_ctx_set_preemption(ctx, 1) allocates two small pinned host words (host memory, freed by moe_ctx_destroy).
+ * moe_ctx_yield_count: launches that ended on a request since the context was created. */
+#define MOE_BOUNDARY_YIELD (-1)
+moe_status moe_ctx_set_preemption(moe_ctx* ctx, int32_t enabled);
+moe_status moe_ctx_request_yield(moe_ctx* ctx, int32_t on);
+int64_t moe_ctx_yield_count(const moe_ctx* ctx);
+
 /* Segment turnstile -- the host-side boundary controller (Sections "Rank-Aligned Segment Boundaries" and
  * "Distributed Segment Turnstile").  Host-only: it orders host enqueue, never waits for GPU work and launches
  * nothing.  One controller per rank keeps the current P epoch e, the largest reached boundary r (-1 at the start

@@ -21,6 +21,7 @@ MOE_ERR_INVALID_ARG, MOE_ERR_CAPACITY, MOE_ERR_STATE, MOE_ERR_UNSUPPORTED = 1, 2
 MOE_ERR_CUDA, MOE_ERR_TIMEOUT, MOE_ERR_BAD_INDEX = 5, 6, 7
 MOE_GEMM_AUTO, MOE_GEMM_LARGE_M, MOE_GEMM_SMALL_M, MOE_GEMM_VALIDATION = 0, 1, 2, 3
 MOE_WEIGHTS_BF16, MOE_WEIGHTS_FP8_E4M3 = 0, 1
+MOE_BOUNDARY_YIELD = -1
 
 STATUS_NAMES = {0: "MOE_OK", 1: "MOE_ERR_INVALID_ARG", 2: "MOE_ERR_CAPACITY", 3: "MOE_ERR_STATE",
                 4: "MOE_ERR_UNSUPPORTED", 5: "MOE_ERR_CUDA", 6: "MOE_ERR_TIMEOUT", 7: "MOE_ERR_BAD_INDEX"}
@@ -33,7 +34,8 @@ EXPORTS = ("moe_version", "moe_ctx_workspace_bytes", "moe_ctx_create", "moe_ctx_
            "moe_dispatch_layout_static", "moe_ctx_set_segments", "moe_ctx_abandon_step", "moe_turnstile_create", "moe_turnstile_destroy",
            "moe_turnstile_set_span", "moe_turnstile_begin_epoch", "moe_turnstile_publish", "moe_turnstile_task_done",
            "moe_turnstile_d_enter", "moe_turnstile_d_release", "moe_turnstile_state", "moe_ctx_set_wait_limit",
-           "moe_ctx_debug_inject_stall", "moe_dispatch_notify", "moe_dispatch_move", "moe_ctx_pending_dispatch")
+           "moe_ctx_debug_inject_stall", "moe_dispatch_notify", "moe_dispatch_move", "moe_ctx_pending_dispatch",
+           "moe_ctx_set_preemption", "moe_ctx_request_yield", "moe_ctx_yield_count")
 
 BOUNDARY_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32)
 
@@ -120,6 +122,12 @@ def load_library() -> ctypes.CDLL:
                        ("moe_turnstile_state", [vp, ctypes.POINTER(i64)] + [ctypes.POINTER(i32)] * 4)):
         getattr(lib, name).restype = i32
         getattr(lib, name).argtypes = args
+    lib.moe_ctx_set_preemption.restype = i32
+    lib.moe_ctx_set_preemption.argtypes = [vp, i32]
+    lib.moe_ctx_request_yield.restype = i32
+    lib.moe_ctx_request_yield.argtypes = [vp, i32]
+    lib.moe_ctx_yield_count.restype = i64
+    lib.moe_ctx_yield_count.argtypes = [vp]
     lib.moe_dispatch_notify.restype = i32
     lib.moe_dispatch_notify.argtypes = [vp, vp, i32, vp, vp, vp, vp]
     lib.moe_dispatch_move.restype = i32
@@ -242,6 +250,16 @@ class MoeContext:
 
     def moe_ctx_abandon_step(self):
         self._check(self.lib.moe_ctx_abandon_step(self.handle))
+
+    def moe_ctx_set_preemption(self, enabled: bool):
+        self._check(self.lib.moe_ctx_set_preemption(self.handle, int(bool(enabled))))
+
+    def moe_ctx_request_yield(self, on: bool) -> int:
+        """Callable from any host thread; returns the status code instead of raising."""
+        return int(self.lib.moe_ctx_request_yield(self.handle, int(bool(on))))
+
+    def moe_ctx_yield_count(self) -> int:
+        return int(self.lib.moe_ctx_yield_count(self.handle))
 
     def moe_ctx_set_wait_limit(self, limit_us: int):
         self._check(self.lib.moe_ctx_set_wait_limit(self.handle, int(limit_us)))

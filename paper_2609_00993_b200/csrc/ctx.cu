@@ -56,7 +56,11 @@ struct Layout {
   int n_sets;
 };
 
-constexpr size_t kStatusBlock = 256;
+// Status block at the start of the workspace: word 0 the device status, word 1 the count of CTAs that stopped on a
+// yield request in the last preemptible launch, and from byte 256 on the per-CTA progress of a preemptible pass.
+constexpr size_t kStatusBlock = 8192;
+constexpr size_t kProgressOffset = 256;
+constexpr int kProgressInts = (int)((kStatusBlock - kProgressOffset) / sizeof(int));
 
 // Walks the carve of one buffer set; with base == nullptr it only measures.
 size_t carve_set(const moe_config& c, char* base, BufferSet* out) {
@@ -192,6 +196,12 @@ struct moe_ctx {
   } slots[MOE_HOST_SLOTS];
   cudaStream_t h2d_stream, d2h_stream;
   bool host_pipeline;
+  // preemption of prefill GEMM passes at tile granularity (off by default)
+  bool preemptible;
+  int* yield_host;    // mapped pinned host word: non-zero = yield requested (written by any host thread)
+  int* yield_dev;     // the same word as the device sees it
+  int* stopped_host;  // pinned host word: CTAs that stopped in the last launch
+  int64_t yields;     // launches that ended on a yield request
   unsigned long long wait_limit_ns;  // time limit of every bounded device-side wait (0 = the kernels' default)
   bool debug_stall;                  // failure-detection hook: the GEMM producers issue no copies
   char err[256];
@@ -292,6 +302,7 @@ int gemm_variant_of(const moe_ctx* ctx, const moe::GemmProblem& p) {
   if (v != MOE_GEMM_AUTO) return v;
   if (ctx->cfg.phase == MOE_PHASE_DECODE) return MOE_GEMM_SMALL_M;
   if (ctx->cfg.row_gather == 1) return MOE_GEMM_LARGE_M;  // only the large-M kernel gathers its rows itself
+  if (ctx->preemptible) return MOE_GEMM_SMALL_M;          // only the small-M kernel can stop between tiles
   const int64_t limit = p.fp8 ? kSmallMRowsFp8 : (p.gated ? kSmallMRowsGated : kSmallMRowsDown);
   return p.rows_bound <= limit * p.E ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M;  // p.E = 1 for a dense problem
 }
@@ -314,6 +325,29 @@ cudaError_t run_gemm(moe_ctx* ctx, moe::GemmProblem p, const moe::GemmDenseGroup
       moe::GemmProblem d{dense->A, dense->W, dense->out, nullptr, dense->rows, dense->rows, dense->rows, 1,
                          dense->n_feat, dense->K, p.gated};
       e = moe::launch_gemm_validation(d, ctx->stream, n);
+    }
+    return e;
+  }
+  if (variant == MOE_GEMM_SMALL_M && ctx->preemptible && !capturing(ctx)) {
+    // A pass that can be asked to stop between tiles: launch, wait on the host for the launch to end, and if
+    // CTAs stopped on a yield request report the boundary and launch again (each CTA resumes where it stopped).
+    int* progress = reinterpret_cast<int*>(ctx->ws + kProgressOffset);
+    int* stopped = ctx->status + 1;
+    if (gemm_ctas(ctx) > kProgressInts) return cudaErrorNotSupported;
+    p.progress = progress;
+    p.stopped = stopped;
+    cudaError_t e = cudaMemsetAsync(progress, 0, sizeof(int) * (size_t)gemm_ctas(ctx), ctx->stream);
+    for (int attempt = 0; e == cudaSuccess; ++attempt) {
+      // a request that is still up after the hook has returned is honoured once more, then overridden: the pass
+      // must end even with a controller that never clears its request
+      p.yield_req = attempt < 64 ? ctx->yield_dev : nullptr;
+      e = cudaMemsetAsync(stopped, 0, sizeof(int), ctx->stream);
+      if (e == cudaSuccess) e = moe::launch_gemm_stream(p, dense, gemm_ctas(ctx), ctx->status, ctx->stream, n);
+      if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->stopped_host, stopped, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream);
+      if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+      if (e != cudaSuccess || *ctx->stopped_host == 0) break;
+      ++ctx->yields;
+      if (ctx->boundary_fn) ctx->boundary_fn(ctx->boundary_user, MOE_BOUNDARY_YIELD, 0);
     }
     return e;
   }
@@ -399,6 +433,9 @@ moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspa
   ctx->host_pipeline = false;
   ctx->wait_limit_ns = 0;
   ctx->debug_stall = false;
+  ctx->preemptible = false;
+  ctx->yield_host = ctx->yield_dev = ctx->stopped_host = nullptr;
+  ctx->yields = 0;
   const size_t staging_bytes = carve_staging(*cfg, nullptr, nullptr);
   for (int s = 0; s < MOE_HOST_SLOTS; ++s) {
     BufferSet st = ctx->sets[s < l.n_sets ? s : 0];
@@ -483,6 +520,8 @@ moe_status moe_ctx_destroy(moe_ctx* ctx) {
   }
   cudaEventDestroy(ctx->done);
   cudaEventDestroy(ctx->notified);
+  if (ctx->yield_host) cudaFreeHost(ctx->yield_host);
+  if (ctx->stopped_host) cudaFreeHost(ctx->stopped_host);
   for (auto& sp : ctx->spans) {
     cudaEventDestroy(sp.beg);
     cudaEventDestroy(sp.end);
@@ -1008,6 +1047,42 @@ moe_status moe_ctx_set_segments(moe_ctx* ctx, int32_t experts_per_segment, moe_b
   ctx->boundary_user = user;
   return MOE_OK;
 }
+
+moe_status moe_ctx_set_preemption(moe_ctx* ctx, int32_t enabled) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->state != ST_IDLE) return fail(ctx, MOE_ERR_STATE, "preemption can only change between steps");
+  if (enabled && ctx->cfg.phase != MOE_PHASE_PREFILL)
+    return fail(ctx, MOE_ERR_INVALID_ARG, "only a PREFILL context can be made preemptible");
+  if (enabled && ctx->yield_host == nullptr) {
+    DeviceGuard guard(ctx->device);
+    void *y = nullptr, *sdev = nullptr, *st = nullptr;
+    cudaError_t e = cudaHostAlloc(&y, 64, cudaHostAllocMapped);
+    if (e == cudaSuccess) e = cudaHostGetDevicePointer(&sdev, y, 0);
+    if (e == cudaSuccess) e = cudaHostAlloc(&st, 64, cudaHostAllocDefault);
+    if (e != cudaSuccess) {
+      if (y) cudaFreeHost(y);
+      if (st) cudaFreeHost(st);
+      return cuda_fail(ctx, e, "moe_ctx_set_preemption");
+    }
+    memset(y, 0, 64);
+    memset(st, 0, 64);
+    ctx->yield_host = static_cast<int*>(y);
+    ctx->yield_dev = static_cast<int*>(sdev);
+    ctx->stopped_host = static_cast<int*>(st);
+  }
+  ctx->preemptible = enabled != 0;
+  if (ctx->yield_host) __atomic_store_n(ctx->yield_host, 0, __ATOMIC_RELEASE);
+  return MOE_OK;
+}
+
+moe_status moe_ctx_request_yield(moe_ctx* ctx, int32_t on) {
+  if (!ctx) return MOE_ERR_INVALID_ARG;
+  if (ctx->yield_host == nullptr) return MOE_ERR_STATE;  // preemption was never switched on (no message: any thread may call)
+  __atomic_store_n(ctx->yield_host, on ? 1 : 0, __ATOMIC_RELEASE);
+  return MOE_OK;
+}
+
+int64_t moe_ctx_yield_count(const moe_ctx* ctx) { return ctx ? ctx->yields : 0; }
 
 moe_status moe_ctx_set_wait_limit(moe_ctx* ctx, int64_t limit_us) {
   if (!ctx) return MOE_ERR_INVALID_ARG;

@@ -79,6 +79,10 @@ struct StreamParams {
   const float* row_scale2;
   const float* w_scale;
   const float* w_scale2;
+  // preemption at tile granularity (all null: off)
+  const int* yield_req;
+  int* progress;
+  int* stopped;
 };
 
 #ifdef MOE_STREAM_PROF
@@ -146,6 +150,26 @@ __device__ __forceinline__ STile decode_tile(int tile, int dense_tiles, int n_ft
   return t;
 }
 
+// mbar_wait that also ends when the producer has announced that wave `w` will not be started (*stop_w <= w).
+// 0: the barrier's phase completed; 1: time limit or abort; 2: the CTA stops before this wave.
+__device__ __forceinline__ int mbar_wait_or_stop(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                 unsigned long long limit_ns, const volatile int* stop_w, int w) {
+  unsigned long long t0 = 0;
+  for (uint32_t i = 0;; ++i) {
+    if (mbar_try_wait(bar, parity)) return 0;
+    if ((i & 31u) == 31u && *stop_w <= w) return mbar_try_wait(bar, parity) ? 0 : 2;
+    if (i >= 256u) {
+      if ((i & 255u) == 0u) {
+        if (*abort_flag) return 1;
+        const unsigned long long now = global_ns();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > limit_ns) return 1;
+      }
+      __nanosleep(64);
+    }
+  }
+}
+
 template <bool GATED, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
@@ -164,7 +188,8 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   const uint32_t bar_tempty = bar_tfull + 16u;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kNB + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* sizes = reinterpret_cast<int*>(tmem_slot + 2);  // slots held by the k-blocks in flight (producer only)
+  volatile int* stop_w = reinterpret_cast<volatile int*>(tmem_slot + 2);  // first wave this CTA will not start
+  int* sizes = reinterpret_cast<int*>(tmem_slot + 3);  // slots held by the k-blocks in flight (producer only)
   int* prefix = sizes + kNB;
   int* order = prefix + (p.E + 1);
   int* beg = order + p.E;
@@ -228,6 +253,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       mbar_init(bar_tempty + 8u * a, kEpilogueWarps);
     }
     *abort_flag = 0;
+    *stop_w = 0x7fffffff;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -238,6 +264,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   const uint32_t tmem_base = *tmem_slot;
   const int total_tiles = dense_tiles + prefix[p.E] * n_ft;
   const uint32_t R = (uint32_t)p.ring_slots;
+  const int w_first = p.progress ? p.progress[unit] : 0;  // a resumed pass continues where this CTA stopped
 
   if (warp == kProducerWarp) {
     // ================================================================= TMA producer (one lane)
@@ -246,9 +273,13 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       bool ok = true;
       [[maybe_unused]] long long prof_wait_empty = 0, prof_tiles = 0;
       [[maybe_unused]] const long long prof_start = clock64();
-      for (int w = 0; w * n_units < total_tiles && ok; ++w) {
+      for (int w = w_first; w * n_units < total_tiles && ok; ++w) {
         const int tile = snake_tile(w, unit, n_units);
         if (tile >= total_tiles) break;
+        if (p.yield_req != nullptr && *reinterpret_cast<const volatile int*>(p.yield_req) != 0) {
+          *stop_w = w;  // the other roles finish the waves below w and leave
+          break;
+        }
         const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
         const uint32_t n = (uint32_t)((t.rows + 15) & ~15);
         const uint32_t s = (uint32_t)kWSlots + (n >> 4);
@@ -306,7 +337,8 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       const uint32_t desc_hi = (uint32_t)(umma_smem_desc(0) >> 32);
       const uint32_t lo_base = (uint32_t)umma_smem_desc(base_addr);  // slot 0
       constexpr uint32_t lo_slot = (uint32_t)kSlotBytes >> 4, lo_box = (uint32_t)kWBoxBytes >> 4;
-      for (int w = 0; w * n_units < total_tiles && ok; ++w) {
+      bool stopped = false;
+      for (int w = w_first; w * n_units < total_tiles && ok && !stopped; ++w) {
         const int tile = snake_tile(w, unit, n_units);
         if (tile >= total_tiles) break;
         const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
@@ -341,9 +373,13 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
           head += s;
           {
             PROF_T0();
-            const bool got = mbar_wait(bar_full + 8u * (kb_idx % kNB), (kb_idx / kNB) & 1u, abort_flag, limit);
+            // the wait for a tile's first k-block also ends when the producer has decided not to start the tile
+            const uint32_t fb = bar_full + 8u * (kb_idx % kNB), fp = (kb_idx / kNB) & 1u;
+            const int got = kb == 0 ? mbar_wait_or_stop(fb, fp, abort_flag, limit, stop_w, w)
+                                    : (mbar_wait(fb, fp, abort_flag, limit) ? 0 : 1);
             PROF_ADD(prof_wait_full);
-            if (!got) { ok = false; break; }
+            if (got == 2) { stopped = true; break; }
+            if (got != 0) { ok = false; break; }
           }
           tc_fence_after();
           const uint32_t lo_w0 = lo_base + pos * lo_slot, lo_w1 = lo_w0 + lo_box, lo_x = lo_w0 + 2 * lo_box;
@@ -362,7 +398,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
           umma_commit(bar_empty + 8u * (kb_idx % kNB));  // the k-block's slots are free once these MMAs have read them
           ++kb_idx;
         }
-        if (!ok) break;
+        if (!ok || stopped) break;
         if (big) {
           umma_commit(bar_tfull);
           umma_commit(bar_tfull + 8u);
@@ -397,7 +433,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
     const uint32_t lane_base = ((uint32_t)(lg * 32)) << 16;
     const int fl = lg * 32 + lane;
     const bool even = (lane & 1) == 0;
-    for (int w = 0; w * n_units < total_tiles && ok; ++w) {
+    for (int w = w_first; w * n_units < total_tiles && ok; ++w) {
       const int tile = snake_tile(w, unit, n_units);
       if (tile >= total_tiles) break;
       const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
@@ -405,8 +441,9 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       const bool big = n > 128u;
       uint32_t h = 0, d_a, d_b;
       if (big) {
-        if (!mbar_wait(bar_tfull, use0 & 1u, abort_flag, limit) ||
-            !mbar_wait(bar_tfull + 8u, use1 & 1u, abort_flag, limit)) { ok = false; break; }
+        const int got = mbar_wait_or_stop(bar_tfull, use0 & 1u, abort_flag, limit, stop_w, w);
+        if (got == 2) break;  // the CTA stops before this wave
+        if (got != 0 || !mbar_wait(bar_tfull + 8u, use1 & 1u, abort_flag, limit)) { ok = false; break; }
         ++use0;
         ++use1;
         d_a = tmem_base;
@@ -414,7 +451,9 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       } else {
         h = next_half;
         next_half ^= 1u;
-        if (!mbar_wait(bar_tfull + 8u * h, (h ? use1 : use0) & 1u, abort_flag, limit)) { ok = false; break; }
+        const int got = mbar_wait_or_stop(bar_tfull + 8u * h, (h ? use1 : use0) & 1u, abort_flag, limit, stop_w, w);
+        if (got == 2) break;
+        if (got != 0) { ok = false; break; }
         if (h) ++use1; else ++use0;
         d_a = tmem_base + 256u * h;
         d_b = d_a + 128u;
@@ -500,6 +539,15 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   // ---- teardown
   tc_fence_before();
   __syncthreads();
+  if (p.progress != nullptr && threadIdx.x == 0) {
+    const int sw = *stop_w;
+    if (sw != 0x7fffffff) {  // stopped on request: the next launch of this pass resumes at wave sw
+      p.progress[unit] = sw;
+      atomicAdd(p.stopped, 1);
+    } else {
+      p.progress[unit] = (total_tiles + n_units - 1) / n_units;  // every wave done: a resumed launch finds nothing
+    }
+  }
   if (*abort_flag) {
     // give copies still in flight time to land in this CTA's shared memory before it is released
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
@@ -597,8 +645,12 @@ cudaError_t launch_gemm_stream(const GemmProblem& p, const GemmDenseGroup* dense
   prm.w_scale = p.w_scale;
   prm.row_scale2 = dense ? dense->row_scale : nullptr;
   prm.w_scale2 = dense ? dense->w_scale : nullptr;
+  const bool preemptible = p.yield_req != nullptr && p.progress != nullptr && p.stopped != nullptr;
+  prm.yield_req = preemptible ? p.yield_req : nullptr;
+  prm.progress = preemptible ? p.progress : nullptr;
+  prm.stopped = preemptible ? p.stopped : nullptr;
 
-  const size_t tail = (2 * kNB + 4) * sizeof(uint64_t) + 2 * sizeof(uint32_t) + kNB * sizeof(int) +
+  const size_t tail = (2 * kNB + 4) * sizeof(uint64_t) + 3 * sizeof(uint32_t) + kNB * sizeof(int) +
                       4 * (size_t)(prm.E + 1) * sizeof(int);
   const int slots = (int)((kSmemBudget - 1024 - (int)tail) / kSlotBytes);
   if (slots < 2 * (kWSlots + kMaxTileRows / 16)) return cudaErrorNotSupported;

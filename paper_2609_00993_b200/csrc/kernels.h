@@ -78,6 +78,14 @@ struct GemmProblem {
   // failure-detection hook (the TMA producer issues nothing, so every consumer wait runs into the limit).
   unsigned long long wait_limit_ns = 0;
   bool debug_stall = false;
+  // Preemption at tile granularity (small-M kernel only; all three null = off).  Before each of its tiles a CTA
+  // reads *yield_req; when it is non-zero the CTA finishes the tiles it has begun, stores the number of tiles it
+  // has done in progress[blockIdx.x], adds one to *stopped and exits.  A launch starts every CTA at
+  // progress[blockIdx.x], so launching the same problem again (same grid) resumes the pass; the caller zeroes
+  // progress before the first launch of a pass.  yield_req and stopped may live in mapped host memory.
+  const int* yield_req = nullptr;
+  int* progress = nullptr;
+  int* stopped = nullptr;
 };
 
 // A dense group (the shared expert) that rides in the same launch as a grouped problem: its tiles are added

@@ -401,6 +401,91 @@ def test_decode_step_admitted_between_notification_and_row_movement(fmt):
     p.close(); d.close()
 
 
+@pytest.mark.parametrize("fmt", [B.MOE_WEIGHTS_BF16, B.MOE_WEIGHTS_FP8_E4M3])
+def test_prefill_pass_yields_between_tiles_and_resumes_bit_identically(fmt):
+    """Preemption at tile granularity: a second host thread raises yield requests at random moments while P
+    steps run; the boundary hook (on P's thread) runs a whole D step on the other stream, lowers the request
+    and returns; the pass resumes.  Every P and every D result equals the one computed alone, bit for bit."""
+    import random
+    import threading
+    import time
+    fp8 = fmt == B.MOE_WEIGHTS_FP8_E4M3
+    shape = wl.LayerShape("t", T=32, H=1024, E=32, k=4, I=512, shared_I=256, select_bias=True)
+    pshape = shape.with_tokens(3000)
+    w = wl.make_weights_fp8(shape, 1, DEV) if fp8 else wl.make_weights(shape, 1, DEV)
+    ad, ap = wl.make_activations(shape, 2, DEV), wl.make_activations(pshape, 3, DEV)
+    sp, sd = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    d = B.MoeContext(B.make_config(1024, 32, 4, 512, 256, 32, B.MOE_PHASE_DECODE, weight_format=fmt), stream=sd)
+    p = B.MoeContext(B.make_config(1024, 32, 4, 512, 256, 3000, B.MOE_PHASE_PREFILL, weight_format=fmt), stream=sp)
+    bd, bp = B.alloc_step_buffers(32, 4, 32, DEV), B.alloc_step_buffers(3000, 4, 32, DEV)
+    d_out, p_out = (torch.empty(32, 1024, dtype=torch.bfloat16, device=DEV),
+                    torch.empty(3000, 1024, dtype=torch.bfloat16, device=DEV))
+
+    def step(ctx, a, out, bufs):
+        if fp8:
+            ctx.layer_fp8(a["x"], a["logits"], a["bias"], w, out=out, bufs=bufs)
+        else:
+            ctx.layer(a["x"], a["logits"], a["bias"], w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"],
+                      out=out, bufs=bufs)
+
+    torch.cuda.synchronize()
+    with torch.cuda.stream(sd):
+        step(d, ad, d_out, bd)
+    with torch.cuda.stream(sp):
+        step(p, ap, p_out, bp)
+    torch.cuda.synchronize()
+    d_alone, p_alone = d_out.clone(), p_out.clone()
+    assert p.moe_ctx_request_yield(True) == B.MOE_ERR_STATE   # preemption has not been switched on
+    p.moe_ctx_set_preemption(True)
+    d_runs = []
+
+    def hook(i, n):
+        assert i == B.MOE_BOUNDARY_YIELD
+        d_out.zero_()
+        with torch.cuda.stream(sd):
+            step(d, ad, d_out, bd)
+        sd.synchronize()
+        d_runs.append(torch.equal(d_out, d_alone))
+        p.moe_ctx_request_yield(False)     # the permit: P may go on
+
+    p.moe_ctx_set_segments(0, hook)
+    rng = random.Random(5)
+    stop = threading.Event()
+
+    def requester():
+        while not stop.is_set():
+            time.sleep(rng.uniform(0.0, 0.0015))
+            p.moe_ctx_request_yield(True)
+            time.sleep(0.0005)
+
+    th = threading.Thread(target=requester, daemon=True)
+    th.start()
+    try:
+        for it in range(40):
+            p_out.zero_()
+            with torch.cuda.stream(sp):
+                step(p, ap, p_out, bp)
+            sp.synchronize()
+            assert torch.equal(p_out, p_alone), f"P step {it} differs after {p.moe_ctx_yield_count()} yields"
+    finally:
+        stop.set()
+        th.join()
+        p.moe_ctx_request_yield(False)
+    assert p.moe_ctx_yield_count() >= 1 and d_runs and all(d_runs)
+    assert p.moe_ctx_status() == B.MOE_OK and d.moe_ctx_status() == B.MOE_OK
+    # with the request permanently up and a hook that never lowers it, a pass still ends
+    p.moe_ctx_set_segments(0, lambda i, n: None)
+    p.moe_ctx_request_yield(True)
+    p_out.zero_()
+    with torch.cuda.stream(sp):
+        step(p, ap, p_out, bp)
+    sp.synchronize()
+    assert torch.equal(p_out, p_alone)
+    p.moe_ctx_request_yield(False)
+    p.moe_ctx_set_preemption(False)
+    p.close(); d.close()
+
+
 def test_decode_step_replays_from_a_cuda_graph():
     """D retains stable graph addresses: a captured D step replays with new inputs written into the same
     tensors and gives the bits of the eager step, with a P context busy on another stream or idle."""
