@@ -2,7 +2,7 @@
 T in {1, 16, 128, 1024, 8192, 32768}.  For every T: layer time and tokens/s, per-stage device times, expert
 load imbalance, and the fraction of the layer's roofline floor that was reached.
 
-    python -m paper_2609_00993_b200.sweep [--tokens 1 16 128 ...] [--iters-min-ms 300] [--fp8]
+    python c5_sweep.py [--tokens 1 16 128 ...] [--iters-min-ms 300] [--fp8]
 
 One JSON object per T on stdout.  The floor of a step is the sum over its stages of
 max(flops / tensor peak, algorithmic bytes / HBM peak); for the grouped GEMMs it is summed per expert
@@ -15,12 +15,16 @@ import argparse
 import json
 import os
 
+import sys
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
 import torch
 
-from . import binding as B
-from . import workloads as wl
-
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+from paper_2609_00993_b200 import binding as B
+from paper_2609_00993_b200 import workloads as wl
 
 
 def load_peaks():

@@ -277,8 +277,11 @@ moe_status moe_ctx_set_segments(moe_ctx* ctx, int32_t experts_per_segment, moe_b
  * when the hook returns, launches the pass again: every CTA resumes where it stopped.  The hook is the permit
  * wait: it should return once the D step has finished on the device and the request has been lowered
  * (moe_ctx_request_yield(ctx, 0)); a request still up is honoured again (up to 64 launches per pass, after which
- * the pass runs to its end regardless).  Results are bit-identical to the unpreempted pass.  The first
- * moe_ctx_set_preemption(ctx, 1) allocates two small pinned host words (host memory, freed by moe_ctx_destroy).
+ * the pass runs to its end regardless).  Results are bit-identical to the unpreempted pass.  The request is a
+ * word in the context's workspace; raising it is a 4-byte asynchronous copy on a private stream of the context
+ * (it reaches the kernels within microseconds), lowering it also waits for that copy, so that a pass launched
+ * after the call returns cannot see a stale request.  The first moe_ctx_set_preemption(ctx, 1) creates that
+ * stream and two small pinned host buffers (host resources, released by moe_ctx_destroy).
  * moe_ctx_yield_count: launches that ended on a request since the context was created. */
 #define MOE_BOUNDARY_YIELD (-1)
 moe_status moe_ctx_set_preemption(moe_ctx* ctx, int32_t enabled);

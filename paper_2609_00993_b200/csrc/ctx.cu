@@ -57,7 +57,9 @@ struct Layout {
 };
 
 // Status block at the start of the workspace: word 0 the device status, word 1 the count of CTAs that stopped on a
-// yield request in the last preemptible launch, and from byte 256 on the per-CTA progress of a preemptible pass.
+// yield request in the last preemptible launch, word 2 the yield request itself (device memory: every CTA polls it
+// before each tile, which a word in host memory would not survive -- 148 SMs reading it over PCIe serialise), and
+// from byte 256 on the per-CTA progress of a preemptible pass.
 constexpr size_t kStatusBlock = 8192;
 constexpr size_t kProgressOffset = 256;
 constexpr int kProgressInts = (int)((kStatusBlock - kProgressOffset) / sizeof(int));
@@ -198,8 +200,10 @@ struct moe_ctx {
   bool host_pipeline;
   // preemption of prefill GEMM passes at tile granularity (off by default)
   bool preemptible;
-  int* yield_host;    // mapped pinned host word: non-zero = yield requested (written by any host thread)
-  int* yield_dev;     // the same word as the device sees it
+  int* yield_src;     // pinned host words {0, 1}: the sources of the copies that lower / raise the request
+  int* yield_dev;     // the request word in the status block
+  cudaStream_t yield_stream;  // private stream of those copies (any host thread may raise a request)
+  std::mutex* yield_mu;
   int* stopped_host;  // pinned host word: CTAs that stopped in the last launch
   int64_t yields;     // launches that ended on a yield request
   unsigned long long wait_limit_ns;  // time limit of every bounded device-side wait (0 = the kernels' default)
@@ -434,7 +438,9 @@ moe_status moe_ctx_create(const moe_config* cfg, void* workspace, size_t workspa
   ctx->wait_limit_ns = 0;
   ctx->debug_stall = false;
   ctx->preemptible = false;
-  ctx->yield_host = ctx->yield_dev = ctx->stopped_host = nullptr;
+  ctx->yield_src = ctx->yield_dev = ctx->stopped_host = nullptr;
+  ctx->yield_stream = nullptr;
+  ctx->yield_mu = nullptr;
   ctx->yields = 0;
   const size_t staging_bytes = carve_staging(*cfg, nullptr, nullptr);
   for (int s = 0; s < MOE_HOST_SLOTS; ++s) {
@@ -520,8 +526,10 @@ moe_status moe_ctx_destroy(moe_ctx* ctx) {
   }
   cudaEventDestroy(ctx->done);
   cudaEventDestroy(ctx->notified);
-  if (ctx->yield_host) cudaFreeHost(ctx->yield_host);
+  if (ctx->yield_src) cudaFreeHost(ctx->yield_src);
   if (ctx->stopped_host) cudaFreeHost(ctx->stopped_host);
+  if (ctx->yield_stream) cudaStreamDestroy(ctx->yield_stream);
+  delete ctx->yield_mu;
   for (auto& sp : ctx->spans) {
     cudaEventDestroy(sp.beg);
     cudaEventDestroy(sp.end);
@@ -1053,33 +1061,45 @@ moe_status moe_ctx_set_preemption(moe_ctx* ctx, int32_t enabled) {
   if (ctx->state != ST_IDLE) return fail(ctx, MOE_ERR_STATE, "preemption can only change between steps");
   if (enabled && ctx->cfg.phase != MOE_PHASE_PREFILL)
     return fail(ctx, MOE_ERR_INVALID_ARG, "only a PREFILL context can be made preemptible");
-  if (enabled && ctx->yield_host == nullptr) {
+  if (enabled && ctx->yield_src == nullptr) {
     DeviceGuard guard(ctx->device);
-    void *y = nullptr, *sdev = nullptr, *st = nullptr;
-    cudaError_t e = cudaHostAlloc(&y, 64, cudaHostAllocMapped);
-    if (e == cudaSuccess) e = cudaHostGetDevicePointer(&sdev, y, 0);
+    void *y = nullptr, *st = nullptr;
+    cudaStream_t ys = nullptr;
+    cudaError_t e = cudaHostAlloc(&y, 64, cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaHostAlloc(&st, 64, cudaHostAllocDefault);
-    if (e != cudaSuccess) {
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ys, cudaStreamNonBlocking);
+    std::mutex* mu = new (std::nothrow) std::mutex();
+    if (e != cudaSuccess || mu == nullptr) {
       if (y) cudaFreeHost(y);
       if (st) cudaFreeHost(st);
-      return cuda_fail(ctx, e, "moe_ctx_set_preemption");
+      if (ys) cudaStreamDestroy(ys);
+      delete mu;
+      return e != cudaSuccess ? cuda_fail(ctx, e, "moe_ctx_set_preemption") : fail(ctx, MOE_ERR_CUDA, "host allocation failed");
     }
     memset(y, 0, 64);
     memset(st, 0, 64);
-    ctx->yield_host = static_cast<int*>(y);
-    ctx->yield_dev = static_cast<int*>(sdev);
+    static_cast<int*>(y)[1] = 1;
+    ctx->yield_src = static_cast<int*>(y);
+    ctx->yield_dev = ctx->status + 2;
     ctx->stopped_host = static_cast<int*>(st);
+    ctx->yield_stream = ys;
+    ctx->yield_mu = mu;
   }
   ctx->preemptible = enabled != 0;
-  if (ctx->yield_host) __atomic_store_n(ctx->yield_host, 0, __ATOMIC_RELEASE);
+  if (ctx->yield_src) return moe_ctx_request_yield(ctx, 0);
   return MOE_OK;
 }
 
 moe_status moe_ctx_request_yield(moe_ctx* ctx, int32_t on) {
   if (!ctx) return MOE_ERR_INVALID_ARG;
-  if (ctx->yield_host == nullptr) return MOE_ERR_STATE;  // preemption was never switched on (no message: any thread may call)
-  __atomic_store_n(ctx->yield_host, on ? 1 : 0, __ATOMIC_RELEASE);
-  return MOE_OK;
+  if (ctx->yield_src == nullptr) return MOE_ERR_STATE;  // preemption was never switched on (no message: any thread may call)
+  DeviceGuard guard(ctx->device);
+  std::lock_guard<std::mutex> lock(*ctx->yield_mu);
+  cudaError_t e = cudaMemcpyAsync(ctx->yield_dev, ctx->yield_src + (on ? 1 : 0), sizeof(int), cudaMemcpyHostToDevice,
+                                  ctx->yield_stream);
+  // lowering is complete when this returns, so that a pass launched afterwards does not see a stale request
+  if (e == cudaSuccess && !on) e = cudaStreamSynchronize(ctx->yield_stream);
+  return e == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 int64_t moe_ctx_yield_count(const moe_ctx* ctx) { return ctx ? ctx->yields : 0; }

@@ -273,12 +273,21 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       bool ok = true;
       [[maybe_unused]] long long prof_wait_empty = 0, prof_tiles = 0;
       [[maybe_unused]] const long long prof_start = clock64();
+      int yield_seen = 0;
+      if (p.yield_req != nullptr)
+        asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(yield_seen) : "l"(p.yield_req) : "memory");
       for (int w = w_first; w * n_units < total_tiles && ok; ++w) {
         const int tile = snake_tile(w, unit, n_units);
         if (tile >= total_tiles) break;
-        if (p.yield_req != nullptr && *reinterpret_cast<const volatile int*>(p.yield_req) != 0) {
-          *stop_w = w;  // the other roles finish the waves below w and leave
-          break;
+        if (p.yield_req != nullptr) {
+          // the request word was read while the previous tile's copies were being issued, so looking at it here
+          // does not stall the pipeline; the read for the next tile goes out now
+          const int y = yield_seen;
+          asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(yield_seen) : "l"(p.yield_req) : "memory");
+          if (y != 0) {
+            *stop_w = w;  // the other roles finish the waves below w and leave
+            break;
+          }
         }
         const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
         const uint32_t n = (uint32_t)((t.rows + 15) & ~15);

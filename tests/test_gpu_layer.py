@@ -183,3 +183,47 @@ def test_c5_skewed_routing(v3_weights, T):
     if T >= 128:
         assert counts.max() * shape.E / counts.sum() > 8, "the Zipf popularity should skew the load"
     ctx.close()
+
+
+def test_c4_to_the_letter_fresh_inputs_every_iteration_with_sm_budgets(v3_weights):
+    """Config 4 as written: 200 iterations, each with fresh inputs (P seed 4000+i, D seed 5000+i), the P batch on
+    stream P and the D batch on stream D side by side with no ordering between them -- P's persistent grids capped
+    to 48 SMs, D's to 100 (the per-phase SM budgets).  Iterations 0, 99 and 199 are kept and must equal, bit for
+    bit, what each phase computes alone without a budget; they are compared with the oracle (every token of the
+    D batch, sampled tokens of the P batch)."""
+    w = v3_weights
+    sp, sd = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    mk = lambda s, ph, st, b: B.MoeContext(B.make_config(s.H, s.E, s.k, s.I, s.shared_I, s.T, ph, sm_budget=b), stream=st)
+    ctx_p, ctx_d = mk(wl.C4_P, B.MOE_PHASE_PREFILL, sp, 48), mk(wl.C4_D, B.MOE_PHASE_DECODE, sd, 100)
+    bp, bd = B.alloc_step_buffers(wl.C4_P.T, 8, 256, DEV), B.alloc_step_buffers(wl.C4_D.T, 8, 256, DEV)
+    op = torch.empty(wl.C4_P.T, 7168, dtype=torch.bfloat16, device=DEV)
+    od = torch.empty(wl.C4_D.T, 7168, dtype=torch.bfloat16, device=DEV)
+    wargs = (w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+    kept = {}
+    torch.cuda.synchronize()
+    for i in range(200):
+        ap, ad = wl.make_activations(wl.C4_P, 4000 + i, DEV), wl.make_activations(wl.C4_D, 5000 + i, DEV)
+        torch.cuda.synchronize()     # inputs are generated outside the concurrent region
+        ctx_p.layer(ap["x"], ap["logits"], ap["bias"], *wargs, out=op, bufs=bp)
+        ctx_d.layer(ad["x"], ad["logits"], ad["bias"], *wargs, out=od, bufs=bd)
+        torch.cuda.synchronize()
+        if i in (0, 99, 199):
+            kept[i] = (op.clone(), od.clone(), {k_: v.clone() for k_, v in bp.items()}, {k_: v.clone() for k_, v in bd.items()})
+    assert ctx_p.moe_ctx_status() == B.MOE_OK and ctx_d.moe_ctx_status() == B.MOE_OK
+    ctx_p.close(); ctx_d.close()
+    ref_p, ref_d = mk(wl.C4_P, B.MOE_PHASE_PREFILL, sp, 0), mk(wl.C4_D, B.MOE_PHASE_DECODE, sd, 0)
+    for i, (kop, kod, kbp, kbd) in kept.items():
+        ap, ad = wl.make_activations(wl.C4_P, 4000 + i, DEV), wl.make_activations(wl.C4_D, 5000 + i, DEV)
+        torch.cuda.synchronize()
+        ref_p.layer(ap["x"], ap["logits"], ap["bias"], *wargs, out=op, bufs=bp)
+        torch.cuda.synchronize()
+        ref_d.layer(ad["x"], ad["logits"], ad["bias"], *wargs, out=od, bufs=bd)
+        torch.cuda.synchronize()
+        assert torch.equal(op, kop) and torch.equal(od, kod), f"iteration {i}: side by side differs from alone"
+        assert torch.equal(bp["perm"], kbp["perm"]) and torch.equal(bd["perm"], kbd["perm"])
+        for name, shape, a, bufs, out in (("C4-P", wl.C4_P, ap, kbp, kop), ("C4-D", wl.C4_D, ad, kbd, kod)):
+            counts, offsets, perm = _check_integers(bufs, a["logits"], a["bias"], shape, shape.T)
+            toks = list(range(shape.T)) if shape.T <= 256 else sample_tokens_wide(shape.T, counts, offsets, perm, shape.k, 24, seed=i)[0]
+            ref, mag, _ = oracle_tokens_grouped(a["x"], bufs["topk_idx"], bufs["topk_w"], w, toks)
+            check_layer(out[toks], ref, mag, literal=False, label=f"{name} iteration {i} ({len(toks)} tokens)")
+    ref_p.close(); ref_d.close()
