@@ -118,11 +118,13 @@ def main():
     ap.add_argument("--experts", type=int, default=wl.C5.E,
                     help="number of routed experts (fewer than 256 keeps the weights small enough for a profiler capture)")
     ap.add_argument("--fp8", action="store_true", help="the FP8 (E4M3) precision variant instead of bf16")
+    ap.add_argument("--zipf", type=float, default=wl.C5.zipf_s,
+                    help="exponent of the expert popularity (0 = uniform routing with a selection bias, as in workloads C2/C4)")
     args = ap.parse_args()
     B.load_library()
     hbm, tfl, src = load_peaks()
     import dataclasses
-    base = dataclasses.replace(wl.C5, E=args.experts)
+    base = dataclasses.replace(wl.C5, E=args.experts, zipf_s=args.zipf, select_bias=args.zipf == 0)
     weights = (wl.make_weights_fp8 if args.fp8 else wl.make_weights)(base, 2, "cuda")
     for T in args.tokens:
         shape = base.with_tokens(T)
