@@ -204,7 +204,25 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   const int dense_tiles = p.rows2 > 0 ? ((p.rows2 + kMaxTileRows - 1) / kMaxTileRows) * n_ft2 : 0;
   const unsigned long long limit = p.wait_limit_ns;
 
-  // ---- set-up: tile list (experts ordered by size, largest first), barriers, TMEM
+  // ---- set-up: barriers and TMEM (before the previous kernel of the stream is known to be complete), then the
+  // tile list (experts ordered by size, largest first)
+  if (threadIdx.x == 32 * kProducerWarp) {
+    for (int s = 0; s < kNB; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, kIssuers);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8u * a, kIssuers);
+      mbar_init(bar_tempty + 8u * a, kEpilogueWarps);
+    }
+    *abort_flag = 0;
+    *stop_w = 0x7fffffff;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+  pdl_wait();
+  pdl_launch_dependents();
   for (int e = threadIdx.x; e < p.E; e += kThreads) {
     const int b = p.offsets ? p.offsets[e] : 0;
     int c = p.offsets ? p.offsets[e + 1] - b : p.fixed_rows;
@@ -243,21 +261,6 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
     }
     if (lane == 0) prefix[p.E] = carry;
   }
-  if (threadIdx.x == 32 * kProducerWarp) {
-    for (int s = 0; s < kNB; ++s) {
-      mbar_init(bar_full + 8u * s, 1);
-      mbar_init(bar_empty + 8u * s, kIssuers);
-    }
-    for (int a = 0; a < 2; ++a) {
-      mbar_init(bar_tfull + 8u * a, kIssuers);
-      mbar_init(bar_tempty + 8u * a, kEpilogueWarps);
-    }
-    *abort_flag = 0;
-    *stop_w = 0x7fffffff;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -573,8 +576,7 @@ cudaError_t launch_variant(Kernel kern, const CUtensorMap& mw, const CUtensorMap
                            const StreamParams& prm, int grid, size_t smem, cudaStream_t stream) {
   cudaError_t err = ensure_dynamic_smem(kern, smem);
   if (err != cudaSuccess) return err;
-  kern<<<grid, kThreads, smem, stream>>>(mw, mw2, xm, prm);
-  return cudaGetLastError();
+  return launch_pdl(kern, dim3(grid), dim3(kThreads), smem, stream, mw, mw2, xm, prm);
 }
 
 }  // namespace

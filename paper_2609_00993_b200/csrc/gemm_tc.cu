@@ -171,7 +171,23 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   constexpr uint32_t acc_cols = 256u;  // TMEM columns per accumulator stage
   constexpr uint32_t tmem_cols = 2u * acc_cols;
 
-  // ---- set-up: tile list, barriers, TMEM
+  // ---- set-up: barriers, TMEM (both before the previous kernel of the stream is known to be complete), tile list
+  if (threadIdx.x == 32) {
+    for (int s = 0; s < p.n_stages; ++s) {
+      mbar_init(bar_full + 8u * s, GATHER ? 1 + kGatherThreads : 1);
+      mbar_init(bar_empty + 8u * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(bar_tfull + 8u * a, 1);
+      mbar_init(bar_tempty + 8u * a, kEpilogueWarps);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), tmem_cols);
+  pdl_wait();
+  pdl_launch_dependents();
   if (warp == 0) {
     int carry = 0;
     for (int b = 0; b < p.E; b += 32) {
@@ -196,20 +212,6 @@ grouped_gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     }
     if (lane == 0) prefix[p.E] = carry;
   }
-  if (threadIdx.x == 32) {
-    for (int s = 0; s < p.n_stages; ++s) {
-      mbar_init(bar_full + 8u * s, GATHER ? 1 + kGatherThreads : 1);
-      mbar_init(bar_empty + 8u * s, 1);
-    }
-    for (int a = 0; a < 2; ++a) {
-      mbar_init(bar_tfull + 8u * a, 1);
-      mbar_init(bar_tempty + 8u * a, kEpilogueWarps);
-    }
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), tmem_cols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -494,8 +496,7 @@ cudaError_t launch_variant(Kernel kern, int threads, const CUtensorMap& mx, cons
                            int grid, size_t smem, cudaStream_t stream) {
   cudaError_t err = ensure_dynamic_smem(kern, smem);
   if (err != cudaSuccess) return err;
-  kern<<<grid, threads, smem, stream>>>(mx, mw, mx2, mw2, om, prm);
-  return cudaGetLastError();
+  return launch_pdl(kern, dim3(grid), dim3(threads), smem, stream, mx, mw, mx2, mw2, om, prm);
 }
 
 }  // namespace

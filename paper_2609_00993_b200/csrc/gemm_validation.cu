@@ -21,6 +21,8 @@ gemm_validation_kernel(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16*
   __shared__ float Wg[kStepK][kTile + 1];
   __shared__ float Wu[GATED ? kStepK : 1][kTile + 1];
   __shared__ int s_e, s_row0, s_rows;
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (threadIdx.x == 0) {  // which expert and which 64-row tile of it does blockIdx.y name?
     int tile = blockIdx.y, e = 0, found = -1, r0 = 0, nr = 0;
@@ -99,8 +101,8 @@ cudaError_t launch_gemm_validation(const GemmProblem& p, cudaStream_t stream, in
   const int E = e_end - e_begin;  // experts of this launch
   const int32_t* offs = p.offsets ? p.offsets + e_begin : nullptr;
   W += (size_t)e_begin * (size_t)(p.gated ? 2 : 1) * p.n_feat * p.K;
-  if (p.gated) gemm_validation_kernel<true><<<grid, 256, 0, stream>>>(A, W, out, offs, p.fixed_rows, E, p.n_feat, p.K);
-  else gemm_validation_kernel<false><<<grid, 256, 0, stream>>>(A, W, out, offs, p.fixed_rows, E, p.n_feat, p.K);
+  if (p.gated) (void)launch_pdl(gemm_validation_kernel<true>, grid, dim3(256), 0, stream, A, W, out, offs, p.fixed_rows, E, p.n_feat, p.K);
+  else (void)launch_pdl(gemm_validation_kernel<false>, grid, dim3(256), 0, stream, A, W, out, offs, p.fixed_rows, E, p.n_feat, p.K);
   cudaError_t err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;

@@ -14,6 +14,34 @@ inline cudaError_t ensure_dynamic_smem(Kernel kern, size_t bytes) {
   return ensure_dynamic_smem_impl(reinterpret_cast<const void*>(kern), bytes);
 }
 
+// Programmatic dependent launch: every kernel of the library is launched with "programmatic stream serialization
+// allowed", so its CTAs may become resident and run their prologue (barrier set-up, tensor-memory allocation,
+// tensor-map prefetch) while the previous kernel of the stream is still draining; pdl_wait() then blocks until that
+// kernel has completed and its writes are visible.  Rules: every thread calls pdl_wait() before its first access to
+// global memory (reads AND writes: the predecessor may still be reading what this kernel overwrites), and
+// pdl_launch_dependents() right after it, which lets the NEXT kernel start its own prologue as soon as SM resources
+// free up.  A step of six dependent kernels sheds the launch latency and prologue of each of them this way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Device status codes (same values as moe_status in the public header).
 constexpr int kStOk = 0;
 constexpr int kStTimeout = 6;

@@ -128,6 +128,8 @@ __global__ void __launch_bounds__(kFusedWarps * 32)
 layout_fused_kernel(const int32_t* __restrict__ topk_idx, int n_slots, int E, int slots_per_warp,
                     int32_t* __restrict__ counts, int32_t* __restrict__ offsets, int32_t* __restrict__ perm,
                     int32_t* __restrict__ inv_perm, int* status) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ int sh[];
   int* hist = sh;
   int* offsets_sh = hist + kFusedWarps * E;
@@ -165,6 +167,8 @@ layout_fused_kernel(const int32_t* __restrict__ topk_idx, int n_slots, int E, in
 __global__ void __launch_bounds__(kChunkWarpsPerBlock * 32)
 layout_count_kernel(const int32_t* __restrict__ topk_idx, int64_t n_slots, int E, int n_chunks,
                     int32_t* __restrict__ chunk_counts, int* status) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ int sh[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunk = blockIdx.x * kChunkWarpsPerBlock + warp;
@@ -185,6 +189,8 @@ layout_count_kernel(const int32_t* __restrict__ topk_idx, int64_t n_slots, int E
 //     at most kBatch chunks (up to 65536 slots) is read once and kept in registers for the second walk.
 __global__ void __launch_bounds__(1024)
 layout_scan_kernel(int32_t* __restrict__ chunk_counts, int n_chunks, int E, int32_t* __restrict__ counts) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ int partial[32][33];
   const int lane = threadIdx.x & 31, part = threadIdx.x >> 5;
   const int e = blockIdx.x * 32 + lane;
@@ -236,6 +242,8 @@ __global__ void __launch_bounds__(kChunkWarpsPerBlock * 32)
 layout_place_kernel(const int32_t* __restrict__ topk_idx, int64_t n_slots, int E, int n_chunks,
                     const int32_t* __restrict__ chunk_prefix, const int32_t* __restrict__ counts,
                     int32_t* __restrict__ offsets, int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm) {
+  pdl_wait();
+  pdl_launch_dependents();
   extern __shared__ int sh[];
   int* counts_sh = sh + kChunkWarpsPerBlock * E;
   int* offsets_sh = counts_sh + E;
@@ -255,6 +263,8 @@ layout_place_kernel(const int32_t* __restrict__ topk_idx, int64_t n_slots, int E
 }
 
 __global__ void layout_empty_kernel(int E, int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+  pdl_wait();
+  pdl_launch_dependents();
   for (int e = threadIdx.x; e <= E; e += blockDim.x) {
     if (e < E) counts[e] = 0;
     offsets[e] = 0;
@@ -268,8 +278,7 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
                           int* n_launches) {
   cudaError_t err;
   if (n_slots <= 0) {
-    layout_empty_kernel<<<1, 256, 0, stream>>>(E, counts, offsets);
-    err = cudaGetLastError();
+    err = launch_pdl(layout_empty_kernel, dim3(1), dim3(256), 0, stream, E, counts, offsets);
     if (err == cudaSuccess && n_launches) *n_launches += 1;
     return err;
   }
@@ -278,22 +287,19 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
     int spw = (int)((n_slots + kFusedWarps - 1) / kFusedWarps);
     spw = (spw + 31) / 32 * 32;
     if ((err = ensure_dynamic_smem(layout_fused_kernel, fused_smem)) != cudaSuccess) return err;
-    layout_fused_kernel<<<1, kFusedWarps * 32, fused_smem, stream>>>(topk_idx, (int)n_slots, E, spw, counts, offsets,
+    err = launch_pdl(layout_fused_kernel, dim3(1), dim3(kFusedWarps * 32), fused_smem, stream, topk_idx, (int)n_slots, E, spw, counts, offsets,
                                                                      perm, inv_perm, status);
-    err = cudaGetLastError();
     if (err == cudaSuccess && n_launches) *n_launches += 1;
     return err;
   }
   const int n_chunks = (int)((n_slots + kLayoutChunk - 1) / kLayoutChunk);
   const int blocks = (n_chunks + kChunkWarpsPerBlock - 1) / kChunkWarpsPerBlock;
   const size_t chunk_smem = (size_t)kChunkWarpsPerBlock * E * sizeof(int);
-  layout_count_kernel<<<blocks, kChunkWarpsPerBlock * 32, chunk_smem, stream>>>(topk_idx, n_slots, E, n_chunks,
-                                                                                scratch, status);
-  if ((err = cudaGetLastError()) != cudaSuccess) return err;
-  layout_scan_kernel<<<(E + 31) / 32, 1024, 0, stream>>>(scratch, n_chunks, E, counts);
-  if ((err = cudaGetLastError()) != cudaSuccess) return err;
+  if ((err = launch_pdl(layout_count_kernel, dim3(blocks), dim3(kChunkWarpsPerBlock * 32), chunk_smem, stream, topk_idx, n_slots, E, n_chunks,
+                                                                                scratch, status)) != cudaSuccess) return err;
+  if ((err = launch_pdl(layout_scan_kernel, dim3((E + 31) / 32), dim3(1024), 0, stream, scratch, n_chunks, E, counts)) != cudaSuccess) return err;
   const size_t place_smem = chunk_smem + ((size_t)E + (E + 1) + 33) * sizeof(int);
-  layout_place_kernel<<<blocks, kChunkWarpsPerBlock * 32, place_smem, stream>>>(topk_idx, n_slots, E, n_chunks,
+  launch_pdl(layout_place_kernel, dim3(blocks), dim3(kChunkWarpsPerBlock * 32), place_smem, stream, topk_idx, n_slots, E, n_chunks,
                                                                                 scratch, counts, offsets, perm,
                                                                                 inv_perm);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;

@@ -32,6 +32,8 @@ __global__ void __launch_bounds__(kQuantThreads)
 quantize_rows_kernel(const uint4* __restrict__ x, long long rows, int n_vec, uint2* __restrict__ q,
                      float* __restrict__ scale) {
   __shared__ uint32_t warp_max[kQuantThreads / 32];
+  pdl_wait();
+  pdl_launch_dependents();
   constexpr int kRowThreads = 32 * ROW_WARPS;
   const int tid = ROW_WARPS == 1 ? (int)(threadIdx.x & 31) : (int)threadIdx.x;
   const long long row = ROW_WARPS == 1 ? (long long)blockIdx.x * (kQuantThreads / 32) + (threadIdx.x >> 5)
@@ -81,15 +83,15 @@ cudaError_t launch_quantize_rows(const void* x, int64_t rows, int n, void* q, fl
   if (rows <= 0) return cudaSuccess;
   if (n <= 0 || n % 8 != 0 || n > 8 * kQuantThreads * kQuantMaxVecs || rows > 0x7fffffffLL) return cudaErrorNotSupported;
   const int n_vec = n / 8;
+  cudaError_t err;
   if (n_vec <= 32 * kQuantMaxVecs) {
     const long long blocks = (rows + kQuantThreads / 32 - 1) / (kQuantThreads / 32);
-    quantize_rows_kernel<1><<<(unsigned)blocks, kQuantThreads, 0, stream>>>(static_cast<const uint4*>(x), rows, n_vec,
-                                                                            static_cast<uint2*>(q), scale);
+    err = launch_pdl(quantize_rows_kernel<1>, dim3((unsigned)blocks), dim3(kQuantThreads), 0, stream,
+                     static_cast<const uint4*>(x), (long long)rows, n_vec, static_cast<uint2*>(q), scale);
   } else {
-    quantize_rows_kernel<4><<<(unsigned)rows, kQuantThreads, 0, stream>>>(static_cast<const uint4*>(x), rows, n_vec,
-                                                                          static_cast<uint2*>(q), scale);
+    err = launch_pdl(quantize_rows_kernel<4>, dim3((unsigned)rows), dim3(kQuantThreads), 0, stream,
+                     static_cast<const uint4*>(x), (long long)rows, n_vec, static_cast<uint2*>(q), scale);
   }
-  cudaError_t err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }

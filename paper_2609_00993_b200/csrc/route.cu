@@ -24,6 +24,8 @@ template <int VPT, bool VEC>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 route_kernel(const float* __restrict__ logits, const float* __restrict__ bias, int T, int E, int k, float scale,
              int32_t* __restrict__ idx, float* __restrict__ w) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int lane = threadIdx.x & 31;
   const int t = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
   if (t >= T) return;
@@ -104,12 +106,12 @@ cudaError_t launch_vpt(bool vec, const float* logits, const float* bias, int T, 
   const int blocks = (T + kWarpsPerBlock - 1) / kWarpsPerBlock;
   if constexpr (VPT >= 4) {
     if (vec) {
-      route_kernel<VPT, true><<<blocks, kWarpsPerBlock * 32, 0, stream>>>(logits, bias, T, E, k, scale, idx, w);
-      return cudaGetLastError();
+      return launch_pdl(route_kernel<VPT, true>, dim3(blocks), dim3(kWarpsPerBlock * 32), 0, stream, logits, bias, T, E, k,
+                        scale, idx, w);
     }
   }
-  route_kernel<VPT, false><<<blocks, kWarpsPerBlock * 32, 0, stream>>>(logits, bias, T, E, k, scale, idx, w);
-  return cudaGetLastError();
+  return launch_pdl(route_kernel<VPT, false>, dim3(blocks), dim3(kWarpsPerBlock * 32), 0, stream, logits, bias, T, E, k, scale,
+                    idx, w);
 }
 
 }  // namespace

@@ -102,6 +102,8 @@ permute_rows_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restri
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncwarp();
+  pdl_wait();  // the barriers are set up; nothing of the previous kernel's results has been touched yet
+  pdl_launch_dependents();
 
   auto item_of = [&](long long n) { return (long long)blockIdx.x + n * gridDim.x; };
   auto issue_load = [&](long long n) {  // lane 0 only
@@ -184,6 +186,8 @@ combine_kernel(const __nv_bfloat16* __restrict__ y_perm, const __nv_bfloat16* __
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (warp == kCombineConsumers / 32) {
     // ============================================================ producer warp: lane j gathers row j
@@ -293,11 +297,9 @@ cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm,
   const long long n_items = (long long)T * col_blocks;
   const long long cap = resident_ctas(reinterpret_cast<const void*>(permute_rows_kernel), 32, smem);
   const int grid = (int)(n_items < cap ? n_items : cap);
-  permute_rows_kernel<<<grid, 32, smem, stream>>>(static_cast<const __nv_bfloat16*>(x), inv_perm,
-                                                  static_cast<__nv_bfloat16*>(x_perm), T, k, H, col_blocks, slot_bytes,
-                                                  row_val, row_val_perm, status,
-                                                  wait_limit_ns ? wait_limit_ns : kWaitLimitNs);
-  err = cudaGetLastError();
+  err = launch_pdl(permute_rows_kernel, dim3(grid), dim3(32), smem, stream, static_cast<const __nv_bfloat16*>(x), inv_perm,
+                   static_cast<__nv_bfloat16*>(x_perm), T, k, H, col_blocks, slot_bytes, row_val, row_val_perm, status,
+                   wait_limit_ns ? wait_limit_ns : kWaitLimitNs);
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }
@@ -320,16 +322,13 @@ cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32
     const long long n_items = (long long)T * col_blocks;
     const long long cap = resident_ctas(reinterpret_cast<const void*>(kern), kCombineThreads, smem);
     const int grid = (int)(n_items < cap ? n_items : cap);
-    kern<<<grid, kCombineThreads, smem, stream>>>(
-        static_cast<const __nv_bfloat16*>(y_perm), static_cast<const __nv_bfloat16*>(y_shared), inv_perm, topk_w,
-        static_cast<__nv_bfloat16*>(out), T, k, H, col_blocks, chunk_bytes, stage_bytes, stages, status,
-        wait_limit_ns ? wait_limit_ns : kWaitLimitNs);
-    return cudaSuccess;
+    return launch_pdl(kern, dim3(grid), dim3(kCombineThreads), smem, stream, static_cast<const __nv_bfloat16*>(y_perm),
+                      static_cast<const __nv_bfloat16*>(y_shared), inv_perm, topk_w, static_cast<__nv_bfloat16*>(out), T, k,
+                      H, col_blocks, chunk_bytes, stage_bytes, stages, status,
+                      wait_limit_ns ? wait_limit_ns : kWaitLimitNs);
   };
   cudaError_t err = k == 8 ? launch(combine_kernel<8>) : k == 4 ? launch(combine_kernel<4>)
                   : k == 2 ? launch(combine_kernel<2>) : launch(combine_kernel<0>);
-  if (err != cudaSuccess) return err;
-  err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }
