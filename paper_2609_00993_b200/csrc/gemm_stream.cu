@@ -490,11 +490,24 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       // values for them (features f, f+1 of one token are one 4-byte store); the odd lane does the same for
       // the odd tokens.  n_feat is a multiple of 8, so a pair is inside the row or outside it as a whole.
       const int f_pair = (GATED ? f_a : 0) & ~1;
+      // the loads of the next 16-token chunk are in flight while this one is converted and stored
+      uint32_t na[16], nb[16];
+      if (c_first < t.rows) {
+        tmem_ld16(d_a + (uint32_t)c_first, na);
+        tmem_ld16(d_b + (uint32_t)c_first, nb);
+      }
       for (int c = c_first; c < t.rows; c += c_step) {
         uint32_t ra[16], rb[16];
-        tmem_ld16(d_a + (uint32_t)c, ra);
-        tmem_ld16(d_b + (uint32_t)c, rb);
         tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          ra[i] = na[i];
+          rb[i] = nb[i];
+        }
+        if (c + c_step < t.rows) {
+          tmem_ld16(d_a + (uint32_t)(c + c_step), na);
+          tmem_ld16(d_b + (uint32_t)(c + c_step), nb);
+        }
         float va[16], vb[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {

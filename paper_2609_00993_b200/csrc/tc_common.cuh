@@ -190,7 +190,21 @@ __device__ __forceinline__ uint32_t umma_idesc_e4m3(uint32_t M, uint32_t N) {
   return (1u << 4) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
-__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
+// silu(g) * u with one special-function operation per element instead of two: t = 2^(-|g| log2 e) in (0,1] comes
+// from ex2.approx; the reciprocal of d = 1 + t in (1,2] is a linear seed (24/17 - 8/17 d, relative error <= 1/17)
+// refined by two Newton steps on the FMA pipe (relative error <= 1.2e-5, far below the bf16 rounding that follows);
+// sigmoid(g) = 1/d for g >= 0 and t/d for g < 0, so small sigmoids keep their relative accuracy.  The epilogue
+// of a GEMM1 tile evaluates 32K of these, and the special-function unit (16 results per clock and SM) is what it
+// waits for.
+__device__ __forceinline__ float silu_mul(float g, float u) {
+  float t;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(-fabsf(g) * 1.4426950408889634f));
+  const float d = 1.0f + t;
+  float r = fmaf(d, -0.47058823529411764f, 1.4117647058823530f);
+  r = r * fmaf(-d, r, 2.0f);
+  r = r * fmaf(-d, r, 2.0f);
+  return g * (g >= 0.f ? r : t * r) * u;
+}
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
