@@ -137,6 +137,102 @@ def test_turnstile_under_skew(seed, span):
             assert since_release <= span, ev                      # R- < G < R+: at most one span between D iterations
 
 
+def _check_turnstile_log(log, span):
+    since_release = 0
+    for ev in log:
+        if ev[0] == "D":
+            _, e, reached, permit, active = ev
+            if active:
+                assert permit == 0 or reached >= permit, ev
+        elif ev[0] == "R":
+            since_release = 0
+        else:
+            _, e, i, permit_seen = ev
+            assert i < permit_seen, ev
+            since_release += 1
+            assert since_release <= span, ev
+
+
+def test_turnstile_stress_at_the_papers_scale():
+    """The model-free rank-skew stress at the scale the paper reports (Section "RQ3"): 2,560 P-segment / D-iteration
+    cycles per seed with up to 20 ms of injected skew on either side, five seeds.  The seeds run side by side
+    (the injected sleeps dominate), each with its own controller, P thread and D thread; every cycle must keep
+    the ordering invariants and every run must complete all 2,560 cycles."""
+    n_epochs, n_segments, span = 40, 64, 1
+    logs, failures = {}, []
+
+    def one(seed):
+        try:
+            log = []
+            _run_protocol(seed, n_epochs, n_segments, span, max_skew_ms=20.0, log=log)
+            logs[seed] = log
+        except BaseException as exc:  # surfaced in the main thread below
+            failures.append((seed, repr(exc)))
+
+    threads = [threading.Thread(target=one, args=(s,)) for s in range(5)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(600)
+    assert not failures, failures
+    for seed in range(5):
+        log = logs[seed]
+        assert sum(1 for x in log if x[0] == "P") == n_epochs * n_segments == 2560, seed
+        _check_turnstile_log(log, span)
+        # with span 1 every P segment was admitted by its own D iteration (plus the one that opens each epoch)
+        assert sum(1 for x in log if x[0] == "R") >= 2560, seed
+
+
+def test_d_release_does_not_wait_for_prefill_gpu_completion():
+    """The delayed-P control (Section "RQ3": P was still incomplete at D's acknowledgement in 20 of 64 steps): the
+    controller orders host ENQUEUE only, so a D iteration is acknowledged while the P segment enqueued before it
+    may still be executing.  P's device work is modelled as completing 4-12 ms after its enqueue; 64 D iterations
+    are counted, and some of them must find the last enqueued P segment incomplete while every ordering invariant
+    still holds."""
+    ts = B.Turnstile(1)
+    rng_p, rng_d = random.Random(11), random.Random(12)
+    complete_at = []          # device completion time of every P segment enqueued so far
+    incomplete_at_ack, acks, log, errors = [0], [0], [], []
+    done = threading.Event()
+
+    def p_thread():
+        assert ts.begin_epoch(0) == OK
+        if ts.publish(0, 0, 20000) != OK:
+            errors.append("publish 0"); return
+        for i in range(64):
+            complete_at.append(time.monotonic() + rng_p.uniform(0.004, 0.012))   # "enqueue": runs for 4-12 ms
+            log.append(("P", 0, i, ts.state()["permit"]))
+            if i + 1 < 64 and ts.publish(0, i + 1, 20000) != OK:
+                errors.append(f"publish {i + 1}"); return
+        assert ts.task_done(0) == OK
+        done.set()
+
+    def d_thread():
+        while not done.is_set():
+            time.sleep(rng_d.uniform(0.0, 0.010))
+            st, active = ts.d_enter(20000)
+            if st != OK:
+                errors.append("d_enter"); return
+            if active and complete_at:
+                acks[0] += 1
+                if time.monotonic() < complete_at[-1]:
+                    incomplete_at_ack[0] += 1                # D goes ahead although P's last segment is still running
+            s_ = ts.state()
+            log.append(("D", s_["epoch"], s_["reached"], s_["permit"], s_["active"]))
+            log.append(("R",))
+            ts.d_release()
+
+    tp, td = threading.Thread(target=p_thread), threading.Thread(target=d_thread)
+    tp.start(); td.start()
+    tp.join(60); td.join(60)
+    assert not tp.is_alive() and not td.is_alive() and not errors, errors
+    _check_turnstile_log(log, 1)
+    assert acks[0] >= 60
+    assert 0 < incomplete_at_ack[0] < acks[0], (incomplete_at_ack[0], acks[0])
+    print(f"P incomplete at D acknowledgement in {incomplete_at_ack[0]} of {acks[0]} steps")
+    assert ts.destroy() == OK
+
+
 def _free_port():
     with socket.socket() as s:
         s.bind(("127.0.0.1", 0))
