@@ -586,10 +586,10 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
 
 template <typename Kernel>
 cudaError_t launch_variant(Kernel kern, const CUtensorMap& mw, const CUtensorMap& mw2, const StreamMaps& xm,
-                           const StreamParams& prm, int grid, size_t smem, cudaStream_t stream) {
+                           const StreamParams& prm, int grid, size_t smem, cudaStream_t stream, bool overlap) {
   cudaError_t err = ensure_dynamic_smem(kern, smem);
   if (err != cudaSuccess) return err;
-  return launch_pdl(kern, dim3(grid), dim3(kThreads), smem, stream, mw, mw2, xm, prm);
+  return launch_pdl(overlap, kern, dim3(grid), dim3(kThreads), smem, stream, mw, mw2, xm, prm);
 }
 
 }  // namespace
@@ -689,13 +689,14 @@ cudaError_t launch_gemm_stream(const GemmProblem& p, const GemmDenseGroup* dense
     tiles += (int64_t)((dense->rows + kMaxTileRows - 1) / kMaxTileRows) * ((dense->n_feat + feat_per_tile - 1) / feat_per_tile);
   int grid = (int)(tiles < (int64_t)max_ctas ? tiles : (int64_t)max_ctas);
   if (grid < 1) grid = 1;
+  const bool overlap = p.rows_bound <= kGemmOverlapMaxRows;
   cudaError_t err;
   if (fp8)
-    err = p.gated ? launch_variant(grouped_gemm_stream_kernel<true, true>, mw, mw2, xm, prm, grid, smem, stream)
-                  : launch_variant(grouped_gemm_stream_kernel<false, true>, mw, mw2, xm, prm, grid, smem, stream);
+    err = p.gated ? launch_variant(grouped_gemm_stream_kernel<true, true>, mw, mw2, xm, prm, grid, smem, stream, overlap)
+                  : launch_variant(grouped_gemm_stream_kernel<false, true>, mw, mw2, xm, prm, grid, smem, stream, overlap);
   else
-    err = p.gated ? launch_variant(grouped_gemm_stream_kernel<true, false>, mw, mw2, xm, prm, grid, smem, stream)
-                  : launch_variant(grouped_gemm_stream_kernel<false, false>, mw, mw2, xm, prm, grid, smem, stream);
+    err = p.gated ? launch_variant(grouped_gemm_stream_kernel<true, false>, mw, mw2, xm, prm, grid, smem, stream, overlap)
+                  : launch_variant(grouped_gemm_stream_kernel<false, false>, mw, mw2, xm, prm, grid, smem, stream, overlap);
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }

@@ -493,10 +493,10 @@ const char* g_init_error = nullptr;
 template <typename Kernel>
 cudaError_t launch_variant(Kernel kern, int threads, const CUtensorMap& mx, const CUtensorMap& mw,
                            const CUtensorMap& mx2, const CUtensorMap& mw2, const OutMaps& om, const TcParams& prm,
-                           int grid, size_t smem, cudaStream_t stream) {
+                           int grid, size_t smem, cudaStream_t stream, bool overlap) {
   cudaError_t err = ensure_dynamic_smem(kern, smem);
   if (err != cudaSuccess) return err;
-  return launch_pdl(kern, dim3(grid), dim3(threads), smem, stream, mx, mw, mx2, mw2, om, prm);
+  return launch_pdl(overlap, kern, dim3(grid), dim3(threads), smem, stream, mx, mw, mx2, mw2, om, prm);
 }
 
 }  // namespace
@@ -692,15 +692,16 @@ cudaError_t launch_gemm_tc(const GemmProblem& p, const GemmDenseGroup* dense, in
 
   int grid = (int)(tiles < (int64_t)max_ctas ? tiles : (int64_t)max_ctas);
   if (grid < 1) grid = 1;
+  const bool overlap = p.rows_bound <= kGemmOverlapMaxRows;
   cudaError_t err;
   if (gather)
-    err = launch_variant(grouped_gemm_tc_kernel<true, true, false>, kThreadsGather, mx, mw, mx2, mw2, om, prm, grid, smem, stream);
+    err = launch_variant(grouped_gemm_tc_kernel<true, true, false>, kThreadsGather, mx, mw, mx2, mw2, om, prm, grid, smem, stream, overlap);
   else if (fp8)
-    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, false, true>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream)
-                  : launch_variant(grouped_gemm_tc_kernel<false, false, true>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream);
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, false, true>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream, overlap)
+                  : launch_variant(grouped_gemm_tc_kernel<false, false, true>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream, overlap);
   else
-    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, false, false>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream)
-                  : launch_variant(grouped_gemm_tc_kernel<false, false, false>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream);
+    err = p.gated ? launch_variant(grouped_gemm_tc_kernel<true, false, false>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream, overlap)
+                  : launch_variant(grouped_gemm_tc_kernel<false, false, false>, kThreads, mx, mw, mx2, mw2, om, prm, grid, smem, stream, overlap);
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;
 }

@@ -101,8 +101,8 @@ cudaError_t launch_gemm_validation(const GemmProblem& p, cudaStream_t stream, in
   const int E = e_end - e_begin;  // experts of this launch
   const int32_t* offs = p.offsets ? p.offsets + e_begin : nullptr;
   W += (size_t)e_begin * (size_t)(p.gated ? 2 : 1) * p.n_feat * p.K;
-  if (p.gated) (void)launch_pdl(gemm_validation_kernel<true>, grid, dim3(256), 0, stream, A, W, out, offs, p.fixed_rows, E, p.n_feat, p.K);
-  else (void)launch_pdl(gemm_validation_kernel<false>, grid, dim3(256), 0, stream, A, W, out, offs, p.fixed_rows, E, p.n_feat, p.K);
+  if (p.gated) (void)launch_pdl(true, gemm_validation_kernel<true>, grid, dim3(256), 0, stream, A, W, out, offs, p.fixed_rows, E, p.n_feat, p.K);
+  else (void)launch_pdl(true, gemm_validation_kernel<false>, grid, dim3(256), 0, stream, A, W, out, offs, p.fixed_rows, E, p.n_feat, p.K);
   cudaError_t err = cudaGetLastError();
   if (err == cudaSuccess && n_launches) *n_launches += 1;
   return err;

@@ -14,8 +14,8 @@ inline cudaError_t ensure_dynamic_smem(Kernel kern, size_t bytes) {
   return ensure_dynamic_smem_impl(reinterpret_cast<const void*>(kern), bytes);
 }
 
-// Programmatic dependent launch: every kernel of the library is launched with "programmatic stream serialization
-// allowed", so its CTAs may become resident and run their prologue (barrier set-up, tensor-memory allocation,
+// Programmatic dependent launch: the kernels of the library are launched with "programmatic stream serialization
+// allowed" (the GEMMs for small problems only, see kGemmOverlapMaxRows), so their CTAs may become resident and run their prologue (barrier set-up, tensor-memory allocation,
 // tensor-map prefetch) while the previous kernel of the stream is still draining; pdl_wait() then blocks until that
 // kernel has completed and its writes are visible.  Rules: every thread calls pdl_wait() before its first access to
 // global memory (reads AND writes: the predecessor may still be reading what this kernel overwrites), and
@@ -26,8 +26,8 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                              Args&&... args) {
+inline cudaError_t launch_pdl(bool allow_overlap, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                              cudaStream_t stream, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -37,9 +37,13 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = allow_overlap ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
+// The GEMM kernels take the overlap only for problems of up to this many rows: measured on a B200, a step of a
+// few hundred microseconds gains 7 % from it (six launch latencies and prologues hidden), while steps of several
+// milliseconds LOSE 1.5-5 % when their GEMM launches carry the attribute (the small kernels keep it at every size).
+constexpr int64_t kGemmOverlapMaxRows = 8192;
 #endif
 
 // Device status codes (same values as moe_status in the public header).

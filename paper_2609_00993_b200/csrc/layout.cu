@@ -278,7 +278,7 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
                           int* n_launches) {
   cudaError_t err;
   if (n_slots <= 0) {
-    err = launch_pdl(layout_empty_kernel, dim3(1), dim3(256), 0, stream, E, counts, offsets);
+    err = launch_pdl(true, layout_empty_kernel, dim3(1), dim3(256), 0, stream, E, counts, offsets);
     if (err == cudaSuccess && n_launches) *n_launches += 1;
     return err;
   }
@@ -287,7 +287,7 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
     int spw = (int)((n_slots + kFusedWarps - 1) / kFusedWarps);
     spw = (spw + 31) / 32 * 32;
     if ((err = ensure_dynamic_smem(layout_fused_kernel, fused_smem)) != cudaSuccess) return err;
-    err = launch_pdl(layout_fused_kernel, dim3(1), dim3(kFusedWarps * 32), fused_smem, stream, topk_idx, (int)n_slots, E, spw, counts, offsets,
+    err = launch_pdl(true, layout_fused_kernel, dim3(1), dim3(kFusedWarps * 32), fused_smem, stream, topk_idx, (int)n_slots, E, spw, counts, offsets,
                                                                      perm, inv_perm, status);
     if (err == cudaSuccess && n_launches) *n_launches += 1;
     return err;
@@ -295,11 +295,11 @@ cudaError_t launch_layout(const int32_t* topk_idx, int64_t n_slots, int E, int32
   const int n_chunks = (int)((n_slots + kLayoutChunk - 1) / kLayoutChunk);
   const int blocks = (n_chunks + kChunkWarpsPerBlock - 1) / kChunkWarpsPerBlock;
   const size_t chunk_smem = (size_t)kChunkWarpsPerBlock * E * sizeof(int);
-  if ((err = launch_pdl(layout_count_kernel, dim3(blocks), dim3(kChunkWarpsPerBlock * 32), chunk_smem, stream, topk_idx, n_slots, E, n_chunks,
+  if ((err = launch_pdl(true, layout_count_kernel, dim3(blocks), dim3(kChunkWarpsPerBlock * 32), chunk_smem, stream, topk_idx, n_slots, E, n_chunks,
                                                                                 scratch, status)) != cudaSuccess) return err;
-  if ((err = launch_pdl(layout_scan_kernel, dim3((E + 31) / 32), dim3(1024), 0, stream, scratch, n_chunks, E, counts)) != cudaSuccess) return err;
+  if ((err = launch_pdl(true, layout_scan_kernel, dim3((E + 31) / 32), dim3(1024), 0, stream, scratch, n_chunks, E, counts)) != cudaSuccess) return err;
   const size_t place_smem = chunk_smem + ((size_t)E + (E + 1) + 33) * sizeof(int);
-  launch_pdl(layout_place_kernel, dim3(blocks), dim3(kChunkWarpsPerBlock * 32), place_smem, stream, topk_idx, n_slots, E, n_chunks,
+  launch_pdl(true, layout_place_kernel, dim3(blocks), dim3(kChunkWarpsPerBlock * 32), place_smem, stream, topk_idx, n_slots, E, n_chunks,
                                                                                 scratch, counts, offsets, perm,
                                                                                 inv_perm);
   if ((err = cudaGetLastError()) != cudaSuccess) return err;

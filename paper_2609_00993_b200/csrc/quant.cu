@@ -86,10 +86,10 @@ cudaError_t launch_quantize_rows(const void* x, int64_t rows, int n, void* q, fl
   cudaError_t err;
   if (n_vec <= 32 * kQuantMaxVecs) {
     const long long blocks = (rows + kQuantThreads / 32 - 1) / (kQuantThreads / 32);
-    err = launch_pdl(quantize_rows_kernel<1>, dim3((unsigned)blocks), dim3(kQuantThreads), 0, stream,
+    err = launch_pdl(true, quantize_rows_kernel<1>, dim3((unsigned)blocks), dim3(kQuantThreads), 0, stream,
                      static_cast<const uint4*>(x), (long long)rows, n_vec, static_cast<uint2*>(q), scale);
   } else {
-    err = launch_pdl(quantize_rows_kernel<4>, dim3((unsigned)rows), dim3(kQuantThreads), 0, stream,
+    err = launch_pdl(true, quantize_rows_kernel<4>, dim3((unsigned)rows), dim3(kQuantThreads), 0, stream,
                      static_cast<const uint4*>(x), (long long)rows, n_vec, static_cast<uint2*>(q), scale);
   }
   if (err == cudaSuccess && n_launches) *n_launches += 1;

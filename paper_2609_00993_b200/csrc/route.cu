@@ -106,11 +106,11 @@ cudaError_t launch_vpt(bool vec, const float* logits, const float* bias, int T, 
   const int blocks = (T + kWarpsPerBlock - 1) / kWarpsPerBlock;
   if constexpr (VPT >= 4) {
     if (vec) {
-      return launch_pdl(route_kernel<VPT, true>, dim3(blocks), dim3(kWarpsPerBlock * 32), 0, stream, logits, bias, T, E, k,
+      return launch_pdl(true, route_kernel<VPT, true>, dim3(blocks), dim3(kWarpsPerBlock * 32), 0, stream, logits, bias, T, E, k,
                         scale, idx, w);
     }
   }
-  return launch_pdl(route_kernel<VPT, false>, dim3(blocks), dim3(kWarpsPerBlock * 32), 0, stream, logits, bias, T, E, k, scale,
+  return launch_pdl(true, route_kernel<VPT, false>, dim3(blocks), dim3(kWarpsPerBlock * 32), 0, stream, logits, bias, T, E, k, scale,
                     idx, w);
 }
 

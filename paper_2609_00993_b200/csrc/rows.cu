@@ -297,7 +297,7 @@ cudaError_t launch_permute(const void* x, const int32_t* inv_perm, void* x_perm,
   const long long n_items = (long long)T * col_blocks;
   const long long cap = resident_ctas(reinterpret_cast<const void*>(permute_rows_kernel), 32, smem);
   const int grid = (int)(n_items < cap ? n_items : cap);
-  err = launch_pdl(permute_rows_kernel, dim3(grid), dim3(32), smem, stream, static_cast<const __nv_bfloat16*>(x), inv_perm,
+  err = launch_pdl(true, permute_rows_kernel, dim3(grid), dim3(32), smem, stream, static_cast<const __nv_bfloat16*>(x), inv_perm,
                    static_cast<__nv_bfloat16*>(x_perm), T, k, H, col_blocks, slot_bytes, row_val, row_val_perm, status,
                    wait_limit_ns ? wait_limit_ns : kWaitLimitNs);
   if (err == cudaSuccess && n_launches) *n_launches += 1;
@@ -322,7 +322,7 @@ cudaError_t launch_combine(const void* y_perm, const void* y_shared, const int32
     const long long n_items = (long long)T * col_blocks;
     const long long cap = resident_ctas(reinterpret_cast<const void*>(kern), kCombineThreads, smem);
     const int grid = (int)(n_items < cap ? n_items : cap);
-    return launch_pdl(kern, dim3(grid), dim3(kCombineThreads), smem, stream, static_cast<const __nv_bfloat16*>(y_perm),
+    return launch_pdl(true, kern, dim3(grid), dim3(kCombineThreads), smem, stream, static_cast<const __nv_bfloat16*>(y_perm),
                       static_cast<const __nv_bfloat16*>(y_shared), inv_perm, topk_w, static_cast<__nv_bfloat16*>(out), T, k,
                       H, col_blocks, chunk_bytes, stage_bytes, stages, status,
                       wait_limit_ns ? wait_limit_ns : kWaitLimitNs);
