@@ -67,7 +67,7 @@ typedef enum {
 
 /* GEMM kernel variants.  AUTO: a DECODE context uses small-M; a PREFILL context chooses per step and pass from
  * the step's rows per expert R = T * top_k / n_experts (small-M up to R = 1024 for the gated pass, 384 for the
- * down pass, 256 with FP8 weights; large-M above) -- a function of T alone, so a step captured in a CUDA graph
+ * down pass; 256 and 128 with FP8 weights; large-M above) -- a function of T alone, so a step captured in a CUDA graph
  * replays the kernels it was captured with. */
 typedef enum {
   MOE_GEMM_AUTO = 0,

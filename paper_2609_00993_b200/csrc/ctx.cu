@@ -294,9 +294,9 @@ int gemm_ctas(const moe_ctx* ctx) {
 // from shared memory, whose bandwidth is what both kernels end up waiting for).  The gated pass (long K on the
 // V3 shape, SwiGLU in the epilogue) is ahead with small-M by 5-13 % up to ~512 rows per expert and level with
 // large-M around 1024; the down pass (short K, so the exposed epilogue of its tiles of more than 128 tokens
-// weighs more) and the FP8 passes (half the operand bytes per flop, so the issue cost of two MMAs per 16
-// K-elements shows) change over near 256-384 rows per expert.
-constexpr int64_t kSmallMRowsGated = 1024, kSmallMRowsDown = 384, kSmallMRowsFp8 = 256;
+// weighs more) changes over near 384 rows per expert, the FP8 passes (half the operand bytes per flop, so the issue
+// cost of two MMAs per 16 K-elements shows) at 256 (gated) and 128 (down).
+constexpr int64_t kSmallMRowsGated = 1024, kSmallMRowsDown = 384, kSmallMRowsFp8Gated = 256, kSmallMRowsFp8Down = 128;
 
 // AUTO: a DECODE context always streams; a PREFILL context chooses per launch from the rows per expert of the
 // problem (T * top_k rows over n_experts; T rows over one group for the shared expert by itself): the choice is
@@ -307,7 +307,8 @@ int gemm_variant_of(const moe_ctx* ctx, const moe::GemmProblem& p) {
   if (ctx->cfg.phase == MOE_PHASE_DECODE) return MOE_GEMM_SMALL_M;
   if (ctx->cfg.row_gather == 1) return MOE_GEMM_LARGE_M;  // only the large-M kernel gathers its rows itself
   if (ctx->preemptible) return MOE_GEMM_SMALL_M;          // only the small-M kernel can stop between tiles
-  const int64_t limit = p.fp8 ? kSmallMRowsFp8 : (p.gated ? kSmallMRowsGated : kSmallMRowsDown);
+  const int64_t limit = p.fp8 ? (p.gated ? kSmallMRowsFp8Gated : kSmallMRowsFp8Down)
+                              : (p.gated ? kSmallMRowsGated : kSmallMRowsDown);
   return p.rows_bound <= limit * p.E ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M;  // p.E = 1 for a dense problem
 }
 
