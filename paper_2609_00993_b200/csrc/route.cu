@@ -1,8 +1,10 @@
 // Stage a1: top-k routing over given router logits.  One warp per token; each lane keeps
-// ceil(E/32) selection keys in registers (128-bit loads when E is a multiple of 128), and k rounds of
-// a warp arg-max on (key descending, expert index ascending) pick the experts.  The arg-max is two integer
-// warp reductions (redux.sync): a max over an order-preserving integer image of the key, then a min over
-// the expert indices that hold it.  The routed weights are a max-subtracted softmax over the k selected
+// ceil(E/32) selection keys in registers (128-bit loads when E is a multiple of 128) as order-preserving integer
+// images.  Selection: k warp maxima over the lanes' own maxima give a threshold that at least k keys reach; the few
+// keys that reach it are compacted into a per-warp list and each is ranked exactly against the others (key
+// descending, expert index ascending).  Only when ties put more than 32 keys at the threshold do k rounds of a
+// warp arg-max over all keys run instead (redux.sync: a max over the key images, then a min over the expert
+// indices that hold it).  The routed weights are a max-subtracted softmax over the k selected
 // unbiased logits, summed in selection order.
 #include "kernels.h"
 
@@ -63,27 +65,83 @@ route_kernel(const float* __restrict__ logits, const float* __restrict__ bias, i
     }
   }
 
-  unsigned taken = 0u;  // bit i: this lane's i-th key is already selected
-  int my_e = 0;         // lane j (< k) ends up holding the j-th selected expert
+  // ---- selection.  Fast path: the k-th largest of the 32 lane maxima is a threshold that at least k keys reach
+  // (the maxima of k different lanes); the keys that reach it -- typically k to 2k of them -- are the only
+  // candidates, and each is ranked exactly against the others (key descending, expert index ascending).  When
+  // ties put more than 32 keys at or above the threshold the k-round warp arg-max below takes over.
+  int my_e = 0;  // lane j (< k) ends up holding the j-th selected expert
+  __shared__ unsigned s_key[kWarpsPerBlock][32];
+  __shared__ int s_idx[kWarpsPerBlock][32];
+  __shared__ int s_sel[kWarpsPerBlock][32];
+  const int wib = threadIdx.x >> 5;
+  unsigned lmax = 0u;  // 0 is below the image of every float
+#pragma unroll
+  for (int i = 0; i < VPT; ++i)
+    if (expert_of(i) < E) lmax = max(lmax, key[i]);
+  unsigned tau = 0u, cur = lmax;
   for (int j = 0; j < k; ++j) {
-    unsigned bv = 0u;
-    int be = 0x7fffffff;
-    bool has = false;
+    tau = __reduce_max_sync(0xffffffffu, cur);
+    const unsigned holders = __ballot_sync(0xffffffffu, cur == tau);
+    if (lane == __ffs(holders) - 1) cur = 0u;  // remove one holder per round
+  }
+  unsigned mine = 0u;  // bit i: this lane's i-th key is a candidate
+  int n_cand = 0;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const bool c = expert_of(i) < E && key[i] >= tau;
+    if (c) mine |= 1u << i;
+    n_cand += __popc(__ballot_sync(0xffffffffu, c));
+  }
+  if (n_cand <= 32) {
+    // compact the candidates into the warp's list (any order), then rank each against all
+    int base = 0;
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
-      const int e = expert_of(i);
-      const bool avail = (e < E) && !((taken >> i) & 1u);
-      if (avail && (!has || key[i] > bv)) {
-        bv = key[i]; be = e; has = true;
+      const bool c = (mine >> i) & 1u;
+      const unsigned b = __ballot_sync(0xffffffffu, c);
+      if (c) {
+        const int pos = base + __popc(b & ((1u << lane) - 1u));
+        s_key[wib][pos] = key[i];
+        s_idx[wib][pos] = expert_of(i);
       }
+      base += __popc(b);
     }
-    // warp arg-max on (key descending, expert index ascending): largest key, then the lowest index holding it
-    const unsigned top = __reduce_max_sync(0xffffffffu, has ? bv : 0u);
-    const int win = (int)__reduce_min_sync(0xffffffffu, (unsigned)((has && bv == top) ? be : 0x7fffffff));
-    const int owner = VEC ? ((win & 127) >> 2) : (win & 31);
-    const int slot = VEC ? (4 * (win >> 7) + (win & 3)) : (win >> 5);
-    if (lane == owner) taken |= (1u << slot);
-    if (lane == j) my_e = win;
+    __syncwarp();
+    if (lane < n_cand) {
+      const unsigned kp = s_key[wib][lane];
+      const int ep = s_idx[wib][lane];
+      int rank = 0;
+      for (int q = 0; q < n_cand; ++q) {
+        const unsigned kq = s_key[wib][q];
+        const int eq = s_idx[wib][q];
+        rank += (kq > kp || (kq == kp && eq < ep)) ? 1 : 0;
+      }
+      if (rank < k) s_sel[wib][rank] = ep;
+    }
+    __syncwarp();
+    if (lane < k) my_e = s_sel[wib][lane];
+  } else {
+    unsigned taken = 0u;  // bit i: this lane's i-th key is already selected
+    for (int j = 0; j < k; ++j) {
+      unsigned bv = 0u;
+      int be = 0x7fffffff;
+      bool has = false;
+#pragma unroll
+      for (int i = 0; i < VPT; ++i) {
+        const int e = expert_of(i);
+        const bool avail = (e < E) && !((taken >> i) & 1u);
+        if (avail && (!has || key[i] > bv)) {
+          bv = key[i]; be = e; has = true;
+        }
+      }
+      // warp arg-max on (key descending, expert index ascending): largest key, then the lowest index holding it
+      const unsigned top = __reduce_max_sync(0xffffffffu, has ? bv : 0u);
+      const int win = (int)__reduce_min_sync(0xffffffffu, (unsigned)((has && bv == top) ? be : 0x7fffffff));
+      const int owner = VEC ? ((win & 127) >> 2) : (win & 31);
+      const int slot = VEC ? (4 * (win >> 7) + (win & 3)) : (win >> 5);
+      if (lane == owner) taken |= (1u << slot);
+      if (lane == j) my_e = win;
+    }
   }
 
   const bool active = lane < k;
