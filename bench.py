@@ -516,7 +516,7 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm, peaks, w):
     def preemptive_run(n_iter, think_ms, seed=0):
         ts = B.Turnstile(1)
         ctx_p.moe_ctx_set_preemption(True)
-        state = {"epoch": -1, "b": 0, "err": None}
+        state = {"epoch": -1, "b": 0, "err": None, "d_waiting": False, "dispatch_boundaries": 0}
 
         def on_yield(i, n):
             st_ = ts.publish(state["epoch"], state["b"], 5000)
@@ -538,6 +538,7 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm, peaks, w):
                 if stop.is_set():
                     break
                 t0 = time.perf_counter()                  # the D batch is ready
+                state["d_waiting"] = True
                 ctx_p.moe_ctx_request_yield(True)
                 st_, _active = ts.d_enter(5000)
                 if st_ != B.MOE_OK:
@@ -551,6 +552,7 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm, peaks, w):
                 lat_wall.append(1e6 * (time.perf_counter() - t0))
                 lat_dev.append(1e3 * e0.elapsed_time(e1))
                 ctx_p.moe_ctx_request_yield(False)
+                state["d_waiting"] = False
                 ts.d_release()
                 j += 1
 
@@ -562,8 +564,18 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm, peaks, w):
         for i in range(n_iter):
             state["epoch"], state["b"] = i, 0
             ts.begin_epoch(i, False)
+            a = aps[i % iters]
             with torch.cuda.stream(sp):
-                p_step(i)
+                # the dispatch in its two halves: after the notification (counts, scan, permutation) comes the first
+                # safe point of the step, before any row has moved; a waiting D batch is admitted there
+                ctx_p.moe_route(a["logits"], a["bias"], bp["topk_idx"], bp["topk_w"])
+                ctx_p.moe_dispatch_notify(bp["topk_idx"], bp["counts"], bp["offsets"], bp["perm"], bp["inv_perm"])
+                if state["d_waiting"]:
+                    state["dispatch_boundaries"] += 1
+                    on_yield(0, 0)
+                ctx_p.moe_dispatch_move(a["x"])
+                ctx_p.moe_grouped_ffn(w["w_gate_up"], w["w_down"], a["x"], w["ws_gate_up"], w["ws_down"])
+                ctx_p.moe_combine(bp["topk_w"], bp["inv_perm"], op)
             sp.synchronize()
             ts.task_done(i)
             if state["err"]:
@@ -578,6 +590,7 @@ def decode_under_prefill(torch, B, wl, dev, iters, warm, peaks, w):
         if state["err"] or not lat_wall:
             return {"think_ms": think_ms, "error": state["err"] or "no D step ran"}
         r = {"think_ms": think_ms, "d_steps": len(lat_wall), "yields": ctx_p.moe_ctx_yield_count() - y0,
+             "admitted_between_notification_and_row_movement": state["dispatch_boundaries"],
              "ready_to_done_us": _stats(lat_wall), "device_us": _stats(lat_dev),
              "prefill_tokens_per_s": wl.C4_P.T * n_iter / p_s}
         r["p99_over_alone"] = r["ready_to_done_us"]["p99"] / res["alone_host_wall_us"]["p99"]
