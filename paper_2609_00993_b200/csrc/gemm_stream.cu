@@ -490,6 +490,77 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       // values for them (features f, f+1 of one token are one 4-byte store); the odd lane does the same for
       // the odd tokens.  n_feat is a multiple of 8, so a pair is inside the row or outside it as a whole.
       const int f_pair = (GATED ? f_a : 0) & ~1;
+      auto release_acc = [&]() {  // hand the accumulator half (or both) back to the MMA issuer
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (big) {
+            mbar_arrive(bar_tempty);
+            mbar_arrive(bar_tempty + 8u);
+          } else {
+            mbar_arrive(bar_tempty + 8u * h);
+          }
+        }
+      };
+      if (GATED && kEpilogueWarps == 8) {
+        // Two phases, so that the accumulator goes back to the MMA issuer as early as possible (a tile of more than
+        // 128 tokens holds all of TMEM, and the issuer waits for it): first every chunk is loaded (the next chunk's
+        // loads in flight meanwhile), put through SwiGLU and packed to bf16 in registers -- a warp has at most 8
+        // chunks of 16 tokens; then the accumulator is released; only then come the lane exchanges and the stores.
+        uint32_t pk[8][8];  // pk[m][i]: this lane's feature for tokens c + 2i (low half) and c + 2i + 1 (high half)
+        uint32_t na[16], nb[16];
+        if (c_first < t.rows) {
+          tmem_ld16(d_a + (uint32_t)c_first, na);
+          tmem_ld16(d_b + (uint32_t)c_first, nb);
+        }
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          const int c = c_first + m * c_step;
+          if (c < t.rows) {
+            float g[16], u[16];
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              g[i] = __uint_as_float(na[i]);
+              u[i] = __uint_as_float(nb[i]);
+            }
+            if (c + c_step < t.rows) {
+              tmem_ld16(d_a + (uint32_t)(c + c_step), na);
+              tmem_ld16(d_b + (uint32_t)(c + c_step), nb);
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              if (FP8) {
+                const float rs = (c + i < t.rows) ? __ldg(rsp + c + i) : 0.f;
+                g[i] *= rs * ws_a;
+                u[i] *= rs * ws_b;
+              }
+              g[i] = silu_mul(g[i], u[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pk[m][i] = pack_bf16(g[2 * i], g[2 * i + 1]);
+          }
+        }
+        release_acc();
+#pragma unroll
+        for (int m = 0; m < 8; ++m) {
+          const int c = c_first + m * c_step;
+          if (c < t.rows) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const uint32_t mine = pk[m][i];
+              const uint32_t nbr = __shfl_xor_sync(0xffffffffu, mine, 1);
+              // even lane (even feature f): token c+2i, features (f, f+1) = (own low, neighbour's low);
+              // odd lane: token c+2i+1, features (f-1, f) = (neighbour's high, own high)
+              const uint32_t pa = even ? __byte_perm(mine, nbr, 0x5410) : __byte_perm(nbr, mine, 0x7632);
+              const int tok = c + 2 * i + (even ? 0 : 1);
+              if (tok < t.rows && f_pair < n_feat)
+                *reinterpret_cast<uint32_t*>(out + (size_t)(t.row0 + tok) * n_feat + f_pair) = pa;
+            }
+          }
+        }
+        continue;
+      }
       // the loads of the next 16-token chunk are in flight while this one is converted and stored
       uint32_t na[16], nb[16];
       if (c_first < t.rows) {
@@ -543,17 +614,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
           }
         }
       }
-      // hand the accumulator half (or both) back to the MMA issuer
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        if (big) {
-          mbar_arrive(bar_tempty);
-          mbar_arrive(bar_tempty + 8u);
-        } else {
-          mbar_arrive(bar_tempty + 8u * h);
-        }
-      }
+      release_acc();
     }
     if (!ok && lane == 0) {
       *abort_flag = 1;
