@@ -8,10 +8,11 @@
 //              gated: gate rows + the matching up rows) and exactly N token rows, fetched as a binary
 //              decomposition of N into TMA boxes of 256/128/64/32/16 rows.  What bounds this regime is the
 //              bytes an SM ingests, so nothing is fetched that is not multiplied.
-//   ring       k-blocks live in a byte ring of 2 KB slots with FIFO allocation (a k-block takes 16 + N/16 slots),
-//              so a tile of few tokens keeps more k-blocks in flight than a tile of many; up to 8 k-blocks in
-//              flight, each with a full/empty mbarrier pair.  Producer and MMA issuer derive the same slot
-//              positions from the same tile sequence.
+//   ring       k-blocks live in a byte ring of 2 KB slots with FIFO allocation (a k-block takes 16 slots for its
+//              weights and N/16 for its token rows, two pieces that need not be adjacent), so a tile of few
+//              tokens keeps more k-blocks in flight than a tile of many; up to 8 k-blocks in flight, each with
+//              a full/empty mbarrier pair.  Producer and MMA issuer derive the same slot positions from the
+//              same tile sequence.
 //   TMEM       512 columns = two halves.  A tile of N <= 128 takes one half (its two accumulators side by side)
 //              and alternates halves, so its epilogue overlaps the next tile's MMAs; a tile of N > 128 takes both.
 //   epilogue   lane = weight row (output feature), column = token: tcgen05.ld -> (scale) -> SwiGLU -> bf16;
@@ -294,36 +295,47 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
         }
         const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
         const uint32_t n = (uint32_t)((t.rows + 15) & ~15);
-        const uint32_t s = (uint32_t)kWSlots + (n >> 4);
         const int w_row0 = t.ft * kFeatPerTile;
         const CUtensorMap* mw = t.dense ? &map_w2 : &map_w;
         const CUtensorMap* mx = (t.dense ? xmaps.x2 : xmaps.x) + ((n >> 4) - 1u);  // the box of exactly n rows
         const int w_e = t.dense ? 0 : p.e_base + t.e;
         const int num_kb = t.dense ? num_kb2 : num_kb1;
         for (int kb = 0, k0 = 0; kb < num_kb && ok; ++kb, k0 += kbk) {
-          const bool wrap = head + s > R;  // a k-block never wraps: it skips what is left at the ring's end
-          const uint32_t pad = wrap ? R - head : 0u;
-          while (free_slots < s + pad || kb_idx - oldest >= (uint32_t)kNB) {
-            PROF_T0();
-            const bool got = mbar_wait(bar_empty + 8u * (oldest % kNB), (oldest / kNB) & 1u, abort_flag, limit);
-            PROF_ADD(prof_wait_empty);
-            if (!got) { ok = false; break; }
-            free_slots += (uint32_t)sizes[oldest % kNB];
-            ++oldest;
-          }
-          if (!ok) break;
-          if (wrap) head = 0;
-          sizes[kb_idx % kNB] = (int)(s + pad);
-          free_slots -= s + pad;
+          // The ring is allocated per operand: the weight boxes and the token rows of a k-block are two contiguous
+          // pieces that need not be adjacent, so the weights of the next k-block go out as soon as 16 slots are
+          // free.  A piece never wraps: it skips what is left at the ring's end.
+          const uint32_t nx = n >> 4;
+          const bool wrap_w = head + (uint32_t)kWSlots > R;
+          const uint32_t pad_w = wrap_w ? R - head : 0u;
+          const uint32_t head_w = wrap_w ? 0u : head;
+          const bool wrap_x = head_w + (uint32_t)kWSlots + nx > R;
+          const uint32_t pad_x = wrap_x ? R - (head_w + (uint32_t)kWSlots) : 0u;
+          const uint32_t head_x = wrap_x ? 0u : head_w + (uint32_t)kWSlots;
+          auto reclaim = [&](uint32_t need, bool count_limit) {
+            while (free_slots < need || (count_limit && kb_idx - oldest >= (uint32_t)kNB)) {
+              PROF_T0();
+              const bool got = mbar_wait(bar_empty + 8u * (oldest % kNB), (oldest / kNB) & 1u, abort_flag, limit);
+              PROF_ADD(prof_wait_empty);
+              if (!got) return false;
+              free_slots += (uint32_t)sizes[oldest % kNB];
+              ++oldest;
+            }
+            return true;
+          };
+          if (!reclaim((uint32_t)kWSlots + pad_w, true)) { ok = false; break; }
+          free_slots -= (uint32_t)kWSlots + pad_w;
           const uint32_t full = bar_full + 8u * (kb_idx % kNB);
-          const uint32_t st = base_addr + head * (uint32_t)kSlotBytes;
           mbar_expect_tx(full, 2u * kWBoxBytes + n * 128u);
           // one copy per operand: both weight boxes (gated: the map's third dimension steps from the gate rows
           // to the up rows; down pass: 256 consecutive rows), then the n token rows
-          if (GATED) tma_load_4d(st, mw, full, k0, w_row0, 0, w_e);
-          else tma_load_3d(st, mw, full, k0, w_row0, w_e);
-          tma_load_2d(st + 2 * kWBoxBytes, mx, full, k0, t.row0);
-          head += s;
+          const uint32_t st_w = base_addr + head_w * (uint32_t)kSlotBytes;
+          if (GATED) tma_load_4d(st_w, mw, full, k0, w_row0, 0, w_e);
+          else tma_load_3d(st_w, mw, full, k0, w_row0, w_e);
+          if (!reclaim(nx + pad_x, false)) { ok = false; break; }
+          free_slots -= nx + pad_x;
+          sizes[kb_idx % kNB] = (int)((uint32_t)kWSlots + pad_w + nx + pad_x);
+          tma_load_2d(base_addr + head_x * (uint32_t)kSlotBytes, mx, full, k0, t.row0);
+          head = head_x + nx;
           ++kb_idx;
         }
       }
@@ -355,7 +367,6 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
         if (tile >= total_tiles) break;
         const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
         const uint32_t n = (uint32_t)((t.rows + 15) & ~15);
-        const uint32_t s = (uint32_t)kWSlots + (n >> 4);
         const bool big = n > 128u;
         uint32_t d_a, d_b;
         PROF_T0();
@@ -380,9 +391,12 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
         const uint32_t idesc = FP8 ? umma_idesc_e4m3(128, n) : umma_idesc(128, n);
         const int num_kb = t.dense ? num_kb2 : num_kb1;
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (head + s > R) head = 0;
-          const uint32_t pos = head;
-          head += s;
+          if (head + (uint32_t)kWSlots > R) head = 0;  // the producer's allocation, step for step
+          const uint32_t pos_w = head;
+          head += (uint32_t)kWSlots;
+          if (head + (n >> 4) > R) head = 0;
+          const uint32_t pos_x = head;
+          head += n >> 4;
           {
             PROF_T0();
             // the wait for a tile's first k-block also ends when the producer has decided not to start the tile
@@ -394,7 +408,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
             if (got != 0) { ok = false; break; }
           }
           tc_fence_after();
-          const uint32_t lo_w0 = lo_base + pos * lo_slot, lo_w1 = lo_w0 + lo_box, lo_x = lo_w0 + 2 * lo_box;
+          const uint32_t lo_w0 = lo_base + pos_w * lo_slot, lo_w1 = lo_w0 + lo_box, lo_x = lo_base + pos_x * lo_slot;
 #pragma unroll
           for (int kk = 0; kk < kBlockK / kUmmaK; ++kk) {
             const uint32_t adv = (uint32_t)((kk * kUmmaK * 2) >> 4);  // +32 bytes per MMA, in 16-byte units
