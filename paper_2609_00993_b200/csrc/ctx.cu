@@ -324,6 +324,9 @@ cudaError_t run_gemm(moe_ctx* ctx, moe::GemmProblem p, const moe::GemmDenseGroup
   const int variant = gemm_variant_of(ctx, p);
   p.wait_limit_ns = ctx->wait_limit_ns;
   p.debug_stall = ctx->debug_stall;
+  // Every GEMM launch comes after the step's row movement (or after another GEMM launch or a quantisation of the
+  // same step), which in turn waited for the layout kernels: the offsets are older than the previous kernel.
+  p.offsets_settled = true;
   if (variant == MOE_GEMM_VALIDATION) {
     cudaError_t e = moe::launch_gemm_validation(p, ctx->stream, n);
     if (e == cudaSuccess && dense != nullptr) {

@@ -84,16 +84,23 @@ struct StreamParams {
   const int* yield_req;
   int* progress;
   int* stopped;
+  // The expert offsets were final before the PREVIOUS kernel of the stream started (and the weights always are):
+  // the tile list is built and weight boxes are fetched before this kernel waits for that previous kernel, which
+  // only the token rows (and the FP8 row scales) depend on.
+  int32_t early_setup;
 };
 
 #ifdef MOE_STREAM_PROF
 // Debug build only: per-CTA role timings of the last launches (8 words per CTA, accumulated).
 __device__ unsigned long long g_stream_prof[8 * 256];
+__device__ unsigned long long g_stream_ts[8 * 256];  // global-timer stamps of the last launch, 8 per CTA
 #define PROF_T0() const long long prof_t0 = clock64()
 #define PROF_ADD(var) var += clock64() - prof_t0
+#define PROF_STAMP(slot) g_stream_ts[8 * blockIdx.x + (slot)] = global_ns()
 #else
 #define PROF_T0()
 #define PROF_ADD(var)
+#define PROF_STAMP(slot)
 #endif
 
 struct StreamMaps {
@@ -198,6 +205,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int unit = (int)blockIdx.x, n_units = (int)gridDim.x;
+  if (threadIdx.x == 0) PROF_STAMP(0);
   constexpr int kFeatPerTile = GATED ? 128 : 256;
   const int n_ft = (p.n_feat + kFeatPerTile - 1) / kFeatPerTile;
   const int num_kb1 = (p.K + kbk - 1) / kbk, num_kb2 = (p.K2 + kbk - 1) / kbk;
@@ -222,8 +230,14 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == kMmaWarp) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-  pdl_wait();
-  pdl_launch_dependents();
+  // With early set-up only the threads that touch what the previous kernel wrote wait for it: the producer before
+  // its first token-row copy, the epilogue warps before their first store.  Dependents are released only by
+  // threads that have waited, so a later kernel never starts before the kernel two places back has completed.
+  if (!p.early_setup) {
+    pdl_wait();
+    pdl_launch_dependents();
+  }
+  if (threadIdx.x == 0) PROF_STAMP(1);
   for (int e = threadIdx.x; e < p.E; e += kThreads) {
     const int b = p.offsets ? p.offsets[e] : 0;
     int c = p.offsets ? p.offsets[e + 1] - b : p.fixed_rows;
@@ -266,6 +280,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) PROF_STAMP(2);
   const int total_tiles = dense_tiles + prefix[p.E] * n_ft;
   const uint32_t R = (uint32_t)p.ring_slots;
   const int w_first = p.progress ? p.progress[unit] : 0;  // a resumed pass continues where this CTA stopped
@@ -275,6 +290,20 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
     if (lane == 0 && !p.inject_producer_stall) {
       uint32_t head = 0, free_slots = R, kb_idx = 0, oldest = 0;
       bool ok = true;
+      // Early set-up: until this thread has waited for the previous kernel, token-row copies are put off (their
+      // ring space is allocated and their bytes announced) while the weight boxes of up to kNB k-blocks go out.
+      bool dep_waited = !p.early_setup;
+      int n_def = 0;
+      uint32_t def_dst[kNB], def_full[kNB];
+      int def_k0[kNB], def_row0[kNB];
+      const CUtensorMap* def_map[kNB];
+      auto dep_wait_and_flush = [&]() {
+        pdl_wait();
+        pdl_launch_dependents();
+        dep_waited = true;
+        for (int i = 0; i < n_def; ++i) tma_load_2d(def_dst[i], def_map[i], def_full[i], def_k0[i], def_row0[i]);
+        n_def = 0;
+      };
       [[maybe_unused]] long long prof_wait_empty = 0, prof_tiles = 0;
       [[maybe_unused]] const long long prof_start = clock64();
       int yield_seen = 0;
@@ -312,6 +341,9 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
           const uint32_t pad_x = wrap_x ? R - (head_w + (uint32_t)kWSlots) : 0u;
           const uint32_t head_x = wrap_x ? 0u : head_w + (uint32_t)kWSlots;
           auto reclaim = [&](uint32_t need, bool count_limit) {
+            // nothing is consumed before the token rows are in: wait for the previous kernel before blocking
+            if (!dep_waited && (free_slots < need || (count_limit && kb_idx - oldest >= (uint32_t)kNB)))
+              dep_wait_and_flush();
             while (free_slots < need || (count_limit && kb_idx - oldest >= (uint32_t)kNB)) {
               PROF_T0();
               const bool got = mbar_wait(bar_empty + 8u * (oldest % kNB), (oldest / kNB) & 1u, abort_flag, limit);
@@ -334,11 +366,21 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
           if (!reclaim(nx + pad_x, false)) { ok = false; break; }
           free_slots -= nx + pad_x;
           sizes[kb_idx % kNB] = (int)((uint32_t)kWSlots + pad_w + nx + pad_x);
-          tma_load_2d(base_addr + head_x * (uint32_t)kSlotBytes, mx, full, k0, t.row0);
+          if (dep_waited) {
+            tma_load_2d(base_addr + head_x * (uint32_t)kSlotBytes, mx, full, k0, t.row0);
+          } else {
+            def_dst[n_def] = base_addr + head_x * (uint32_t)kSlotBytes;
+            def_full[n_def] = full;
+            def_map[n_def] = mx;
+            def_k0[n_def] = k0;
+            def_row0[n_def] = t.row0;
+            ++n_def;
+          }
           head = head_x + nx;
           ++kb_idx;
         }
       }
+      if (!dep_waited) dep_wait_and_flush();
       if (!ok) {
         *abort_flag = 1;
         atomicCAS(p.status, kStOk, kStTimeout);
@@ -407,6 +449,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
             if (got == 2) { stopped = true; break; }
             if (got != 0) { ok = false; break; }
           }
+          if (kb_idx == 0) PROF_STAMP(3);
           tc_fence_after();
           const uint32_t lo_w0 = lo_base + pos_w * lo_slot, lo_w1 = lo_w0 + lo_box, lo_x = lo_base + pos_x * lo_slot;
 #pragma unroll
@@ -438,6 +481,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
         *abort_flag = 1;
         atomicCAS(p.status, kStOk, kStTimeout);
       }
+      PROF_STAMP(4);
 #ifdef MOE_STREAM_PROF
       if (warp == kMmaWarp)
       atomicAdd(&g_stream_prof[8 * unit + 2], (unsigned long long)(clock64() - prof_start));
@@ -452,6 +496,10 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   } else {
     // ================================================================= epilogue (warps 0-3)
     // lane = weight row (output feature) of each box, TMEM column = token
+    if (p.early_setup) {
+      pdl_wait();
+      pdl_launch_dependents();
+    }
     uint32_t use0 = 0, use1 = 0, next_half = 0;
     bool ok = true;
     const int lg = warp & 3;                         // TMEM lane group of this warp: lanes 32 lg .. 32 lg + 31
@@ -637,8 +685,10 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   }
 
   // ---- teardown
+  if (threadIdx.x == 0) PROF_STAMP(5);
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) PROF_STAMP(6);
   if (p.progress != nullptr && threadIdx.x == 0) {
     const int sw = *stop_w;
     if (sw != 0x7fffffff) {  // stopped on request: the next launch of this pass resumes at wave sw
@@ -745,6 +795,7 @@ cudaError_t launch_gemm_stream(const GemmProblem& p, const GemmDenseGroup* dense
   prm.row_scale2 = dense ? dense->row_scale : nullptr;
   prm.w_scale2 = dense ? dense->w_scale : nullptr;
   const bool preemptible = p.yield_req != nullptr && p.progress != nullptr && p.stopped != nullptr;
+  prm.early_setup = (p.offsets_settled && !preemptible) ? 1 : 0;  // a resumed pass reads its progress words first
   prm.yield_req = preemptible ? p.yield_req : nullptr;
   prm.progress = preemptible ? p.progress : nullptr;
   prm.stopped = preemptible ? p.stopped : nullptr;
@@ -778,6 +829,9 @@ cudaError_t launch_gemm_stream(const GemmProblem& p, const GemmDenseGroup* dense
 
 #ifdef MOE_STREAM_PROF
 }  // namespace moe
+extern "C" int moe_debug_stream_ts(unsigned long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, moe::g_stream_ts, sizeof(unsigned long long) * 8 * 256);
+}
 extern "C" int moe_debug_stream_prof(unsigned long long* host, int clear) {
   cudaError_t e = cudaMemcpyFromSymbol(host, moe::g_stream_prof, sizeof(unsigned long long) * 8 * 256);
   if (e == cudaSuccess && clear) {

@@ -43,7 +43,10 @@ inline cudaError_t launch_pdl(bool allow_overlap, void (*kern)(KArgs...), dim3 g
 // The GEMM kernels take the overlap only for problems of up to this many rows: measured on a B200, a step of a
 // few hundred microseconds gains 7 % from it (six launch latencies and prologues hidden), while steps of several
 // milliseconds LOSE 1.5-5 % when their GEMM launches carry the attribute (the small kernels keep it at every size).
-constexpr int64_t kGemmOverlapMaxRows = 8192;
+#ifndef MOE_GEMM_OVERLAP_MAX_ROWS
+#define MOE_GEMM_OVERLAP_MAX_ROWS 8192
+#endif
+constexpr int64_t kGemmOverlapMaxRows = MOE_GEMM_OVERLAP_MAX_ROWS;
 #endif
 
 // Device status codes (same values as moe_status in the public header).
@@ -118,6 +121,9 @@ struct GemmProblem {
   const int* yield_req = nullptr;
   int* progress = nullptr;
   int* stopped = nullptr;
+  // Small-M kernel: `offsets` was final before the previous kernel of the stream started, so the kernel may read it
+  // (and fetch weights) before it waits for that kernel; only the rows of A (and the FP8 row scales) wait.
+  bool offsets_settled = false;
 };
 
 // A dense group (the shared expert) that rides in the same launch as a grouped problem: its tiles are added
