@@ -327,6 +327,7 @@ cudaError_t run_gemm(moe_ctx* ctx, moe::GemmProblem p, const moe::GemmDenseGroup
   // Every GEMM launch comes after the step's row movement (or after another GEMM launch or a quantisation of the
   // same step), which in turn waited for the layout kernels: the offsets are older than the previous kernel.
   p.offsets_settled = true;
+  p.max_group_rows = T;
   if (variant == MOE_GEMM_VALIDATION) {
     cudaError_t e = moe::launch_gemm_validation(p, ctx->stream, n);
     if (e == cudaSuccess && dense != nullptr) {

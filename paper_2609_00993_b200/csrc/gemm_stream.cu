@@ -26,6 +26,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "kernels.h"
 #include "tc_common.cuh"
 
@@ -88,6 +90,7 @@ struct StreamParams {
   // the tile list is built and weight boxes are fetched before this kernel waits for that previous kernel, which
   // only the token rows (and the FP8 row scales) depend on.
   int32_t early_setup;
+  int32_t sort_tiles;  // 0: every group has at most one tile of the smallest size, so their order does not matter
 };
 
 #ifdef MOE_STREAM_PROF
@@ -248,7 +251,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   __syncthreads();
   for (int e = threadIdx.x; e < p.E; e += kThreads) {
     int rank = e;  // more than kSortMaxExperts experts: the natural order
-    if (p.E <= kSortMaxExperts) {
+    if (p.sort_tiles && p.E <= kSortMaxExperts) {
       const int c = cnts[e];
       rank = 0;
       for (int j = 0; j < p.E; ++j) {
@@ -795,6 +798,7 @@ cudaError_t launch_gemm_stream(const GemmProblem& p, const GemmDenseGroup* dense
   prm.row_scale2 = dense ? dense->row_scale : nullptr;
   prm.w_scale2 = dense ? dense->w_scale : nullptr;
   const bool preemptible = p.yield_req != nullptr && p.progress != nullptr && p.stopped != nullptr;
+  prm.sort_tiles = (p.max_group_rows > 0 && p.max_group_rows <= 16) ? 0 : 1;
   prm.early_setup = (p.offsets_settled && !preemptible) ? 1 : 0;  // a resumed pass reads its progress words first
   prm.yield_req = preemptible ? p.yield_req : nullptr;
   prm.progress = preemptible ? p.progress : nullptr;
@@ -805,6 +809,12 @@ cudaError_t launch_gemm_stream(const GemmProblem& p, const GemmDenseGroup* dense
   const int slots = (int)((kSmemBudget - 1024 - (int)tail) / kSlotBytes);
   if (slots < 2 * (kWSlots + kMaxTileRows / 16)) return cudaErrorNotSupported;
   prm.ring_slots = slots;
+#ifdef MOE_STREAM_PROF
+  if (const char* rs = getenv("MOE_STREAM_RING_SLOTS")) {  // debug build only: a smaller ring, to see what in-flight bytes buy
+    const int v = atoi(rs);
+    if (v >= 2 * (kWSlots + kMaxTileRows / 16) && v < slots) prm.ring_slots = v;
+  }
+#endif
   const size_t smem = 1024 + (size_t)slots * kSlotBytes + tail;
 
   const int feat_per_tile = p.gated ? 128 : 256;

@@ -124,6 +124,9 @@ struct GemmProblem {
   // Small-M kernel: `offsets` was final before the previous kernel of the stream started, so the kernel may read it
   // (and fetch weights) before it waits for that kernel; only the rows of A (and the FP8 row scales) wait.
   bool offsets_settled = false;
+  // Upper bound on the rows of any one group (a token reaches an expert at most once, so T), or 0 if unknown.  With
+  // at most 16, every non-empty group is one tile of the same cost and the small-M kernel skips ordering them.
+  int32_t max_group_rows = 0;
 };
 
 // A dense group (the shared expert) that rides in the same launch as a grouped problem: its tiles are added
