@@ -18,7 +18,7 @@ constexpr int kWarpsPerBlock = 8;
 // which keeps the IEEE tie between the two zeros.
 __device__ __forceinline__ unsigned ordered_bits(float v) {
   const unsigned u = __float_as_uint(v);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return u ^ ((unsigned)((int)u >> 31) | 0x80000000u);  // negative: all bits flipped; else the sign bit set
 }
 
 // VPT: keys per lane (power of two >= ceil(E/32)).  VEC: lanes own runs of 4 consecutive experts.
@@ -70,8 +70,7 @@ route_kernel(const float* __restrict__ logits, const float* __restrict__ bias, i
   // candidates, and each is ranked exactly against the others (key descending, expert index ascending).  When
   // ties put more than 32 keys at or above the threshold the k-round warp arg-max below takes over.
   int my_e = 0;  // lane j (< k) ends up holding the j-th selected expert
-  __shared__ unsigned s_key[kWarpsPerBlock][32];
-  __shared__ int s_idx[kWarpsPerBlock][32];
+  __shared__ unsigned long long s_cand[kWarpsPerBlock][32];
   __shared__ int s_sel[kWarpsPerBlock][32];
   const int wib = threadIdx.x >> 5;
   unsigned lmax = 0u;  // 0 is below the image of every float
@@ -84,39 +83,28 @@ route_kernel(const float* __restrict__ logits, const float* __restrict__ bias, i
     const unsigned holders = __ballot_sync(0xffffffffu, cur == tau);
     if (lane == __ffs(holders) - 1) cur = 0u;  // remove one holder per round
   }
-  unsigned mine = 0u;  // bit i: this lane's i-th key is a candidate
+  // One pass compacts the candidates into the warp's list (any order) as (key image << 32 | ~expert index) -- a
+  // larger entry comes earlier in (key descending, expert index ascending) -- and counts them; places beyond the
+  // list's 32 are not written.
+  unsigned lt_mask;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(lt_mask));
   int n_cand = 0;
 #pragma unroll
   for (int i = 0; i < VPT; ++i) {
     const bool c = expert_of(i) < E && key[i] >= tau;
-    if (c) mine |= 1u << i;
-    n_cand += __popc(__ballot_sync(0xffffffffu, c));
+    const unsigned b = __ballot_sync(0xffffffffu, c);
+    const int pos = n_cand + __popc(b & lt_mask);
+    if (c && pos < 32) s_cand[wib][pos] = ((unsigned long long)key[i] << 32) | (unsigned)(0x7fffffff - expert_of(i));
+    n_cand += __popc(b);
   }
   if (n_cand <= 32) {
-    // compact the candidates into the warp's list (any order), then rank each against all
-    int base = 0;
-#pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-      const bool c = (mine >> i) & 1u;
-      const unsigned b = __ballot_sync(0xffffffffu, c);
-      if (c) {
-        const int pos = base + __popc(b & ((1u << lane) - 1u));
-        s_key[wib][pos] = key[i];
-        s_idx[wib][pos] = expert_of(i);
-      }
-      base += __popc(b);
-    }
+    // rank each candidate against all
     __syncwarp();
     if (lane < n_cand) {
-      const unsigned kp = s_key[wib][lane];
-      const int ep = s_idx[wib][lane];
+      const unsigned long long pc = s_cand[wib][lane];
       int rank = 0;
-      for (int q = 0; q < n_cand; ++q) {
-        const unsigned kq = s_key[wib][q];
-        const int eq = s_idx[wib][q];
-        rank += (kq > kp || (kq == kp && eq < ep)) ? 1 : 0;
-      }
-      if (rank < k) s_sel[wib][rank] = ep;
+      for (int q = 0; q < n_cand; ++q) rank += s_cand[wib][q] > pc ? 1 : 0;
+      if (rank < k) s_sel[wib][rank] = 0x7fffffff - (int)(unsigned)(pc & 0xffffffffull);
     }
     __syncwarp();
     if (lane < k) my_e = s_sel[wib][lane];
