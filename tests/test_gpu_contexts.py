@@ -486,6 +486,50 @@ def test_prefill_pass_yields_between_tiles_and_resumes_bit_identically(fmt):
     p.close(); d.close()
 
 
+@pytest.mark.parametrize("phase,T", [(B.MOE_PHASE_DECODE, 48), (B.MOE_PHASE_PREFILL, 700)])
+@pytest.mark.parametrize("fmt", [B.MOE_WEIGHTS_BF16, B.MOE_WEIGHTS_FP8_E4M3])
+def test_steps_enqueued_back_to_back_equal_the_same_steps_run_one_at_a_time(phase, T, fmt):
+    """Every kernel is launched with the programmatic launch overlap, and the small-M GEMM builds its tile list and
+    requests weight boxes before it waits for the previous kernel of the stream.  Steps whose routing differs,
+    enqueued right behind one another without a host synchronisation, must give the bits each gives by itself."""
+    shape = wl.LayerShape("t", T=T, H=512, E=16, k=4, I=256, shared_I=128, select_bias=True)
+    fp8 = fmt == B.MOE_WEIGHTS_FP8_E4M3
+    w = wl.make_weights_fp8(shape, 1, DEV) if fp8 else wl.make_weights(shape, 1, DEV)
+    acts = [wl.make_activations(shape, 40 + i, DEV) for i in range(4)]  # four different routings
+    stream = torch.cuda.Stream()
+    ctx = B.MoeContext(B.make_config(512, 16, 4, 256, 128, T, phase, weight_format=fmt), stream=stream)
+
+    def step(a, out, bufs):
+        if fp8:
+            ctx.layer_fp8(a["x"], a["logits"], a["bias"], w, out=out, bufs=bufs)
+        else:
+            ctx.layer(a["x"], a["logits"], a["bias"], w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"],
+                      out=out, bufs=bufs)
+
+    bufs = [B.alloc_step_buffers(T, 4, 16, DEV) for _ in acts]
+    alone = [torch.empty(T, 512, dtype=torch.bfloat16, device=DEV) for _ in acts]
+    counts_alone = []
+    torch.cuda.synchronize()
+    for a, o, b in zip(acts, alone, bufs):
+        with torch.cuda.stream(stream):
+            step(a, o, b)
+        torch.cuda.synchronize()
+        counts_alone.append(b["counts"].clone())
+    assert not torch.equal(counts_alone[0], counts_alone[1])  # the routing really changes from step to step
+    outs = [torch.zeros_like(o) for o in alone]
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        for rep in range(3):
+            for a, o, b in zip(acts, outs, bufs):
+                step(a, o, b)
+    torch.cuda.synchronize()
+    assert ctx.moe_ctx_status() == B.MOE_OK
+    for i, (o, ref) in enumerate(zip(outs, alone)):
+        assert torch.equal(o, ref), f"step {i} differs when enqueued behind another step"
+        assert torch.equal(bufs[i]["counts"], counts_alone[i])
+    ctx.close()
+
+
 def test_decode_step_replays_from_a_cuda_graph():
     """D retains stable graph addresses: a captured D step replays with new inputs written into the same
     tensors and gives the bits of the eager step, with a P context busy on another stream or idle."""
