@@ -5,9 +5,9 @@
 //              (rounded up to 16), so an expert of up to 256 rows is ONE tile per feature tile and its weights
 //              enter an SM once; the MMA N is the chunk's row count rounded up to 16 (16..256).
 //   operands   a k-block (64 K-elements = 128-byte rows, 128-byte swizzle) is two 128-row weight boxes (32 KB,
-//              gated: gate rows + the matching up rows) and exactly N token rows, fetched as a binary
-//              decomposition of N into TMA boxes of 256/128/64/32/16 rows.  What bounds this regime is the
-//              bytes an SM ingests, so nothing is fetched that is not multiplied.
+//              gated: gate rows + the matching up rows; one TMA copy through a 4-D map) and exactly N token rows
+//              (one TMA copy through the map whose box has N rows: 16 maps, one per multiple of 16).  What bounds
+//              this regime is the bytes an SM ingests, so nothing is fetched that is not multiplied.
 //   ring       k-blocks live in a byte ring of 2 KB slots with FIFO allocation (a k-block takes 16 slots for its
 //              weights and N/16 for its token rows, two pieces that need not be adjacent), so a tile of few
 //              tokens keeps more k-blocks in flight than a tile of many; up to 8 k-blocks in flight, each with
@@ -16,9 +16,13 @@
 //   TMEM       512 columns = two halves.  A tile of N <= 128 takes one half (its two accumulators side by side)
 //              and alternates halves, so its epilogue overlaps the next tile's MMAs; a tile of N > 128 takes both.
 //   epilogue   lane = weight row (output feature), column = token: tcgen05.ld -> (scale) -> SwiGLU -> bf16;
-//              neighbouring lanes exchange values so that every store writes a feature pair.
+//              neighbouring lanes exchange values so that every store writes a feature pair.  The gated epilogue
+//              hands the accumulator back before its exchanges and stores.
+//   set-up     with the launch overlap, the tile list is built and weight boxes are requested before the kernel
+//              waits for the previous kernel of the stream; only the token rows and the stores wait for it.
 //
-// Warp roles (192 threads): warps 0-3 epilogue, warp 4 TMA producer, warp 5 MMA issuer and TMEM owner.
+// Warp roles (320 threads): warps 0-7 epilogue (two per TMEM lane group), warp 8 TMA producer, warp 9 MMA issuer
+// and TMEM owner.
 // Every mbarrier wait is bounded: on expiry the kernel records a timeout in the status word, raises a CTA-wide
 // abort flag, lets copies in flight land, frees its TMEM and returns.
 // The same kernel serves E4M3 operands (kind::f8f6f4, 128 K-elements per k-block, accumulator scaled by the
@@ -497,7 +501,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
 #endif
     }
   } else {
-    // ================================================================= epilogue (warps 0-3)
+    // ================================================================= epilogue (warps 0-7)
     // lane = weight row (output feature) of each box, TMEM column = token
     if (p.early_setup) {
       pdl_wait();
