@@ -3,6 +3,7 @@ T in {1, 16, 128, 1024, 8192, 32768}.  For every T: layer time and tokens/s, per
 load imbalance, and the fraction of the layer's roofline floor that was reached.
 
     python c5_sweep.py [--tokens 1 16 128 ...] [--iters-min-ms 300] [--fp8]
+    python c5_sweep.py --route-only [--tokens ...]     # stage a1 by itself (no weights are allocated)
 
 One JSON object per T on stdout.  The floor of a step is the sum over its stages of
 max(flops / tensor peak, algorithmic bytes / HBM peak); for the grouped GEMMs it is summed per expert
@@ -111,6 +112,42 @@ def run_one(shape, weights, min_ms, dev="cuda", fp8=False):
     return step_us, n, {k_: round(1e3 * ms / c, 1) for k_, (ms, c) in prof.items() if c}, counts
 
 
+def route_only(tokens, E, k, zipf, hbm, src, launches=200):
+    """Stage a1 by itself on the sweep's logits: microseconds per launch (back to back on one stream, so the figure
+    includes the launch rate of tiny problems) and the achieved fraction of the HBM copy rate."""
+    dev = "cuda"
+    for T in tokens:
+        shape = wl.LayerShape("route", T=T, H=64, E=E, k=k, I=64, zipf_s=zipf, select_bias=zipf == 0)
+        acts = [wl.make_activations(shape, 600 + i, dev) for i in range(3)]
+        stream = torch.cuda.Stream()
+        ctx = B.MoeContext(B.make_config(64, E, k, 64, 0, T, B.MOE_PHASE_PREFILL), stream=stream)
+        idx = torch.empty(T, k, dtype=torch.int32, device=dev)
+        w = torch.empty(T, k, dtype=torch.float32, device=dev)
+
+        def run(n):
+            for i in range(n):
+                a = acts[i % 3]
+                ctx.moe_route(a["logits"], a["bias"], idx, w)
+                ctx.moe_ctx_abandon_step()
+
+        with torch.cuda.stream(stream):
+            run(5)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            run(launches)
+            e1.record(stream)
+        torch.cuda.synchronize()
+        us = 1e3 * e0.elapsed_time(e1) / launches
+        by = 4.0 * T * E + 4.0 * E + 8.0 * T * k
+        assert ctx.moe_ctx_status() == B.MOE_OK
+        ctx.close()
+        print(json.dumps({"workload": f"route only, E={E} top-{k} T={T}", "us_per_launch": round(us, 2),
+                          "algorithmic_bytes": by, "GBps": round(by / us / 1e3, 1),
+                          "frac_hbm": round(by / us / 1e3 / hbm, 3), "peak_source": src}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--tokens", type=int, nargs="*", default=list(wl.C5_TOKENS))
@@ -120,9 +157,13 @@ def main():
     ap.add_argument("--fp8", action="store_true", help="the FP8 (E4M3) precision variant instead of bf16")
     ap.add_argument("--zipf", type=float, default=wl.C5.zipf_s,
                     help="exponent of the expert popularity (0 = uniform routing with a selection bias, as in workloads C2/C4)")
+    ap.add_argument("--route-only", action="store_true", help="time stage a1 (routing) by itself; no weights are allocated")
     args = ap.parse_args()
     B.load_library()
     hbm, tfl, src = load_peaks()
+    if args.route_only:
+        route_only(args.tokens, args.experts, wl.C5.k, args.zipf, hbm, src)
+        return
     import dataclasses
     base = dataclasses.replace(wl.C5, E=args.experts, zipf_s=args.zipf, select_bias=args.zipf == 0)
     weights = (wl.make_weights_fp8 if args.fp8 else wl.make_weights)(base, 2, "cuda")
