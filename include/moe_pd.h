@@ -268,13 +268,14 @@ moe_status moe_ctx_set_segments(moe_ctx* ctx, int32_t experts_per_segment, moe_b
  * The paper lets successive D iterations advance through one long P execution at backend-provided boundaries
  * (Section "In-Place P/D Execution"); on one GPU, where P and D compete for the same SMs and the same HBM, the
  * finest boundary that costs nothing while no D is waiting is the end of a GEMM tile.  With preemption on (PREFILL
- * contexts only), every GEMM pass of moe_grouped_ffn uses the small-M kernel, whose CTAs look at a yield request
- * before each tile (tens of microseconds apart).  moe_ctx_request_yield(ctx, 1) -- callable from any host thread,
- * typically the one about to enqueue a D step -- raises the request: every CTA finishes the tile it is in, saves
- * its position and exits, so the SMs are free within one tile's time.  moe_grouped_ffn, which in this mode WAITS
+ * contexts only), every GEMM pass of moe_grouped_ffn uses the small-M kernel, whose CTAs take their tiles from a
+ * counter in the context's workspace and look at a yield request before they take one (tens of microseconds
+ * apart).  moe_ctx_request_yield(ctx, 1) -- callable from any host thread, typically the one about to enqueue a D
+ * step -- raises the request: every CTA finishes the tiles it has taken (the one it is in and at most the next) and
+ * exits, so the SMs are free within a tile or two.  moe_grouped_ffn, which in this mode WAITS
  * ON THE HOST for each of its launches (eager variable-length P; it cannot be captured in a graph and costs a
  * host round trip of ~10 us per launch), then calls the boundary hook as fn(user, MOE_BOUNDARY_YIELD, 0) and,
- * when the hook returns, launches the pass again: every CTA resumes where it stopped.  The hook is the permit
+ * when the hook returns, launches the pass again: the counter goes on with the tiles not yet taken.  The hook is the permit
  * wait: it should return once the D step has finished on the device and the request has been lowered
  * (moe_ctx_request_yield(ctx, 0)); a request still up is honoured again (up to 64 launches per pass, after which
  * the pass runs to its end regardless).  Results are bit-identical to the unpreempted pass.  The request is a

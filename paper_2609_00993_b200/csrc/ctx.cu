@@ -59,10 +59,10 @@ struct Layout {
 // Status block at the start of the workspace: word 0 the device status, word 1 the count of CTAs that stopped on a
 // yield request in the last preemptible launch, word 2 the yield request itself (device memory: every CTA polls it
 // before each tile, which a word in host memory would not survive -- 148 SMs reading it over PCIe serialise), and
-// from byte 256 on the per-CTA progress of a preemptible pass.
+// from byte 64 on four pairs {next tile, CTAs finished} that the small-M GEMM launches use in rotation.
 constexpr size_t kStatusBlock = 8192;
-constexpr size_t kProgressOffset = 256;
-constexpr int kProgressInts = (int)((kStatusBlock - kProgressOffset) / sizeof(int));
+constexpr size_t kTileCounterOffset = 64;
+constexpr int kTileCounterPairs = 4;
 
 // Walks the carve of one buffer set; with base == nullptr it only measures.
 size_t carve_set(const moe_config& c, char* base, BufferSet* out) {
@@ -179,6 +179,7 @@ struct moe_ctx {
   bool pending_dispatch;
   cudaEvent_t notified;
   bool split_step;   // the step in progress went through the split entry points (boundary numbering)
+  unsigned gemm_seq = 0;  // GEMM launches so far: selects the tile-counter pair of the next one
   // prefill segmentation (off by default)
   int seg_experts;
   moe_boundary_fn boundary_fn;
@@ -327,6 +328,7 @@ cudaError_t run_gemm(moe_ctx* ctx, moe::GemmProblem p, const moe::GemmDenseGroup
   // Every GEMM launch comes after the step's row movement (or after another GEMM launch or a quantisation of the
   // same step), which in turn waited for the layout kernels: the offsets are older than the previous kernel.
   p.offsets_settled = true;
+  p.tile_counters = reinterpret_cast<int*>(ctx->ws + kTileCounterOffset) + 2 * (ctx->gemm_seq++ % kTileCounterPairs);
   p.max_group_rows = T;
   if (variant == MOE_GEMM_VALIDATION) {
     cudaError_t e = moe::launch_gemm_validation(p, ctx->stream, n);
@@ -339,13 +341,11 @@ cudaError_t run_gemm(moe_ctx* ctx, moe::GemmProblem p, const moe::GemmDenseGroup
   }
   if (variant == MOE_GEMM_SMALL_M && ctx->preemptible && !capturing(ctx)) {
     // A pass that can be asked to stop between tiles: launch, wait on the host for the launch to end, and if
-    // CTAs stopped on a yield request report the boundary and launch again (each CTA resumes where it stopped).
-    int* progress = reinterpret_cast<int*>(ctx->ws + kProgressOffset);
+    // CTAs stopped on a yield request report the boundary and launch again with the same tile counter, which
+    // goes on with the tiles not yet taken.
     int* stopped = ctx->status + 1;
-    if (gemm_ctas(ctx) > kProgressInts) return cudaErrorNotSupported;
-    p.progress = progress;
     p.stopped = stopped;
-    cudaError_t e = cudaMemsetAsync(progress, 0, sizeof(int) * (size_t)gemm_ctas(ctx), ctx->stream);
+    cudaError_t e = cudaMemsetAsync(p.tile_counters, 0, 2 * sizeof(int), ctx->stream);  // (an abandoned pass may have left them)
     for (int attempt = 0; e == cudaSuccess; ++attempt) {
       // a request that is still up after the hook has returned is honoured once more, then overridden: the pass
       // must end even with a controller that never clears its request

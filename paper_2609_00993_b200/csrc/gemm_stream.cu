@@ -18,6 +18,10 @@
 //   epilogue   lane = weight row (output feature), column = token: tcgen05.ld -> (scale) -> SwiGLU -> bf16;
 //              neighbouring lanes exchange values so that every store writes a feature pair.  The gated epilogue
 //              hands the accumulator back before its exchanges and stores.
+//   schedule   the tile list is ordered by expert size, largest first.  Its first waves are dealt statically (CTAs
+//              in step share weights and rows through L2), the last two waves' worth of tiles -- the smallest -- are
+//              handed out by an atomic counter to whichever CTA is free; the producer publishes the tiles it takes
+//              in a four-entry queue that the MMA issuer and the epilogue warps follow.
 //   set-up     with the launch overlap, the tile list is built and weight boxes are requested before the kernel
 //              waits for the previous kernel of the stream; only the token rows and the stores wait for it.
 //
@@ -63,6 +67,11 @@ constexpr int kMaxTileRows = 256;                       // largest MMA N
 constexpr int kNB = 8;                                  // k-blocks in flight at most (barrier pairs)
 constexpr int kXMaps = 16;                              // token-row boxes of 16 (b + 1) rows
 constexpr uint32_t kTmemCols = 512;
+constexpr int kQ = 4;                                   // entries of the CTA's tile queue
+#ifndef MOE_STREAM_DYN_WAVES
+#define MOE_STREAM_DYN_WAVES 2
+#endif
+constexpr int kDynWaves = MOE_STREAM_DYN_WAVES;         // waves' worth of tiles, at the list's end, handed out dynamically
 
 struct StreamParams {
   const int32_t* offsets;  // [E+1] (already advanced to the first expert of the launch) or nullptr
@@ -86,9 +95,12 @@ struct StreamParams {
   const float* row_scale2;
   const float* w_scale;
   const float* w_scale2;
-  // preemption at tile granularity (all null: off)
+  // The launch's tile counter and the count of CTAs that have finished (two words in device memory, zero before the
+  // first launch that uses them; the last CTA to finish puts them back to zero).
+  int* tile_ctr;
+  int* done_ctr;
+  // preemption at tile granularity (both null: off)
   const int* yield_req;
-  int* progress;
   int* stopped;
   // The expert offsets were final before the PREVIOUS kernel of the stream started (and the weights always are):
   // the tile list is built and weight boxes are fetched before this kernel waits for that previous kernel, which
@@ -125,12 +137,6 @@ __device__ __forceinline__ void chunking(int cnt, int& tiles, int& chunk) {
   chunk = tiles > 0 ? (((cnt + tiles - 1) / tiles) + 15) & ~15 : 0;
 }
 
-// Position of a CTA's w-th tile in the tile list: the list is dealt in waves of n_units tiles, alternately
-// forwards and backwards, so that with tiles ordered by cost no CTA always gets the costliest tile of a wave.
-__device__ __forceinline__ int snake_tile(int w, int unit, int n_units) {
-  return w * n_units + ((w & 1) ? n_units - 1 - unit : unit);
-}
-
 // tile -> (expert, first row, valid rows, feature tile).  The dense group's tiles come first (chunk major),
 // then the experts' in the order `order` (largest first): prefix[i] = chunks of the experts at positions < i.
 __device__ __forceinline__ STile decode_tile(int tile, int dense_tiles, int n_ft2, int rows2, int n_ft, int E,
@@ -165,34 +171,14 @@ __device__ __forceinline__ STile decode_tile(int tile, int dense_tiles, int n_ft
   return t;
 }
 
-// mbar_wait that also ends when the producer has announced that wave `w` will not be started (*stop_w <= w).
-// 0: the barrier's phase completed; 1: time limit or abort; 2: the CTA stops before this wave.
-__device__ __forceinline__ int mbar_wait_or_stop(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                                 unsigned long long limit_ns, const volatile int* stop_w, int w) {
-  unsigned long long t0 = 0;
-  for (uint32_t i = 0;; ++i) {
-    if (mbar_try_wait(bar, parity)) return 0;
-    if ((i & 31u) == 31u && *stop_w <= w) return mbar_try_wait(bar, parity) ? 0 : 2;
-    if (i >= 256u) {
-      if ((i & 255u) == 0u) {
-        if (*abort_flag) return 1;
-        const unsigned long long now = global_ns();
-        if (t0 == 0) t0 = now;
-        else if (now - t0 > limit_ns) return 1;
-      }
-      __nanosleep(64);
-    }
-  }
-}
-
 template <bool GATED, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
                            const __grid_constant__ StreamMaps xmaps, const __grid_constant__ StreamParams p) {
   constexpr int kbk = FP8 ? 2 * kBlockK : kBlockK;  // K elements per k-block
   extern __shared__ uint8_t smem_raw[];
-  // carve: ring (ring_slots x 2 KB) | full[kNB] empty[kNB] tfull[2] tempty[2] | tmem slot | abort | sizes[kNB]
-  //        | prefix[E+1] | order[E] | beg[E] | cnts[E]
+  // carve: ring (ring_slots x 2 KB) | full[kNB] empty[kNB] tfull[2] tempty[2] tqfull[kQ] tqempty[kQ] | tmem slot
+  //        | abort | stopped | sizes[kNB] | tq[kQ] | prefix[E+1] | order[E] | beg[E] | cnts[E]
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t base_addr = (raw_addr + 1023u) & ~1023u;
   uint8_t* base = smem_raw + (base_addr - raw_addr);
@@ -201,17 +187,20 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   const uint32_t bar_empty = bar_full + 8u * kNB;
   const uint32_t bar_tfull = bar_empty + 8u * kNB;
   const uint32_t bar_tempty = bar_tfull + 16u;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kNB + 4);
+  const uint32_t bar_tqfull = bar_tempty + 16u;         // the tile queue: an entry has been published
+  const uint32_t bar_tqempty = bar_tqfull + 8u * kQ;    // ... and read by the issuer and every epilogue warp
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kNB + 4 + 2 * kQ);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* stop_w = reinterpret_cast<volatile int*>(tmem_slot + 2);  // first wave this CTA will not start
+  volatile int* stopped_here = reinterpret_cast<volatile int*>(tmem_slot + 2);  // the producer stopped on request
   int* sizes = reinterpret_cast<int*>(tmem_slot + 3);  // slots held by the k-blocks in flight (producer only)
-  int* prefix = sizes + kNB;
+  volatile int* tq = reinterpret_cast<volatile int*>(sizes + kNB);  // tile queue entries (-1: no more tiles)
+  int* prefix = sizes + kNB + kQ;
   int* order = prefix + (p.E + 1);
   int* beg = order + p.E;
   int* cnts = beg + p.E;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int unit = (int)blockIdx.x, n_units = (int)gridDim.x;
+  [[maybe_unused]] const int unit = (int)blockIdx.x;
   if (threadIdx.x == 0) PROF_STAMP(0);
   constexpr int kFeatPerTile = GATED ? 128 : 256;
   const int n_ft = (p.n_feat + kFeatPerTile - 1) / kFeatPerTile;
@@ -231,8 +220,12 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       mbar_init(bar_tfull + 8u * a, kIssuers);
       mbar_init(bar_tempty + 8u * a, kEpilogueWarps);
     }
+    for (int q = 0; q < kQ; ++q) {
+      mbar_init(bar_tqfull + 8u * q, 1);
+      mbar_init(bar_tqempty + 8u * q, kIssuers + kEpilogueWarps);
+    }
     *abort_flag = 0;
-    *stop_w = 0x7fffffff;
+    *stopped_here = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -290,7 +283,6 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   if (threadIdx.x == 0) PROF_STAMP(2);
   const int total_tiles = dense_tiles + prefix[p.E] * n_ft;
   const uint32_t R = (uint32_t)p.ring_slots;
-  const int w_first = p.progress ? p.progress[unit] : 0;  // a resumed pass continues where this CTA stopped
 
   if (warp == kProducerWarp) {
     // ================================================================= TMA producer (one lane)
@@ -316,19 +308,49 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       int yield_seen = 0;
       if (p.yield_req != nullptr)
         asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(yield_seen) : "l"(p.yield_req) : "memory");
-      for (int w = w_first; w * n_units < total_tiles && ok; ++w) {
-        const int tile = snake_tile(w, unit, n_units);
-        if (tile >= total_tiles) break;
-        if (p.yield_req != nullptr) {
-          // the request word was read while the previous tile's copies were being issued, so looking at it here
-          // does not stall the pipeline; the read for the next tile goes out now
-          const int y = yield_seen;
-          asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(yield_seen) : "l"(p.yield_req) : "memory");
-          if (y != 0) {
-            *stop_w = w;  // the other roles finish the waves below w and leave
-            break;
-          }
+      // Tiles are handed out by a counter in device memory, in the list's order (largest experts first): a CTA
+      // that finishes early takes the next tile, whichever CTA would have had it.  The producer publishes every tile
+      // it takes -- and finally -1 -- in a small queue that the issuer and the epilogue warps follow.
+      uint32_t tcount = 0;
+      auto publish = [&](int tile) -> bool {
+        const uint32_t q = tcount % kQ, par = ((tcount / kQ) & 1u) ^ 1u;
+        // the epilogue warps free an entry only after the tile before it, which needs its token rows: the copies
+        // put off by the early set-up go out before this thread blocks
+        if (!dep_waited && !mbar_try_wait(bar_tqempty + 8u * q, par)) dep_wait_and_flush();
+        if (!mbar_wait(bar_tqempty + 8u * q, par, abort_flag, limit)) return false;
+        tq[q] = tile;
+        mbar_arrive(bar_tqfull + 8u * q);
+        ++tcount;
+        return true;
+      };
+      // The counter is read a few k-blocks before the current tile's last copy, so that the atomic's round trip hides
+      // behind those copies -- and no earlier, so that a CTA does not hold a second tile while another CTA has none.
+      // A stop on request therefore takes effect after the tile that had already been taken.
+      // The first waves are dealt statically (wave w: tile w * grid + the CTA's index, alternately forwards and
+      // backwards): CTAs that run in step start the tiles that share an expert's weights or rows together, and the
+      // second reader finds them in L2.  The last kDynWaves waves' worth of tiles -- the smallest ones, the list being
+      // ordered by size -- go to whichever CTA is free, which evens out what the static part left uneven.  A pass that
+      // can be stopped on request is dynamic throughout: its next launch only needs the counter to go on.
+      const int grid = (int)gridDim.x;
+      // (At least the first wave is static, which also spares every CTA a contended atomic at the start.)
+      const int w_static = p.yield_req != nullptr ? 0 : max(1, total_tiles / grid - kDynWaves);
+      int sw = 0;
+      auto next_tile = [&]() -> int {
+        if (sw < w_static) {
+          const int w = sw++;
+          return w * grid + ((w & 1) ? grid - 1 - (int)blockIdx.x : (int)blockIdx.x);
         }
+        return w_static * grid + atomicAdd(p.tile_ctr, 1);
+      };
+      int taken = next_tile();
+      for (;;) {
+        const int tile = taken < total_tiles ? taken : -1;
+        if (!publish(tile)) {
+          ok = false;
+          break;
+        }
+        if (tile < 0) break;
+        bool stop_after = false;
         const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
         const uint32_t n = (uint32_t)((t.rows + 15) & ~15);
         const int w_row0 = t.ft * kFeatPerTile;
@@ -336,7 +358,17 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
         const CUtensorMap* mx = (t.dense ? xmaps.x2 : xmaps.x) + ((n >> 4) - 1u);  // the box of exactly n rows
         const int w_e = t.dense ? 0 : p.e_base + t.e;
         const int num_kb = t.dense ? num_kb2 : num_kb1;
+        const int fetch_kb = num_kb > 4 ? num_kb - 4 : 0;
         for (int kb = 0, k0 = 0; kb < num_kb && ok; ++kb, k0 += kbk) {
+          if (kb == fetch_kb) {
+            if (p.yield_req != nullptr) {
+              // the request word was read a tile ago, so looking at it here does not stall the pipeline; the read for
+              // the next tile goes out now
+              stop_after = yield_seen != 0;
+              asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(yield_seen) : "l"(p.yield_req) : "memory");
+            }
+            if (!stop_after) taken = next_tile();
+          }
           // The ring is allocated per operand: the weight boxes and the token rows of a k-block are two contiguous
           // pieces that need not be adjacent, so the weights of the next k-block go out as soon as 16 slots are
           // free.  A piece never wraps: it skips what is left at the ring's end.
@@ -386,6 +418,11 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
           head = head_x + nx;
           ++kb_idx;
         }
+        if (stop_after && ok) {
+          *stopped_here = 1;  // no further tile is taken: the other roles finish the published ones and leave
+          if (!publish(-1)) ok = false;
+          break;
+        }
       }
       if (!dep_waited) dep_wait_and_flush();
       if (!ok) {
@@ -410,10 +447,17 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       const uint32_t desc_hi = (uint32_t)(umma_smem_desc(0) >> 32);
       const uint32_t lo_base = (uint32_t)umma_smem_desc(base_addr);  // slot 0
       constexpr uint32_t lo_slot = (uint32_t)kSlotBytes >> 4, lo_box = (uint32_t)kWBoxBytes >> 4;
-      bool stopped = false;
-      for (int w = w_first; w * n_units < total_tiles && ok && !stopped; ++w) {
-        const int tile = snake_tile(w, unit, n_units);
-        if (tile >= total_tiles) break;
+      uint32_t tcount = 0;
+      for (;;) {
+        const uint32_t q = tcount % kQ;
+        if (!mbar_wait(bar_tqfull + 8u * q, (tcount / kQ) & 1u, abort_flag, limit)) {
+          ok = false;
+          break;
+        }
+        const int tile = tq[q];
+        mbar_arrive(bar_tqempty + 8u * q);
+        ++tcount;
+        if (tile < 0) break;
         const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
         const uint32_t n = (uint32_t)((t.rows + 15) & ~15);
         const bool big = n > 128u;
@@ -448,13 +492,9 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
           head += n >> 4;
           {
             PROF_T0();
-            // the wait for a tile's first k-block also ends when the producer has decided not to start the tile
-            const uint32_t fb = bar_full + 8u * (kb_idx % kNB), fp = (kb_idx / kNB) & 1u;
-            const int got = kb == 0 ? mbar_wait_or_stop(fb, fp, abort_flag, limit, stop_w, w)
-                                    : (mbar_wait(fb, fp, abort_flag, limit) ? 0 : 1);
+            const bool got = mbar_wait(bar_full + 8u * (kb_idx % kNB), (kb_idx / kNB) & 1u, abort_flag, limit);
             PROF_ADD(prof_wait_full);
-            if (got == 2) { stopped = true; break; }
-            if (got != 0) { ok = false; break; }
+            if (!got) { ok = false; break; }
           }
           if (kb_idx == 0) PROF_STAMP(3);
           tc_fence_after();
@@ -474,7 +514,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
           umma_commit(bar_empty + 8u * (kb_idx % kNB));  // the k-block's slots are free once these MMAs have read them
           ++kb_idx;
         }
-        if (!ok || stopped) break;
+        if (!ok) break;
         if (big) {
           umma_commit(bar_tfull);
           umma_commit(bar_tfull + 8u);
@@ -514,17 +554,25 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
     const uint32_t lane_base = ((uint32_t)(lg * 32)) << 16;
     const int fl = lg * 32 + lane;
     const bool even = (lane & 1) == 0;
-    for (int w = w_first; w * n_units < total_tiles && ok; ++w) {
-      const int tile = snake_tile(w, unit, n_units);
-      if (tile >= total_tiles) break;
+    uint32_t tcount = 0;
+    for (;;) {
+      const uint32_t q = tcount % kQ;
+      if (!mbar_wait(bar_tqfull + 8u * q, (tcount / kQ) & 1u, abort_flag, limit)) {
+        ok = false;
+        break;
+      }
+      const int tile = tq[q];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tqempty + 8u * q);
+      ++tcount;
+      if (tile < 0) break;
       const STile t = decode_tile(tile, dense_tiles, n_ft2, p.rows2, n_ft, p.E, prefix, order, beg, cnts);
       const uint32_t n = (uint32_t)((t.rows + 15) & ~15);
       const bool big = n > 128u;
       uint32_t h = 0, d_a, d_b;
       if (big) {
-        const int got = mbar_wait_or_stop(bar_tfull, use0 & 1u, abort_flag, limit, stop_w, w);
-        if (got == 2) break;  // the CTA stops before this wave
-        if (got != 0 || !mbar_wait(bar_tfull + 8u, use1 & 1u, abort_flag, limit)) { ok = false; break; }
+        if (!mbar_wait(bar_tfull, use0 & 1u, abort_flag, limit) ||
+            !mbar_wait(bar_tfull + 8u, use1 & 1u, abort_flag, limit)) { ok = false; break; }
         ++use0;
         ++use1;
         d_a = tmem_base;
@@ -532,9 +580,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       } else {
         h = next_half;
         next_half ^= 1u;
-        const int got = mbar_wait_or_stop(bar_tfull + 8u * h, (h ? use1 : use0) & 1u, abort_flag, limit, stop_w, w);
-        if (got == 2) break;
-        if (got != 0) { ok = false; break; }
+        if (!mbar_wait(bar_tfull + 8u * h, (h ? use1 : use0) & 1u, abort_flag, limit)) { ok = false; break; }
         if (h) ++use1; else ++use0;
         d_a = tmem_base + 256u * h;
         d_b = d_a + 128u;
@@ -696,13 +742,15 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0) PROF_STAMP(6);
-  if (p.progress != nullptr && threadIdx.x == 0) {
-    const int sw = *stop_w;
-    if (sw != 0x7fffffff) {  // stopped on request: the next launch of this pass resumes at wave sw
-      p.progress[unit] = sw;
-      atomicAdd(p.stopped, 1);
-    } else {
-      p.progress[unit] = (total_tiles + n_units - 1) / n_units;  // every wave done: a resumed launch finds nothing
+  if (threadIdx.x == 0) {
+    // The last CTA to get here puts the counters back for the next launch that uses them.  After a stop on request
+    // the tile counter stays: the next launch of the pass goes on where this one stopped taking tiles.
+    if (*stopped_here) atomicAdd(p.stopped, 1);
+    __threadfence();
+    if (atomicAdd(p.done_ctr, 1) == (int)gridDim.x - 1) {
+      const bool any_stopped = p.stopped != nullptr && *reinterpret_cast<volatile int*>(p.stopped) != 0;
+      *p.done_ctr = 0;
+      if (!any_stopped) *p.tile_ctr = 0;
     }
   }
   if (*abort_flag) {
@@ -801,14 +849,16 @@ cudaError_t launch_gemm_stream(const GemmProblem& p, const GemmDenseGroup* dense
   prm.w_scale = p.w_scale;
   prm.row_scale2 = dense ? dense->row_scale : nullptr;
   prm.w_scale2 = dense ? dense->w_scale : nullptr;
-  const bool preemptible = p.yield_req != nullptr && p.progress != nullptr && p.stopped != nullptr;
+  if (p.tile_counters == nullptr) return cudaErrorInvalidValue;
+  prm.tile_ctr = p.tile_counters;
+  prm.done_ctr = p.tile_counters + 1;
+  const bool preemptible = p.yield_req != nullptr && p.stopped != nullptr;
   prm.sort_tiles = (p.max_group_rows > 0 && p.max_group_rows <= 16) ? 0 : 1;
-  prm.early_setup = (p.offsets_settled && !preemptible) ? 1 : 0;  // a resumed pass reads its progress words first
+  prm.early_setup = (p.offsets_settled && !preemptible) ? 1 : 0;
   prm.yield_req = preemptible ? p.yield_req : nullptr;
-  prm.progress = preemptible ? p.progress : nullptr;
   prm.stopped = preemptible ? p.stopped : nullptr;
 
-  const size_t tail = (2 * kNB + 4) * sizeof(uint64_t) + 3 * sizeof(uint32_t) + kNB * sizeof(int) +
+  const size_t tail = (2 * kNB + 4 + 2 * kQ) * sizeof(uint64_t) + 3 * sizeof(uint32_t) + (kNB + kQ) * sizeof(int) +
                       4 * (size_t)(prm.E + 1) * sizeof(int);
   const int slots = (int)((kSmemBudget - 1024 - (int)tail) / kSlotBytes);
   if (slots < 2 * (kWSlots + kMaxTileRows / 16)) return cudaErrorNotSupported;

@@ -113,13 +113,16 @@ struct GemmProblem {
   // failure-detection hook (the TMA producer issues nothing, so every consumer wait runs into the limit).
   unsigned long long wait_limit_ns = 0;
   bool debug_stall = false;
-  // Preemption at tile granularity (small-M kernel only; all three null = off).  Before each of its tiles a CTA
-  // reads *yield_req; when it is non-zero the CTA finishes the tiles it has begun, stores the number of tiles it
-  // has done in progress[blockIdx.x], adds one to *stopped and exits.  A launch starts every CTA at
-  // progress[blockIdx.x], so launching the same problem again (same grid) resumes the pass; the caller zeroes
-  // progress before the first launch of a pass.  yield_req and stopped may live in mapped host memory.
+  // Small-M kernel: two words of device memory, {next tile, CTAs finished}, zero before the launch; the launch's CTAs
+  // take their tiles from the first (an atomic counter over the size-ordered tile list) and the last CTA to finish
+  // puts both back to zero.  Consecutive launches of a stream must use different pairs: with the launch overlap the
+  // next kernel's CTAs take tiles while this one's are still finishing.
+  int* tile_counters = nullptr;
+  // Preemption at tile granularity (small-M kernel only; both null = off).  Before it takes a tile a CTA reads
+  // *yield_req; when it is non-zero the CTA finishes the tiles it has taken, adds one to *stopped and exits, and the
+  // tile counter is left where it is: launching the same problem again with the same tile_counters goes on with the
+  // tiles not yet taken.
   const int* yield_req = nullptr;
-  int* progress = nullptr;
   int* stopped = nullptr;
   // Small-M kernel: `offsets` was final before the previous kernel of the stream started, so the kernel may read it
   // (and fetch weights) before it waits for that kernel; only the rows of A (and the FP8 row scales) wait.
