@@ -345,6 +345,7 @@ cudaError_t run_gemm(moe_ctx* ctx, moe::GemmProblem p, const moe::GemmDenseGroup
     // goes on with the tiles not yet taken.
     int* stopped = ctx->status + 1;
     p.stopped = stopped;
+    p.resumable = true;
     cudaError_t e = cudaMemsetAsync(p.tile_counters, 0, 2 * sizeof(int), ctx->stream);  // (an abandoned pass may have left them)
     for (int attempt = 0; e == cudaSuccess; ++attempt) {
       // a request that is still up after the hook has returned is honoured once more, then overridden: the pass

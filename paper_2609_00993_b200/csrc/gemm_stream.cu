@@ -99,6 +99,7 @@ struct StreamParams {
   // first launch that uses them; the last CTA to finish puts them back to zero).
   int* tile_ctr;
   int* done_ctr;
+  int32_t all_dynamic;  // every tile comes from the counter (a pass that may be launched again to go on)
   // preemption at tile granularity (both null: off)
   const int* yield_req;
   int* stopped;
@@ -333,7 +334,7 @@ grouped_gemm_stream_kernel(const __grid_constant__ CUtensorMap map_w, const __gr
       // can be stopped on request is dynamic throughout: its next launch only needs the counter to go on.
       const int grid = (int)gridDim.x;
       // (At least the first wave is static, which also spares every CTA a contended atomic at the start.)
-      const int w_static = p.yield_req != nullptr ? 0 : max(1, total_tiles / grid - kDynWaves);
+      const int w_static = p.all_dynamic ? 0 : max(1, total_tiles / grid - kDynWaves);
       int sw = 0;
       auto next_tile = [&]() -> int {
         if (sw < w_static) {
@@ -852,6 +853,7 @@ cudaError_t launch_gemm_stream(const GemmProblem& p, const GemmDenseGroup* dense
   if (p.tile_counters == nullptr) return cudaErrorInvalidValue;
   prm.tile_ctr = p.tile_counters;
   prm.done_ctr = p.tile_counters + 1;
+  prm.all_dynamic = p.resumable ? 1 : 0;
   const bool preemptible = p.yield_req != nullptr && p.stopped != nullptr;
   prm.sort_tiles = (p.max_group_rows > 0 && p.max_group_rows <= 16) ? 0 : 1;
   prm.early_setup = (p.offsets_settled && !preemptible) ? 1 : 0;

@@ -124,6 +124,9 @@ struct GemmProblem {
   // tiles not yet taken.
   const int* yield_req = nullptr;
   int* stopped = nullptr;
+  // Every launch of a pass that may be stopped and launched again sets this (also a launch without yield_req that
+  // finishes such a pass): all its tiles come from the counter, none is dealt statically.
+  bool resumable = false;
   // Small-M kernel: `offsets` was final before the previous kernel of the stream started, so the kernel may read it
   // (and fetch weights) before it waits for that kernel; only the rows of A (and the FP8 row scales) wait.
   bool offsets_settled = false;

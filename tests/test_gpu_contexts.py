@@ -484,6 +484,22 @@ def test_prefill_pass_yields_between_tiles_and_resumes_bit_identically(fmt):
     p.moe_ctx_request_yield(False)
     p.moe_ctx_set_preemption(False)
     p.close(); d.close()
+    # the same on four CTAs, where a launch that stops at once gets through four tiles: a request that stays up is
+    # honoured 64 times per pass and then overridden by a launch that runs to the pass's end
+    p4 = B.MoeContext(B.make_config(1024, 32, 4, 512, 256, 3000, B.MOE_PHASE_PREFILL, sm_budget=4, weight_format=fmt),
+                      stream=sp)
+    p4.moe_ctx_set_preemption(True)
+    p4.moe_ctx_set_segments(0, lambda i, n: None)
+    p4.moe_ctx_request_yield(True)
+    p_out.zero_()
+    with torch.cuda.stream(sp):
+        step(p4, ap, p_out, bp)
+    sp.synchronize()
+    assert p4.moe_ctx_yield_count() >= 128   # 64 in each of the two passes
+    assert torch.equal(p_out, p_alone)
+    p4.moe_ctx_request_yield(False)
+    assert p4.moe_ctx_status() == B.MOE_OK
+    p4.close()
 
 
 @pytest.mark.parametrize("phase,T", [(B.MOE_PHASE_DECODE, 48), (B.MOE_PHASE_PREFILL, 700)])
