@@ -654,6 +654,31 @@ def c5_block(torch, w, peaks, min_ms=100.0):
             "floor": "sum over stages of max(flops / sustained bf16 peak, algorithmic bytes / HBM copy rate), per expert for the GEMMs"}
 
 
+def paper_shape_block(torch, peaks, dev, min_ms=100.0):
+    """The model shape the paper names (hidden 2,560, 512 routed experts, top-8; Section "Evaluation"), whose expert
+    intermediate size it does not state: I = 1024 is this build's choice.  A decode-sized and two prefill-sized
+    batches, uniform routing with a selection bias, each timed for >= min_ms: tokens/s and the fraction of the
+    per-expert roofline floor."""
+    import c5_sweep
+    from paper_2609_00993_b200 import workloads as wl
+    hbm, tfl = peaks["hbm_gbs"], peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    base = wl.LayerShape("paper-shape", T=64, H=2560, E=512, k=8, I=1024, shared_I=0, select_bias=True)
+    w = wl.make_weights(base, 7, dev)
+    rows = []
+    for T in (64, 4096, 32768):
+        shape = base.with_tokens(T)
+        step_us, n, stages, counts = c5_sweep.run_one(shape, w, min_ms)
+        floor_us, _, _ = c5_sweep.layer_floor_us(shape, counts, hbm, tfl)
+        rows.append({"T": T, "phase": "decode" if T <= 256 else "prefill", "step_us": round(step_us, 1),
+                     "tokens_per_s": round(T / (step_us * 1e-6), 1), "roofline_floor_us": round(floor_us, 1),
+                     "frac_of_roofline": round(floor_us / step_us, 3), "nonempty_experts": int((counts > 0).sum()),
+                     "stages_us": stages, "iters": n})
+    del w
+    torch.cuda.empty_cache()
+    return {"workload": "H=2560, E=512, top-8 (the paper's model shape), I=1024 (not stated in the paper: chosen here), "
+                        "no shared expert, bf16, 8.05 GB of expert weights", "rows": rows}
+
+
 def run_ours(args):
     import torch
     from paper_2609_00993_b200 import binding as B
@@ -949,6 +974,11 @@ def run_ours(args):
         except Exception as exc:
             line["c5"] = {"error": repr(exc)}
         del w_v3
+        torch.cuda.empty_cache()
+        try:
+            line["paper_shape"] = paper_shape_block(torch, peaks, dev)
+        except Exception as exc:
+            line["paper_shape"] = {"error": repr(exc)}
     print(json.dumps(line))
     if dist is not None:
         dist.barrier()
