@@ -66,9 +66,11 @@ typedef enum {
 } moe_status;
 
 /* GEMM kernel variants.  AUTO: a DECODE context uses small-M; a PREFILL context chooses per step and pass from
- * the step's rows per expert R = T * top_k / n_experts (small-M up to R = 1024 for the gated pass, 384 for the
- * down pass; 256 and 128 with FP8 weights; large-M above) -- a function of T alone, so a step captured in a CUDA graph
- * replays the kernels it was captured with. */
+ * the step's rows per expert R = T * top_k / n_experts and the pass's K (hidden for the gated pass, inter for the
+ * down pass): small-M for every problem of up to 8192 rows; above that, the gated pass up to R = 1024 (with
+ * K < 4096 only from R = 448 on) and the down pass up to R = 320 when its K is at least 1536; with FP8 weights
+ * up to R = 256 and 128; large-M otherwise -- a function of T alone, so a step captured in a CUDA graph replays
+ * the kernels it was captured with. */
 typedef enum {
   MOE_GEMM_AUTO = 0,
   MOE_GEMM_LARGE_M = 1,  /* tokens fill the 128-row MMA dimension; for experts of many hundreds of rows,

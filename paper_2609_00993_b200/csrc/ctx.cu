@@ -289,28 +289,46 @@ int gemm_ctas(const moe_ctx* ctx) {
   return (ctx->cfg.sm_budget > 0 && ctx->cfg.sm_budget < ctx->n_sms) ? ctx->cfg.sm_budget : ctx->n_sms;
 }
 
-// Steps of up to this many rows per expert on average go to the small-M variant, per pass.  Measured on a B200
-// (DeepSeek-V3- and Qwen3-30B-shaped layers, uniform and Zipf routing): with tiles of up to 256 tokens the small-M
-// kernel moves fewer bytes through shared memory per flop than the large-M kernel (one CTA's MMA operands come
-// from shared memory, whose bandwidth is what both kernels end up waiting for).  The gated pass (long K on the
-// V3 shape, SwiGLU in the epilogue) is ahead with small-M by 5-13 % up to ~512 rows per expert and level with
-// large-M around 1024; the down pass (short K, so the exposed epilogue of its tiles of more than 128 tokens
-// weighs more) changes over near 384 rows per expert, the FP8 passes (half the operand bytes per flop, so the issue
-// cost of two MMAs per 16 K-elements shows) at 256 (gated) and 128 (down).
-constexpr int64_t kSmallMRowsGated = 1024, kSmallMRowsDown = 384, kSmallMRowsFp8Gated = 256, kSmallMRowsFp8Down = 128;
+// The choice between the two tensor-core variants for a PREFILL context, per pass, from the rows per expert
+// R = rows / experts and the pass's K.  Measured on a B200 with the variants interleaved in long blocks
+// (DeepSeek-V3- and Qwen3-30B-shaped layers, uniform and Zipf routing, whole steps and per-pass stage times):
+//  * with tiles of up to 256 tokens the small-M kernel moves fewer bytes through shared memory per flop than the
+//    large-M kernel (one CTA's MMA operands come from shared memory, whose bandwidth both end up waiting for), but
+//    its tiles of more than 128 tokens fill tensor memory, so their epilogue is exposed: the longer K is, the less
+//    that weighs;
+//  * gated pass: K = 7168 -- small-M ahead by 4-13 % at every R up to 1024; K = 2048 -- level or ahead from R = 448
+//    to 1024, behind by 3-10 % below that;
+//  * down pass: K = 2048 -- small-M ahead up to R ~ 320 and 10-17 % behind above; K = 768 (12 k-blocks per tile: an
+//    exposed epilogue is a quarter of a tile) -- behind by 9-25 % at every R;
+//  * problems of up to 8192 rows, whose launches overlap with their neighbours, are 1.5-6 % faster on the small-M
+//    kernel at any shape: it builds its tile list and fetches weights before the previous kernel has finished;
+//  * FP8 (half the operand bytes per flop, so the issue cost of two MMAs per 16 K-elements shows): small-M up to
+//    R = 256 (gated) and 128 (down).
+constexpr int64_t kSmallMRowsGated = 1024, kSmallMRowsGatedShortKFrom = 448, kSmallMRowsDown = 320;
+constexpr int64_t kSmallMRowsFp8Gated = 256, kSmallMRowsFp8Down = 128;
+constexpr int kLongK = 4096, kShortDownK = 1536;
 
-// AUTO: a DECODE context always streams; a PREFILL context chooses per launch from the rows per expert of the
-// problem (T * top_k rows over n_experts; T rows over one group for the shared expert by itself): the choice is
-// a function of T alone, so it is the same on every replay of a graph.
+// AUTO: a DECODE context always streams; a PREFILL context chooses per launch from the problem's rows (T * top_k
+// rows over n_experts; T rows over one group for the shared expert by itself) and K: the choice is a function of T
+// alone, so it is the same on every replay of a graph.
 int gemm_variant_of(const moe_ctx* ctx, const moe::GemmProblem& p) {
   const int v = ctx->cfg.gemm_variant;
   if (v != MOE_GEMM_AUTO) return v;
   if (ctx->cfg.phase == MOE_PHASE_DECODE) return MOE_GEMM_SMALL_M;
   if (ctx->cfg.row_gather == 1) return MOE_GEMM_LARGE_M;  // only the large-M kernel gathers its rows itself
   if (ctx->preemptible) return MOE_GEMM_SMALL_M;          // only the small-M kernel can stop between tiles
-  const int64_t limit = p.fp8 ? (p.gated ? kSmallMRowsFp8Gated : kSmallMRowsFp8Down)
-                              : (p.gated ? kSmallMRowsGated : kSmallMRowsDown);
-  return p.rows_bound <= limit * p.E ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M;  // p.E = 1 for a dense problem
+  const int64_t E = p.E;  // 1 for a dense problem
+  bool small;
+  if (p.fp8) {
+    small = p.rows_bound <= (p.gated ? kSmallMRowsFp8Gated : kSmallMRowsFp8Down) * E;
+  } else if (p.rows_bound <= moe::kGemmOverlapMaxRows) {
+    small = true;
+  } else if (p.gated) {
+    small = p.rows_bound <= kSmallMRowsGated * E && (p.K >= kLongK || p.rows_bound >= kSmallMRowsGatedShortKFrom * E);
+  } else {
+    small = p.K >= kShortDownK && p.rows_bound <= kSmallMRowsDown * E;
+  }
+  return small ? MOE_GEMM_SMALL_M : MOE_GEMM_LARGE_M;
 }
 
 // GEMM1 gathers its rows itself only on the large-M tensor-core variant.
