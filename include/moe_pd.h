@@ -69,7 +69,7 @@ typedef enum {
  * the step's rows per expert R = T * top_k / n_experts and the pass's K (hidden for the gated pass, inter for the
  * down pass): small-M for every problem of up to 8192 rows; above that, the gated pass up to R = 1024 (with
  * K < 4096 only from R = 448 on) and the down pass up to R = 320 when its K is at least 1536; with FP8 weights
- * up to R = 256 and 128; large-M otherwise -- a function of T alone, so a step captured in a CUDA graph replays
+ * up to R = 256 (K >= 4096) and 128 (K >= 1536); large-M otherwise -- a function of T alone, so a step captured in a CUDA graph replays
  * the kernels it was captured with. */
 typedef enum {
   MOE_GEMM_AUTO = 0,

@@ -303,7 +303,8 @@ int gemm_ctas(const moe_ctx* ctx) {
 //  * problems of up to 8192 rows, whose launches overlap with their neighbours, are 1.5-6 % faster on the small-M
 //    kernel at any shape: it builds its tile list and fetches weights before the previous kernel has finished;
 //  * FP8 (half the operand bytes per flop, so the issue cost of two MMAs per 16 K-elements shows): small-M up to
-//    R = 256 (gated) and 128 (down).
+//    R = 256 (gated, K >= 4096) and 128 (down, K >= 1536); with shorter K (half as many k-blocks per tile as bf16)
+//    large-M is 8-10 % ahead above the launch-overlap regime.
 constexpr int64_t kSmallMRowsGated = 1024, kSmallMRowsGatedShortKFrom = 448, kSmallMRowsDown = 320;
 constexpr int64_t kSmallMRowsFp8Gated = 256, kSmallMRowsFp8Down = 128;
 constexpr int kLongK = 4096, kShortDownK = 1536;
@@ -319,10 +320,10 @@ int gemm_variant_of(const moe_ctx* ctx, const moe::GemmProblem& p) {
   if (ctx->preemptible) return MOE_GEMM_SMALL_M;          // only the small-M kernel can stop between tiles
   const int64_t E = p.E;  // 1 for a dense problem
   bool small;
-  if (p.fp8) {
-    small = p.rows_bound <= (p.gated ? kSmallMRowsFp8Gated : kSmallMRowsFp8Down) * E;
-  } else if (p.rows_bound <= moe::kGemmOverlapMaxRows) {
+  if (p.rows_bound <= moe::kGemmOverlapMaxRows) {
     small = true;
+  } else if (p.fp8) {
+    small = p.K >= (p.gated ? kLongK : kShortDownK) && p.rows_bound <= (p.gated ? kSmallMRowsFp8Gated : kSmallMRowsFp8Down) * E;
   } else if (p.gated) {
     small = p.rows_bound <= kSmallMRowsGated * E && (p.K >= kLongK || p.rows_bound >= kSmallMRowsGatedShortKFrom * E);
   } else {
