@@ -42,7 +42,9 @@ inline cudaError_t launch_pdl(bool allow_overlap, void (*kern)(KArgs...), dim3 g
 }
 // The GEMM kernels take the overlap only for problems of up to this many rows: measured on a B200, a step of a
 // few hundred microseconds gains 7 % from it (six launch latencies and prologues hidden), while steps of several
-// milliseconds LOSE 1.5-5 % when their GEMM launches carry the attribute (the small kernels keep it at every size).
+// milliseconds LOSE 1.5-5 % when their GEMM launches carry the attribute (the small kernels keep it at every size;
+// re-measured in the sustained regime with the small-M kernel's early set-up: a limit of 32768 rows or none at all
+// changes nothing on the weight-streaming workloads and costs 3-6 % on the tensor-bound one).
 #ifndef MOE_GEMM_OVERLAP_MAX_ROWS
 #define MOE_GEMM_OVERLAP_MAX_ROWS 8192
 #endif
