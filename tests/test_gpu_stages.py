@@ -247,3 +247,29 @@ def test_combine_alone_matches_oracle():
     assert np.all(np.abs(got - ref) <= np.abs(ref) * 2 ** -8 + 1e-6)
     assert (got != rounded).mean() < 1e-2
     ctx.close()
+
+
+@pytest.mark.parametrize("phase", [B.MOE_PHASE_DECODE, B.MOE_PHASE_PREFILL])
+@pytest.mark.parametrize("T,H,E,k,I,shared_I", [
+    (300, 512, 16, 4, 192, 128),   # ragged tiles and a shared expert
+    (1100, 256, 3, 2, 128, 0),     # several token chunks per expert
+    (90, 320, 40, 8, 64, 0),       # many small experts, some empty
+])
+def test_the_result_does_not_depend_on_the_number_of_ctas(phase, T, H, E, k, I, shared_I):
+    """The small-M kernel deals the first waves of its tile list statically and hands the rest out through an atomic
+    counter; whatever the grid -- one CTA, a few, all -- every tile is computed exactly once and the layer's bits
+    are the same."""
+    shape = wl.LayerShape("t", T=T, H=H, E=E, k=k, I=I, shared_I=shared_I, select_bias=True)
+    w, a = wl.make_weights(shape, 21, DEV), wl.make_activations(shape, 22, DEV)
+    outs = {}
+    for budget in (0, 1, 2, 5, 37):
+        ctx = _ctx(H=H, E=E, k=k, I=I, shared_I=shared_I, max_tokens=T, phase=phase, variant=B.MOE_GEMM_SMALL_M,
+                   sm_budget=budget)
+        for rep in range(2):  # twice: the second step finds the counters the first one left
+            out, _ = ctx.layer(a["x"], a["logits"], a["bias"], w["w_gate_up"], w["w_down"], w["ws_gate_up"], w["ws_down"])
+        torch.cuda.synchronize()
+        assert ctx.moe_ctx_status() == B.MOE_OK
+        outs[budget] = out.clone()
+        ctx.close()
+    for budget, out in outs.items():
+        assert torch.equal(out, outs[0]), f"sm_budget = {budget} changes the result"
